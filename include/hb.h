@@ -1,0 +1,240 @@
+/*
+ * hb.h -- C ABI of the heterogeneous-batching step library (B200 / sm_100a).
+ *
+ * One call, hb_mixed_step, runs ONE transformer forward over a ragged mixed
+ * batch: the "forward" stage of the paper's inference loop (Algorithm 1) over
+ * the batch unit of Section 3.2 (embedding chunks, generation prefill chunks,
+ * decode tokens), followed by the two output paths of Algorithm 1: the
+ * incremental pooler of Section 3.3 (Eq. 1-2 and the last-token head) on the
+ * embedding rows and the logits for the sampler on the generation rows.
+ *
+ * Conventions
+ *  - every function returns an int status: HB_OK (0) or a negative HB_ERR_*;
+ *    nothing throws or aborts across this boundary;
+ *  - "host" / "device" is stated for every pointer; device pointers are plain
+ *    CUDA device addresses on the current device; `stream` is a cudaStream_t
+ *    passed as void* (NULL = the legacy default stream);
+ *  - the library never frees caller memory; hb_mixed_step allocates nothing;
+ *  - all work is enqueued on `stream`; outputs are valid once the caller has
+ *    synchronised that stream;
+ *  - there is no CPU path: without a CUDA device every compute call fails.
+ */
+#ifndef HB_H_
+#define HB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HB_API __attribute__((visibility("default")))
+#else
+#define HB_API
+#endif
+
+/* ---- status codes ------------------------------------------------------- */
+enum {
+  HB_OK = 0,
+  HB_ERR_BAD_ARG = -1,       /* null pointer, bad size, double free ...        */
+  HB_ERR_CUDA = -2,          /* a CUDA runtime/driver call failed              */
+  HB_ERR_OOM_PAGES = -3,     /* hb_kv_alloc_pages: not enough free pages       */
+  HB_ERR_OOM_SLOTS = -4,     /* hb_pool_alloc_slot: no free slot               */
+  HB_ERR_TOO_LARGE = -5,     /* batch exceeds the limits given to hb_create    */
+  HB_ERR_BAD_DESC = -6,      /* batch descriptor failed validation             */
+  HB_ERR_DEVICE_STATUS = -7, /* a kernel reported a bounded-wait expiry/index  */
+  HB_ERR_UNSUPPORTED = -8    /* model shape outside what the kernels cover     */
+};
+
+/* Row kinds of the batch unit (Section 3.2).  Rows of one kind are contiguous
+ * and kinds appear in this order (the scheduler "outputs batches sorted by
+ * request type"). */
+enum { HB_KIND_DECODE = 0, HB_KIND_PREFILL_CHUNK = 1, HB_KIND_EMBED_CHUNK = 2 };
+
+/* Pooling heads (Section 3.3): additive mean (Eq. 1-2 with w = 1) and the
+ * positional last-token head. */
+enum { HB_POOL_NONE = 0, HB_POOL_MEAN = 1, HB_POOL_LAST = 2 };
+
+typedef struct hb_ctx hb_ctx;
+typedef struct hb_kv hb_kv;
+typedef struct hb_pool hb_pool;
+
+/* Decoder-only model: pre-norm RMSNorm, rotate-half RoPE, grouped-query causal
+ * attention, SwiGLU FFN, no biases, untied LM head.  head_dim must be 64 or
+ * 128; d_model, n_heads*head_dim, d_ffn multiples of 64; page_size 16. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t page_size;    /* tokens per KV page (16)                              */
+  int32_t max_pos;      /* largest position + 1 any request may reach          */
+  float rope_theta;
+  float rms_eps;
+} hb_model_cfg;
+
+/* All weights are bf16, row-major [out, in] (y = x * W^T), device memory owned
+ * by the caller.
+ *   wqkv      [(n_heads + 2 n_kv_heads) * head_dim, d_model]: q rows, then k, then v
+ *   wo        [d_model, n_heads * head_dim]
+ *   w_gate_up [2 * d_ffn, d_model]: row 2j = gate row j, row 2j+1 = up row j
+ *   w_down    [d_model, d_ffn]
+ *   attn_norm, ffn_norm, final_norm [d_model] gains
+ *   tok_emb, lm_head [vocab, d_model] */
+typedef struct {
+  const void* attn_norm;
+  const void* wqkv;
+  const void* wo;
+  const void* ffn_norm;
+  const void* w_gate_up;
+  const void* w_down;
+} hb_layer_weights;
+
+typedef struct {
+  const void* tok_emb;               /* device */
+  const hb_layer_weights* layers;    /* HOST array [n_layers] of device ptrs   */
+  const void* final_norm;            /* device */
+  const void* lm_head;               /* device */
+} hb_weights;
+
+/* One segment = the rows one request contributes to this step (Section 3.2).
+ *   kind        HB_KIND_*
+ *   q_start     first token row of the segment (prefix sum of q_len)
+ *   q_len       rows: 1 for DECODE, chunk size c_k otherwise (>= 1)
+ *   pos_start   tokens of this request already in the KV cache; row j has
+ *               position pos_start + j, writes its K/V there and attends to
+ *               positions 0 .. pos_start + j of its own request
+ *   pt_start    offset of this request's page list inside page_ids
+ *   pt_len      entries of that list; must cover pos_start + q_len tokens
+ *   pool_slot   pool slot (EMBED_CHUNK) or -1
+ *   pool_mode   HB_POOL_* (NONE unless EMBED_CHUNK)
+ *   is_final    last chunk of the request: emit embedding / logits
+ *   logits_row  row of out_logits to write (DECODE, final PREFILL_CHUNK), else -1
+ *   emb_row     row of out_emb to write (final EMBED_CHUNK), else -1 */
+typedef struct {
+  int32_t kind, q_start, q_len, pos_start;
+  int32_t pt_start, pt_len, pool_slot, pool_mode;
+  int32_t is_final, logits_row, emb_row, reserved;
+} hb_seg;
+
+/* Batch descriptor; every pointer is HOST memory, read during the call only. */
+typedef struct {
+  int32_t n_tokens;       /* total rows T                                       */
+  int32_t n_segs;         /* segments R                                         */
+  int32_t n_page_ids;     /* length of page_ids                                 */
+  int32_t n_logit_rows;   /* rows of out_logits produced this step              */
+  int32_t n_emb_rows;     /* rows of out_emb produced this step                 */
+  const int32_t* token_ids; /* [n_tokens] ids in [0, vocab)                     */
+  const hb_seg* segs;       /* [n_segs]                                         */
+  const int32_t* page_ids;  /* [n_page_ids] physical page numbers               */
+} hb_batch_desc;
+
+/* ---- context -------------------------------------------------------------- */
+
+/* Bytes of device workspace a context needs for steps of at most max_tokens
+ * rows, max_segs segments and max_page_ids page-list entries.  Host only. */
+HB_API int hb_workspace_bytes(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs,
+                       int32_t max_page_ids, size_t* out_bytes);
+
+/* Create a context on the current device.  `workspace` (device, 256-byte
+ * aligned, hb_workspace_bytes big) stays owned by the caller; pass NULL to let
+ * the library allocate (and later free) it.  Builds the rotary table and the
+ * activation tensor maps.  Synchronises the device once. */
+HB_API int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs,
+              int32_t max_page_ids, void* workspace, size_t workspace_bytes,
+              hb_ctx** out);
+HB_API int hb_destroy(hb_ctx* ctx);
+
+/* ---- paged KV cache ------------------------------------------------------- */
+
+/* Bytes of one page across all layers, and of an arena of n_pages.  Arena
+ * layout (bf16): [layer][page][K|V][kv_head][slot 0..page_size)[head_dim], so
+ * the K (or V) rows of one (layer, page, head) are contiguous.  Host only. */
+HB_API int hb_kv_arena_bytes(const hb_model_cfg* cfg, int32_t n_pages, size_t* out_bytes);
+
+/* Wrap a caller-owned device arena.  Only the free list lives in the library
+ * (host memory); no device work.  `arena` may be NULL for host-side
+ * bookkeeping tests. */
+HB_API int hb_kv_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32_t n_pages,
+                 hb_kv** out);
+HB_API int hb_kv_destroy(hb_kv* kv);
+/* Take n pages (lowest free ids first); all-or-nothing: HB_ERR_OOM_PAGES. */
+HB_API int hb_kv_alloc_pages(hb_kv* kv, int32_t n, int32_t* out_ids /* host [n] */);
+/* Return pages; a page not currently allocated -> HB_ERR_BAD_ARG, nothing freed. */
+HB_API int hb_kv_free_pages(hb_kv* kv, int32_t n, const int32_t* ids /* host [n] */);
+HB_API int hb_kv_free_count(const hb_kv* kv, int32_t* out_free);
+
+/* ---- pooling state (Section 3.3: O(d) state per request) ------------------ */
+
+/* Arena layout: float sum[n_slots][d_model], then uint32 meta[n_slots][4] =
+ * {count, chunks, mode, state}; state 0 = open, 1 = emitted.  Host only. */
+HB_API int hb_pool_arena_bytes(const hb_model_cfg* cfg, int32_t n_slots, size_t* out_bytes);
+HB_API int hb_pool_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32_t n_slots,
+                   hb_pool** out);
+HB_API int hb_pool_destroy(hb_pool* pool);
+/* Take a slot (lowest free id).  No device work: the first chunk of a request
+ * (pos_start == 0) overwrites the slot, which realises S(0) = 0, W(0) = 0. */
+HB_API int hb_pool_alloc_slot(hb_pool* pool, int32_t* out_slot);
+HB_API int hb_pool_free_slot(hb_pool* pool, int32_t slot);
+
+/* ---- the step ------------------------------------------------------------- */
+
+/* Host-only validation of a descriptor against the limits (what hb_mixed_step
+ * checks before it enqueues anything): sizes, kind order, q_start prefix sums,
+ * page lists cover pos_start + q_len, page ids in [0, n_pages), a page written
+ * this step belongs to one segment only, pool slots in range and used once,
+ * output rows in range and used once, token ids in range. */
+HB_API int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs,
+                     int32_t max_page_ids, int32_t n_pages, int32_t n_slots,
+                     const hb_batch_desc* desc);
+
+/* One forward step over the mixed batch (Algorithm 1: Forward, IncPooler,
+ * and the logits the Sampler consumes).
+ *   desc        host descriptor (copied; may be reused after return)
+ *   w           host struct of device weight pointers
+ *   kv, pool    caches created above; K/V of every row is appended to its
+ *               page; pool slots of EMBED_CHUNK segments are updated
+ *   out_logits  device float [>= n_logit_rows, vocab]; row seg.logits_row gets
+ *               the logits of the segment's last row
+ *   out_emb     device float [>= n_emb_rows, d_model]; row seg.emb_row gets the
+ *               L2-normalised embedding of a request whose final chunk ran
+ * Rows of the outputs not named by a segment are left untouched.  Returns
+ * after enqueueing; no synchronisation, no allocation.  A failed validation
+ * enqueues nothing. */
+HB_API int hb_mixed_step(hb_ctx* ctx, const hb_batch_desc* desc, const hb_weights* w, hb_kv* kv,
+                  hb_pool* pool, float* out_logits, float* out_emb, void* stream);
+
+/* Greedy sampler over logits rows (Algorithm 1 "Sampler", greedy case): lowest
+ * index of the maximum of each row.  logits device float [n_rows, vocab],
+ * out_tokens device int32 [n_rows]. */
+HB_API int hb_argmax(hb_ctx* ctx, const float* logits, int32_t n_rows, int32_t* out_tokens,
+              void* stream);
+
+/* Read (and clear) the device status word; synchronises `stream`.  0 = clean.
+ * Non-zero: a bounded wait inside a kernel expired or an index check failed;
+ * *out_code holds the kernel-specific code.  Returns HB_ERR_DEVICE_STATUS then. */
+HB_API int hb_status_poll(hb_ctx* ctx, void* stream, uint32_t* out_code);
+
+/* Kernels launched by the last hb_mixed_step on this context. */
+HB_API int hb_last_launch_count(const hb_ctx* ctx, int32_t* out_count);
+
+/* ---- kernel-level entry points (used by the parity tests) ----------------- */
+
+/* Epilogues of the projection GEMM (the dense contractions of the forward,
+ * Section 3.1 "attention and feed-forward layers"). */
+enum {
+  HB_EPI_BF16 = 0,      /* C bf16 [M,N] = A * B^T                               */
+  HB_EPI_F32 = 1,       /* C float [M,N] = A * B^T                              */
+  HB_EPI_RESID_F32 = 2, /* C float [M,N] += A * B^T (residual stream update)    */
+  HB_EPI_SWIGLU = 3     /* C bf16 [M,N/2]: silu(acc[2j]) * acc[2j+1]            */
+};
+
+/* C = epilogue(A * B^T): A bf16 [M,K] row-major, B bf16 [N,K] row-major (both
+ * K-major), fp32 accumulation on the tcgen05 tensor cores.  All device
+ * pointers, 16-byte aligned; K and N multiples of 8.  M may be any value >= 1. */
+HB_API int hb_gemm(hb_ctx* ctx, const void* A, const void* B, void* C, int32_t M, int32_t N,
+            int32_t K, int32_t epilogue, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HB_H_ */

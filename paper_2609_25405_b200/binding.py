@@ -1,0 +1,356 @@
+"""ctypes binding of libhb.so: argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels; torch is used
+here for device memory and streams.  Importing this module loads the library
+and raises if it has not been built -- there is no fallback of any kind.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhb.so")
+
+HB_OK = 0
+ERRORS = {0: "HB_OK", -1: "HB_ERR_BAD_ARG", -2: "HB_ERR_CUDA", -3: "HB_ERR_OOM_PAGES",
+          -4: "HB_ERR_OOM_SLOTS", -5: "HB_ERR_TOO_LARGE", -6: "HB_ERR_BAD_DESC",
+          -7: "HB_ERR_DEVICE_STATUS", -8: "HB_ERR_UNSUPPORTED"}
+KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK = 0, 1, 2
+POOL_NONE, POOL_MEAN, POOL_LAST = 0, 1, 2
+EPI_BF16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU = 0, 1, 2, 3
+
+
+class HbError(RuntimeError):
+    def __init__(self, code, what):
+        super().__init__(f"{what}: {ERRORS.get(code, code)}")
+        self.code = code
+
+
+class ModelCfg(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ffn", C.c_int32),
+                ("vocab", C.c_int32), ("page_size", C.c_int32), ("max_pos", C.c_int32),
+                ("rope_theta", C.c_float), ("rms_eps", C.c_float)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")]
+
+
+class Weights(C.Structure):
+    _fields_ = [("tok_emb", C.c_void_p), ("layers", C.POINTER(LayerWeights)),
+                ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)]
+
+
+class Seg(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("kind", "q_start", "q_len", "pos_start", "pt_start", "pt_len",
+                                         "pool_slot", "pool_mode", "is_final", "logits_row", "emb_row",
+                                         "reserved")]
+
+
+class BatchDesc(C.Structure):
+    _fields_ = [("n_tokens", C.c_int32), ("n_segs", C.c_int32), ("n_page_ids", C.c_int32),
+                ("n_logit_rows", C.c_int32), ("n_emb_rows", C.c_int32),
+                ("token_ids", C.POINTER(C.c_int32)), ("segs", C.POINTER(Seg)),
+                ("page_ids", C.POINTER(C.c_int32))]
+
+
+SEG_DTYPE = np.dtype([(n, np.int32) for n, _ in Seg._fields_])
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_25405_b200.build` "
+                      "(there is no CPU fallback)")
+lib = C.CDLL(LIB_PATH)
+
+_P = C.c_void_p
+_sig = {
+    "hb_workspace_bytes": [C.POINTER(ModelCfg), C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)],
+    "hb_create": [C.POINTER(ModelCfg), C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, C.POINTER(_P)],
+    "hb_destroy": [_P],
+    "hb_kv_arena_bytes": [C.POINTER(ModelCfg), C.c_int32, C.POINTER(C.c_size_t)],
+    "hb_kv_create": [C.POINTER(ModelCfg), _P, C.c_size_t, C.c_int32, C.POINTER(_P)],
+    "hb_kv_destroy": [_P],
+    "hb_kv_alloc_pages": [_P, C.c_int32, C.POINTER(C.c_int32)],
+    "hb_kv_free_pages": [_P, C.c_int32, C.POINTER(C.c_int32)],
+    "hb_kv_free_count": [_P, C.POINTER(C.c_int32)],
+    "hb_pool_arena_bytes": [C.POINTER(ModelCfg), C.c_int32, C.POINTER(C.c_size_t)],
+    "hb_pool_create": [C.POINTER(ModelCfg), _P, C.c_size_t, C.c_int32, C.POINTER(_P)],
+    "hb_pool_destroy": [_P],
+    "hb_pool_alloc_slot": [_P, C.POINTER(C.c_int32)],
+    "hb_pool_free_slot": [_P, C.c_int32],
+    "hb_validate_desc": [C.POINTER(ModelCfg), C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                         C.POINTER(BatchDesc)],
+    "hb_mixed_step": [_P, C.POINTER(BatchDesc), C.POINTER(Weights), _P, _P, _P, _P, _P],
+    "hb_argmax": [_P, _P, C.c_int32, _P, _P],
+    "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
+    "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
+    "hb_gemm": [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
+}
+for _name, _args in _sig.items():
+    _f = getattr(lib, _name)
+    _f.argtypes = _args
+    _f.restype = C.c_int
+EXPORTS = tuple(_sig)
+
+
+def check(code, what):
+    if code != HB_OK:
+        raise HbError(code, what)
+
+
+def model_cfg(shape, max_pos):
+    """hb_model_cfg from a synth.ModelShape-like object."""
+    return ModelCfg(shape.L, shape.d, shape.Hq, shape.Hkv, shape.Dh, shape.F, shape.V,
+                    shape.page_size, int(max_pos), float(shape.rope_theta), float(shape.rms_eps))
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def bf16_from_f32(a, device="cuda"):
+    """numpy float32 (bf16-exact values) -> torch bf16 tensor on `device`, bit-exact."""
+    bits = (np.ascontiguousarray(a, dtype=np.float32).view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+    return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+
+
+class DeviceWeights:
+    """Weights resident in HBM in the library's layout, plus the hb_weights struct."""
+
+    def __init__(self, n_layers):
+        self.tensors = []          # keep-alive
+        self.layers = (LayerWeights * n_layers)()
+        self.struct = Weights()
+        self.struct.layers = C.cast(self.layers, C.POINTER(LayerWeights))
+
+    def _keep(self, t):
+        self.tensors.append(t)
+        return t.data_ptr()
+
+    @classmethod
+    def from_synth(cls, W, device="cuda"):
+        """Upload synth.Weights: q/k/v rows are concatenated, gate/up rows interleaved."""
+        s = W.shape
+        self = cls(s.L)
+        up = lambda a: self._keep(bf16_from_f32(a, device))
+        self.struct.tok_emb = up(W.tok_emb)
+        self.struct.lm_head = up(W.lm_head)
+        self.struct.final_norm = up(W.final_norm)
+        for l in range(s.L):
+            w = W.layer(l)
+            lw = self.layers[l]
+            lw.attn_norm = up(w["attn_norm"])
+            lw.ffn_norm = up(w["ffn_norm"])
+            lw.wqkv = up(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0))
+            lw.wo = up(w["wo"])
+            gu = np.empty((2 * s.F, s.d), dtype=np.float32)
+            gu[0::2] = w["wg"]
+            gu[1::2] = w["wu"]
+            lw.w_gate_up = up(gu)
+            lw.w_down = up(w["wd"])
+        return self
+
+    @classmethod
+    def random_on_device(cls, shape, seed=0, std=0.02, device="cuda"):
+        """N(0, std^2) bf16 weights drawn on the device (benchmarks; not bit-matched to the
+        host generator)."""
+        self = cls(shape.L)
+        g = torch.Generator(device=device)
+        g.manual_seed(seed)
+
+        def rnd(r, c):
+            t = torch.empty((r, c), dtype=torch.bfloat16, device=device)
+            t.normal_(0.0, std, generator=g)
+            return self._keep(t)
+
+        ones = lambda: self._keep(torch.ones(shape.d, dtype=torch.bfloat16, device=device))
+        self.struct.tok_emb = rnd(shape.V, shape.d)
+        self.struct.lm_head = rnd(shape.V, shape.d)
+        self.struct.final_norm = ones()
+        for l in range(shape.L):
+            lw = self.layers[l]
+            lw.attn_norm = ones()
+            lw.ffn_norm = ones()
+            lw.wqkv = rnd(shape.n_qkv, shape.d)
+            lw.wo = rnd(shape.d, shape.Hq * shape.Dh)
+            lw.w_gate_up = rnd(2 * shape.F, shape.d)
+            lw.w_down = rnd(shape.d, shape.F)
+        return self
+
+
+class KvCache:
+    """Caller-owned KV arena (torch) + the library's page free list."""
+
+    def __init__(self, cfg, n_pages, device="cuda", fill=None):
+        self.cfg = cfg
+        self.n_pages = n_pages
+        nbytes = C.c_size_t()
+        check(lib.hb_kv_arena_bytes(C.byref(cfg), n_pages, C.byref(nbytes)), "hb_kv_arena_bytes")
+        self.handle = C.c_void_p()
+        if device is None:      # bookkeeping only (host tests): no arena
+            self.arena = None
+            check(lib.hb_kv_create(C.byref(cfg), None, 0, n_pages, C.byref(self.handle)), "hb_kv_create")
+            return
+        self.arena = torch.empty(nbytes.value // 2, dtype=torch.int16, device=device)
+        if fill is not None:
+            self.arena.fill_(fill)
+        check(lib.hb_kv_create(C.byref(cfg), C.c_void_p(self.arena.data_ptr()), nbytes.value, n_pages,
+                               C.byref(self.handle)), "hb_kv_create")
+
+    def view(self):
+        """bf16 view [L, page, 2, Hkv, P, Dh]."""
+        c = self.cfg
+        return self.arena.view(torch.bfloat16).view(c.n_layers, self.n_pages, 2, c.n_kv_heads,
+                                                    c.page_size, c.head_dim)
+
+    def alloc(self, n):
+        ids = (C.c_int32 * max(n, 1))()
+        check(lib.hb_kv_alloc_pages(self.handle, n, ids), "hb_kv_alloc_pages")
+        return list(ids[:n])
+
+    def free(self, ids):
+        arr = (C.c_int32 * max(len(ids), 1))(*ids)
+        check(lib.hb_kv_free_pages(self.handle, len(ids), arr), "hb_kv_free_pages")
+
+    def free_count(self):
+        n = C.c_int32()
+        check(lib.hb_kv_free_count(self.handle, C.byref(n)), "hb_kv_free_count")
+        return n.value
+
+    def close(self):
+        if self.handle:
+            lib.hb_kv_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Pool:
+    """Caller-owned pooling arena (torch) + the library's slot free list."""
+
+    def __init__(self, cfg, n_slots, device="cuda", fill=None):
+        self.cfg = cfg
+        self.n_slots = n_slots
+        nbytes = C.c_size_t()
+        check(lib.hb_pool_arena_bytes(C.byref(cfg), n_slots, C.byref(nbytes)), "hb_pool_arena_bytes")
+        self.handle = C.c_void_p()
+        if device is None:      # bookkeeping only (host tests): no arena
+            self.arena = None
+            check(lib.hb_pool_create(C.byref(cfg), None, 0, n_slots, C.byref(self.handle)), "hb_pool_create")
+            return
+        self.arena = torch.empty((nbytes.value + 3) // 4, dtype=torch.int32, device=device)
+        if fill is not None:
+            self.arena.fill_(fill)
+        check(lib.hb_pool_create(C.byref(cfg), C.c_void_p(self.arena.data_ptr()), nbytes.value, n_slots,
+                                 C.byref(self.handle)), "hb_pool_create")
+
+    def sums(self):
+        d = self.cfg.d_model
+        return self.arena[: self.n_slots * d].view(torch.float32).view(self.n_slots, d)
+
+    def meta(self):
+        d = self.cfg.d_model
+        return self.arena[self.n_slots * d: self.n_slots * d + self.n_slots * 4].view(self.n_slots, 4)
+
+    def alloc(self):
+        s = C.c_int32()
+        check(lib.hb_pool_alloc_slot(self.handle, C.byref(s)), "hb_pool_alloc_slot")
+        return s.value
+
+    def free(self, slot):
+        check(lib.hb_pool_free_slot(self.handle, slot), "hb_pool_free_slot")
+
+    def close(self):
+        if self.handle:
+            lib.hb_pool_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Batch:
+    """Host descriptor arrays (numpy, kept alive) and the hb_batch_desc over them."""
+
+    def __init__(self, token_ids, segs, page_ids, n_logit_rows, n_emb_rows):
+        self.token_ids = np.ascontiguousarray(token_ids, dtype=np.int32)
+        self.segs = np.ascontiguousarray(segs, dtype=SEG_DTYPE)
+        self.page_ids = np.ascontiguousarray(page_ids, dtype=np.int32)
+        self.desc = BatchDesc(len(self.token_ids), len(self.segs), len(self.page_ids), n_logit_rows,
+                              n_emb_rows,
+                              self.token_ids.ctypes.data_as(C.POINTER(C.c_int32)),
+                              self.segs.ctypes.data_as(C.POINTER(Seg)),
+                              self.page_ids.ctypes.data_as(C.POINTER(C.c_int32)))
+
+    @property
+    def n_tokens(self):
+        return len(self.token_ids)
+
+    def host_bytes(self):
+        return self.token_ids.nbytes + self.segs.nbytes + self.page_ids.nbytes
+
+
+class Context:
+    def __init__(self, cfg, max_tokens, max_segs, max_page_ids):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libhb needs a CUDA device (B200); there is no CPU path")
+        self.cfg = cfg
+        self.handle = C.c_void_p()
+        check(lib.hb_create(C.byref(cfg), max_tokens, max_segs, max_page_ids, None, 0, C.byref(self.handle)),
+              "hb_create")
+
+    def mixed_step(self, batch, weights, kv, pool, out_logits, out_emb, stream=None):
+        check(lib.hb_mixed_step(self.handle, C.byref(batch.desc), C.byref(weights.struct), kv.handle,
+                                pool.handle if pool is not None else None,
+                                C.c_void_p(out_logits.data_ptr()) if out_logits is not None else None,
+                                C.c_void_p(out_emb.data_ptr()) if out_emb is not None else None,
+                                _stream_ptr(stream)), "hb_mixed_step")
+
+    def argmax(self, logits, n_rows, out_tokens, stream=None):
+        check(lib.hb_argmax(self.handle, C.c_void_p(logits.data_ptr()), n_rows,
+                            C.c_void_p(out_tokens.data_ptr()), _stream_ptr(stream)), "hb_argmax")
+
+    def gemm(self, A, B, Cout, M, N, K, epilogue, stream=None):
+        check(lib.hb_gemm(self.handle, C.c_void_p(A.data_ptr()), C.c_void_p(B.data_ptr()),
+                          C.c_void_p(Cout.data_ptr()), M, N, K, epilogue, _stream_ptr(stream)), "hb_gemm")
+
+    def status_poll(self, stream=None):
+        """Synchronises the stream; returns the device status code (0 = clean)."""
+        code = C.c_uint32()
+        rc = lib.hb_status_poll(self.handle, _stream_ptr(stream), C.byref(code))
+        if rc not in (HB_OK, -7):
+            raise HbError(rc, "hb_status_poll")
+        return code.value
+
+    def last_launch_count(self):
+        n = C.c_int32()
+        check(lib.hb_last_launch_count(self.handle, C.byref(n)), "hb_last_launch_count")
+        return n.value
+
+    def close(self):
+        if self.handle:
+            lib.hb_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def validate_desc(cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, batch):
+    """Host-only descriptor validation; returns the status code."""
+    return lib.hb_validate_desc(C.byref(cfg), max_tokens, max_segs, max_page_ids, n_pages, n_slots,
+                                C.byref(batch.desc))

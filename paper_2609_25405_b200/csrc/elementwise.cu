@@ -1,0 +1,373 @@
+// Memory-bound stages of the mixed step: token gather + RMSNorm, RMSNorm, rotary + KV-page
+// append, final RMSNorm fused with the incremental pooler (Section 3.3, Eq. 1-2 and the
+// last-token head) and with the hi/lo split that feeds the LM head, greedy argmax.
+// All global accesses are 16-byte vectors; row statistics use warp shuffles; sums run in a
+// fixed order (no floating-point atomics), so results do not depend on what else is batched.
+#include "hb_internal.h"
+
+namespace {
+
+constexpr int NORM_THREADS = 256;
+constexpr int MAX_VEC = 8;  // float4 per thread held in registers: d_model <= 256 * 4 * 8 = 8192
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over the block; every thread gets the result.  red must hold 32 floats.
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  v = warp_sum(v);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = (lane < (blockDim.x >> 5)) ? red[lane] : 0.0f;
+  t = warp_sum(t);
+  return t;
+}
+
+__device__ __forceinline__ void bf16x4_to_float4(uint2 raw, float4& o) {
+  const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+  const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+  o = make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+
+__device__ __forceinline__ uint2 float4_to_bf16x4(float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 r;
+  r.x = *reinterpret_cast<uint32_t*>(&a);
+  r.y = *reinterpret_cast<uint32_t*>(&b);
+  return r;
+}
+
+// x[t,:] = E[tok[t],:] (kept in fp32 as the residual stream); h[t,:] = bf16(rmsnorm(x) * gain).
+// GATHER = false: x is read instead.
+template <bool GATHER>
+__global__ void __launch_bounds__(NORM_THREADS)
+norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E,
+            const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __nv_bfloat16* __restrict__ h,
+            int d, float eps) {
+  __shared__ float red[32];
+  const int t = blockIdx.x;
+  const int nv = d >> 2;
+  float4 buf[MAX_VEC];
+  float ss = 0.0f;
+  float* xrow = x + static_cast<size_t>(t) * d;
+  const __nv_bfloat16* erow = GATHER ? E + static_cast<size_t>(tok[t]) * d : nullptr;
+#pragma unroll
+  for (int i = 0; i < MAX_VEC; ++i) {
+    const int v = threadIdx.x + i * NORM_THREADS;
+    if (v < nv) {
+      if (GATHER) {
+        bf16x4_to_float4(*reinterpret_cast<const uint2*>(erow + 4 * v), buf[i]);
+        *reinterpret_cast<float4*>(xrow + 4 * v) = buf[i];
+      } else {
+        buf[i] = *reinterpret_cast<const float4*>(xrow + 4 * v);
+      }
+      ss += buf[i].x * buf[i].x + buf[i].y * buf[i].y + buf[i].z * buf[i].z + buf[i].w * buf[i].w;
+    }
+  }
+  const float tot = block_sum(ss, red);
+  const float rstd = rsqrtf(tot / static_cast<float>(d) + eps);
+  __nv_bfloat16* hrow = h + static_cast<size_t>(t) * d;
+#pragma unroll
+  for (int i = 0; i < MAX_VEC; ++i) {
+    const int v = threadIdx.x + i * NORM_THREADS;
+    if (v < nv) {
+      float4 g;
+      bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
+      float4 o = make_float4(buf[i].x * rstd * g.x, buf[i].y * rstd * g.y, buf[i].z * rstd * g.z,
+                             buf[i].w * rstd * g.w);
+      *reinterpret_cast<uint2*>(hrow + 4 * v) = float4_to_bf16x4(o);
+    }
+  }
+}
+
+// Rotary embedding of q and k (rotate-half pairing: element i pairs with i + Dh/2, angle
+// pos * theta^(-2i/Dh) from a host-built table) and append of k, v to the request's KV page:
+// position pos lives in page pages[pt_start + pos / P], slot pos % P.
+__global__ void __launch_bounds__(256)
+rope_append_kernel(const float* __restrict__ qkv, __nv_bfloat16* __restrict__ q_out, KvGeom kv, int layer,
+                   const int32_t* __restrict__ row_seg, const int32_t* __restrict__ row_pos,
+                   const hb_seg* __restrict__ segs, const int32_t* __restrict__ pages,
+                   const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int Hq, int max_pos,
+                   uint32_t* status) {
+  const int t = blockIdx.x;
+  const int Dh = kv.Dh, Hkv = kv.Hkv, half = Dh >> 1;
+  const int pos = row_pos[t];
+  const hb_seg sg = segs[row_seg[t]];
+  const int blk = pos / kv.P, slot = pos - blk * kv.P;
+  int page = (blk < sg.pt_len) ? pages[sg.pt_start + blk] : -1;
+  if (page < 0 || page >= kv.n_pages || pos >= max_pos) {
+    if (threadIdx.x == 0) atomicOr(status, HB_DEV_APPEND_BAD_INDEX);
+    return;  // skip the access
+  }
+  const int n_qkv = (Hq + 2 * Hkv) * Dh;
+  const float* row = qkv + static_cast<size_t>(t) * n_qkv;
+  __nv_bfloat16* kbase = kv.arena + layer * kv.layer_stride + page * kv.page_stride + slot * Dh;
+  const int64_t head_stride = static_cast<int64_t>(kv.P) * Dh;
+  const float* cs = rope_cos + static_cast<size_t>(pos) * half;
+  const float* sn = rope_sin + static_cast<size_t>(pos) * half;
+  const int units_per_head = half >> 2;                 // 4 pairs per unit
+  const int rot_units = (Hq + Hkv) * units_per_head;
+  const int v_units = Hkv * (Dh >> 2);                  // 4 elements per unit
+  for (int u = threadIdx.x; u < rot_units + v_units; u += blockDim.x) {
+    if (u < rot_units) {
+      const int head = u / units_per_head, i = (u - head * units_per_head) << 2;
+      const float* src = row + head * Dh + i;
+      const float4 a = *reinterpret_cast<const float4*>(src);
+      const float4 b = *reinterpret_cast<const float4*>(src + half);
+      const float4 c = *reinterpret_cast<const float4*>(cs + i);
+      const float4 s = *reinterpret_cast<const float4*>(sn + i);
+      const float4 lo = make_float4(a.x * c.x - b.x * s.x, a.y * c.y - b.y * s.y, a.z * c.z - b.z * s.z,
+                                    a.w * c.w - b.w * s.w);
+      const float4 hi = make_float4(b.x * c.x + a.x * s.x, b.y * c.y + a.y * s.y, b.z * c.z + a.z * s.z,
+                                    b.w * c.w + a.w * s.w);
+      __nv_bfloat16* dst = (head < Hq) ? q_out + static_cast<size_t>(t) * Hq * Dh + head * Dh + i
+                                       : kbase + (head - Hq) * head_stride + i;
+      *reinterpret_cast<uint2*>(dst) = float4_to_bf16x4(lo);
+      *reinterpret_cast<uint2*>(dst + half) = float4_to_bf16x4(hi);
+    } else {
+      const int w = u - rot_units;
+      const int head = w / (Dh >> 2), i = (w - head * (Dh >> 2)) << 2;
+      const float4 a = *reinterpret_cast<const float4*>(row + (Hq + Hkv + head) * Dh + i);
+      __nv_bfloat16* dst = kbase + (Hkv + head) * head_stride + i;
+      *reinterpret_cast<uint2*>(dst) = float4_to_bf16x4(a);
+    }
+  }
+}
+
+// Final RMSNorm of the rows that feed the LM head, written as a (hi, lo) bf16 pair:
+// hi = bf16(y), lo = bf16(y - hi), interleaved in blocks of 64 columns
+// ([hi 0..63 | lo 0..63 | hi 64..127 | ...]).  The LM-head GEMM runs over 2d columns with each
+// weight k-block used twice, which restores near-fp32 input precision for the logits.
+__global__ void __launch_bounds__(NORM_THREADS)
+final_logit_rows_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
+                        const int32_t* __restrict__ logit_src, __nv_bfloat16* __restrict__ out, int d, float eps) {
+  __shared__ float red[32];
+  const int i = blockIdx.x;
+  const int t = logit_src[i];
+  const int nv = d >> 2;
+  const float* xrow = x + static_cast<size_t>(t) * d;
+  float4 buf[MAX_VEC];
+  float ss = 0.0f;
+#pragma unroll
+  for (int k = 0; k < MAX_VEC; ++k) {
+    const int v = threadIdx.x + k * NORM_THREADS;
+    if (v < nv) {
+      buf[k] = *reinterpret_cast<const float4*>(xrow + 4 * v);
+      ss += buf[k].x * buf[k].x + buf[k].y * buf[k].y + buf[k].z * buf[k].z + buf[k].w * buf[k].w;
+    }
+  }
+  const float rstd = rsqrtf(block_sum(ss, red) / static_cast<float>(d) + eps);
+  __nv_bfloat16* orow = out + static_cast<size_t>(i) * 2 * d;
+#pragma unroll
+  for (int k = 0; k < MAX_VEC; ++k) {
+    const int v = threadIdx.x + k * NORM_THREADS;
+    if (v < nv) {
+      float4 g;
+      bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
+      const float4 y = make_float4(buf[k].x * rstd * g.x, buf[k].y * rstd * g.y, buf[k].z * rstd * g.z,
+                                   buf[k].w * rstd * g.w);
+      const uint2 hi = float4_to_bf16x4(y);
+      float4 hf;
+      bf16x4_to_float4(hi, hf);
+      const uint2 lo = float4_to_bf16x4(make_float4(y.x - hf.x, y.y - hf.y, y.z - hf.z, y.w - hf.w));
+      const int c = 4 * v;
+      __nv_bfloat16* dst = orow + (c >> 6) * 128 + (c & 63);
+      *reinterpret_cast<uint2*>(dst) = hi;
+      *reinterpret_cast<uint2*>(dst + 64) = lo;
+    }
+  }
+}
+
+// Final RMSNorm fused with the incremental pooler.  One block per work item = a block of rows
+// of one embedding segment.  Phase 1: one warp per row, shuffle-reduced sum of squares.
+// Phase 2: each thread owns column vectors and adds x * rstd over the item's rows in row
+// order.  The block's partial sum goes to scratch; the block that arrives last for a segment
+// adds the partials in block order, applies the gain, and updates the slot:
+//   S <- S + partial, count <- count + q_len            (Eq. 1-2 with w = 1)
+// (a request's first chunk overwrites instead, i.e. S(0) = 0, W(0) = 0).  On the final chunk
+// it emits S / count (mean) or the normed last row (last-token head), L2-normalised.
+__global__ void __launch_bounds__(NORM_THREADS)
+final_pool_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
+                  const PoolItem* __restrict__ items, const hb_seg* __restrict__ segs, float* __restrict__ part,
+                  uint32_t* __restrict__ counters, float* __restrict__ pool_sum, uint32_t* __restrict__ pool_meta,
+                  float* __restrict__ out_emb, int d, float eps, int n_slots, uint32_t* status) {
+  __shared__ float red[32];
+  __shared__ float rstd_s[32];
+  __shared__ uint32_t is_last_s;
+  const PoolItem it = items[blockIdx.x];
+  const hb_seg sg = segs[it.seg];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nv = d >> 2;
+  if (sg.pool_slot < 0 || sg.pool_slot >= n_slots) {
+    if (threadIdx.x == 0) atomicOr(status, HB_DEV_POOL_BAD_INDEX);
+    return;
+  }
+  // phase 1: row statistics (item rows <= 32)
+  for (int r = warp; r < it.n_rows; r += NORM_THREADS / 32) {
+    const float* xrow = x + static_cast<size_t>(it.row0 + r) * d;
+    float ss = 0.0f;
+    for (int v = lane; v < nv; v += 32) {
+      const float4 a = *reinterpret_cast<const float4*>(xrow + 4 * v);
+      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) rstd_s[r] = rsqrtf(ss / static_cast<float>(d) + eps);
+  }
+  __syncthreads();
+  // phase 2: column sums over the item's rows, fixed row order
+  float* my_part = part + static_cast<size_t>(it.part_base + it.block) * d;
+#pragma unroll 1
+  for (int v = threadIdx.x; v < nv; v += NORM_THREADS) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int r = 0; r < it.n_rows; ++r) {
+      const float4 a = *reinterpret_cast<const float4*>(x + static_cast<size_t>(it.row0 + r) * d + 4 * v);
+      const float s = rstd_s[r];
+      acc.x += a.x * s; acc.y += a.y * s; acc.z += a.z * s; acc.w += a.w * s;
+    }
+    *reinterpret_cast<float4*>(my_part + 4 * v) = acc;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t prev = atomicAdd(counters + it.seg, 1u);
+    is_last_s = (prev + 1u == static_cast<uint32_t>(it.n_blocks)) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!is_last_s) return;
+  __threadfence();
+  // segment tail: combine partials in block order, update the slot, maybe emit
+  const bool first_chunk = (sg.pos_start == 0);
+  float* S = pool_sum + static_cast<size_t>(sg.pool_slot) * d;
+  uint32_t* meta = pool_meta + static_cast<size_t>(sg.pool_slot) * 4;
+  const uint32_t old_count = first_chunk ? 0u : meta[0];
+  const uint32_t old_chunks = first_chunk ? 0u : meta[1];
+  const uint32_t new_count = old_count + static_cast<uint32_t>(sg.q_len);
+  const bool mean = (sg.pool_mode == HB_POOL_MEAN);
+  const bool emit = (sg.is_final != 0);
+  float4 e[MAX_VEC];
+  float nrm = 0.0f;
+#pragma unroll
+  for (int k = 0; k < MAX_VEC; ++k) {
+    const int v = threadIdx.x + k * NORM_THREADS;
+    e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (v < nv && (mean || emit)) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int b = 0; b < it.n_blocks; ++b) {
+        const float4 p = __ldcg(reinterpret_cast<const float4*>(part + static_cast<size_t>(it.part_base + b) * d + 4 * v));
+        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+      }
+      float4 g;
+      bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
+      acc.x *= g.x; acc.y *= g.y; acc.z *= g.z; acc.w *= g.w;
+      if (mean) {
+        if (!first_chunk) {
+          const float4 o = *reinterpret_cast<const float4*>(S + 4 * v);
+          acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+        }
+        *reinterpret_cast<float4*>(S + 4 * v) = acc;
+        const float inv = 1.0f / static_cast<float>(new_count);
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      }
+      e[k] = acc;
+      nrm += acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
+    }
+  }
+  if (emit) {
+    const float tot = block_sum(nrm, red);
+    const float inv = 1.0f / fmaxf(sqrtf(tot), 1e-12f);
+    float* o = out_emb + static_cast<size_t>(sg.emb_row) * d;
+#pragma unroll
+    for (int k = 0; k < MAX_VEC; ++k) {
+      const int v = threadIdx.x + k * NORM_THREADS;
+      if (v < nv)
+        *reinterpret_cast<float4*>(o + 4 * v) = make_float4(e[k].x * inv, e[k].y * inv, e[k].z * inv, e[k].w * inv);
+    }
+  }
+  if (threadIdx.x == 0) {
+    meta[0] = new_count;
+    meta[1] = old_chunks + 1u;
+    meta[2] = static_cast<uint32_t>(sg.pool_mode);
+    meta[3] = emit ? 1u : 0u;
+    counters[it.seg] = 0u;  // ready for the next step
+  }
+}
+
+__global__ void __launch_bounds__(256)
+argmax_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out) {
+  __shared__ float bv[8];
+  __shared__ int bi[8];
+  const float* row = logits + static_cast<size_t>(blockIdx.x) * V;
+  float best = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) {
+    const float v = row[c];
+    if (v > best || (v == best && c < idx)) { best = v; idx = c; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+    if (ov > best || (ov == best && oi < idx)) { best = ov; idx = oi; }
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { bv[warp] = best; bi[warp] = idx; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w)
+      if (bv[w] > best || (bv[w] == best && bi[w] < idx)) { best = bv[w]; idx = bi[w]; }
+    out[blockIdx.x] = idx;
+  }
+}
+
+int check_launch() { return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA; }
+
+}  // namespace
+
+int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s) {
+  norm_kernel<true><<<c->dd.T, NORM_THREADS, 0, s>>>(c->dd.tok, static_cast<const __nv_bfloat16*>(tok_emb),
+                                                     static_cast<const __nv_bfloat16*>(gain), c->x, c->h,
+                                                     c->cfg.d_model, c->cfg.rms_eps);
+  return check_launch();
+}
+
+int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s) {
+  norm_kernel<false><<<c->dd.T, NORM_THREADS, 0, s>>>(nullptr, nullptr, static_cast<const __nv_bfloat16*>(gain), c->x,
+                                                      c->h, c->cfg.d_model, c->cfg.rms_eps);
+  return check_launch();
+}
+
+int hb_launch_rope_append(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s) {
+  rope_append_kernel<<<c->dd.T, 256, 0, s>>>(c->qkv, c->q, kv, layer, c->dd.row_seg, c->dd.row_pos, c->dd.segs,
+                                             c->dd.pages, c->rope_cos, c->rope_sin, c->cfg.n_heads, c->cfg.max_pos,
+                                             c->status);
+  return check_launch();
+}
+
+int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta, int n_slots,
+                    float* out_emb, cudaStream_t s) {
+  const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(gain);
+  if (c->dd.n_logit > 0) {
+    final_logit_rows_kernel<<<c->dd.n_logit, NORM_THREADS, 0, s>>>(c->x, g, c->dd.logit_src, c->logit_in,
+                                                                   c->cfg.d_model, c->cfg.rms_eps);
+    if (check_launch() != HB_OK) return HB_ERR_CUDA;
+  }
+  if (c->dd.n_pool_items > 0) {
+    final_pool_kernel<<<c->dd.n_pool_items, NORM_THREADS, 0, s>>>(
+        c->x, g, c->dd.pool_items, c->dd.segs, c->pool_part, c->counters, pool_sum, pool_meta, out_emb,
+        c->cfg.d_model, c->cfg.rms_eps, n_slots, c->status);
+    if (check_launch() != HB_OK) return HB_ERR_CUDA;
+  }
+  return HB_OK;
+}
+
+int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s) {
+  if (n_rows <= 0) return HB_OK;
+  argmax_kernel<<<n_rows, 256, 0, s>>>(logits, V, out);
+  return check_launch();
+}

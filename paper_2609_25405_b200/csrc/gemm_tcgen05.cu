@@ -1,0 +1,438 @@
+// Projection GEMM for sm_100a: C = epilogue(A * B^T), A [M,K] and B [N,K] bf16 K-major,
+// fp32 accumulation in tensor memory.
+//
+// These are the dense contractions of the shared forward pass (Section 3.1 of the paper:
+// the forward "applies attention and feed-forward layers" to every row of the mixed
+// batch): QKV, O, gate/up, down and the LM head.
+//
+// Structure (one persistent CTA per SM, 192 threads):
+//   warp 0   TMA producer: cp.async.bulk.tensor 2-D tiles (128B swizzle) into a ring of
+//            shared-memory stages, completion on mbarriers
+//   warp 1   MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=16) from shared
+//            memory descriptors into one of two TMEM accumulators; tcgen05.commit
+//            releases stages and publishes finished accumulators
+//   warps 2-5 epilogue: tcgen05.ld the accumulator (each warp owns 32 TMEM lanes), apply
+//            the epilogue, store with 16-byte vectors; overlaps the next tile's main loop
+// Every mbarrier wait is bounded in time; on expiry the CTA raises a status bit, stops
+// issuing work, lets outstanding copies land, frees its TMEM and returns.
+#include "hb_internal.h"
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+
+template <int BN>
+struct Tile {
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TMEM_COLS = 2 * BN;  // two accumulators; 256 or 512 (powers of two)
+  static constexpr int BAR_BYTES = 256;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false if the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c_inner, int c_outer) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
+      : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart,
+// 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);        // start address
+  d |= static_cast<uint64_t>(1) << 16;                        // leading byte offset (unused with swizzle)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                        // descriptor version (Blackwell)
+  d |= static_cast<uint64_t>(2) << 61;                        // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = BN.
+template <int BN>
+__device__ __forceinline__ constexpr uint32_t make_idesc() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+         (static_cast<uint32_t>(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+
+// Store one thread's 32 consecutive accumulator columns of one row.
+template <int EPI>
+__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32]) {
+  // col0 is a multiple of 32; N is a multiple of 8, so validity is decided per group of 8
+  if constexpr (EPI == HB_EPI_BF16) {
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + static_cast<size_t>(row) * g.ldc + col0;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      if (col0 + v * 8 < g.N) {
+        uint4 pk;
+        pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+        pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+        pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+        pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+        *reinterpret_cast<uint4*>(out + v * 8) = pk;
+      }
+    }
+  } else if constexpr (EPI == HB_EPI_F32 || EPI == HB_EPI_RESID_F32) {
+    float* out = static_cast<float*>(g.C) + static_cast<size_t>(row) * g.ldc + col0;
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      if (col0 + v * 4 < g.N) {
+        float4 o;
+        o.x = __uint_as_float(r[v * 4 + 0]);
+        o.y = __uint_as_float(r[v * 4 + 1]);
+        o.z = __uint_as_float(r[v * 4 + 2]);
+        o.w = __uint_as_float(r[v * 4 + 3]);
+        if constexpr (EPI == HB_EPI_RESID_F32) {
+          const float4 old = *reinterpret_cast<const float4*>(out + v * 4);
+          o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+        }
+        *reinterpret_cast<float4*>(out + v * 4) = o;
+      }
+    }
+  } else {  // HB_EPI_SWIGLU: columns (2j, 2j+1) = (gate_j, up_j) -> out column j
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + static_cast<size_t>(row) * g.ldc + col0 / 2;
+#pragma unroll
+    for (int v = 0; v < 2; ++v) {
+      if (col0 + v * 16 < g.N) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float g0 = __uint_as_float(r[v * 16 + j * 4 + 0]), u0 = __uint_as_float(r[v * 16 + j * 4 + 1]);
+          const float g1 = __uint_as_float(r[v * 16 + j * 4 + 2]), u1 = __uint_as_float(r[v * 16 + j * 4 + 3]);
+          pk[j] = pack_bf16(silu_f(g0) * u0, silu_f(g1) * u1);
+        }
+        *reinterpret_cast<uint4*>(out + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+    }
+  }
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const GemmArgs g) {
+  using T = Tile<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + T::STAGES * T::STAGE_BYTES;
+  // barrier layout (8 B each): full[STAGES], empty[STAGES], tfull[2], tempty[2]; then tmem slot, abort flag
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (T::STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * T::STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * T::STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_gen + T::STAGES * T::STAGE_BYTES + 8 * (2 * T::STAGES + 4));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  const int m_tiles = (g.M + BM - 1) / BM;
+  const int n_tiles = (g.N + BN - 1) / BN;
+  const int total_tiles = m_tiles * n_tiles;
+  const int k_blocks = (g.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T::STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(static_cast<uint32_t>(T::TMEM_COLS))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const int m0 = (tile % m_tiles) * BM;
+        const int n0 = (tile / m_tiles) * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = smem_base + stage * T::STAGE_BYTES;
+          const uint32_t b_dst = a_dst + T::A_BYTES;
+          mbar_arrive_expect_tx(full_bar(stage), T::STAGE_BYTES);
+          tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, m0);
+          tma_load_2d(b_dst, &tmB, full_bar(stage), (kb >> g.b_kshift) * BK, n0);
+          if (++stage == T::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // give copies already in flight time to land before shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc<BN>();
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tcgen05_fence_after();
+          const uint32_t a_addr = smem_base + stage * T::STAGE_BYTES;
+          const uint64_t adesc = make_smem_desc(a_addr);
+          const uint64_t bdesc = make_smem_desc(a_addr + T::A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing 16 elements along K inside the 128-byte swizzle row = +32 B = +2 in the address field
+            umma_bf16(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));  // stage is free once these MMAs have read it
+          if (++stage == T::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));      // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------- epilogue (warps 2..5) ----------------
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const int m0 = (tile % m_tiles) * BM;
+      const int n0 = (tile / m_tiles) * BN;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tcgen05_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(t_row + static_cast<uint32_t>(c), r);
+        if (row < g.M && n0 + c < g.N) epilogue_store<EPI>(g, row, n0 + c, r);
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(g.status, HB_DEV_GEMM_WAIT_EXPIRED);
+  if (warp == 1) {
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(T::TMEM_COLS))
+                 : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+template <int BN, int EPI>
+int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& a, int num_sms, cudaStream_t s) {
+  using T = Tile<BN>;
+  static bool configured = false;
+  auto kern = hb_gemm_tcgen05_kernel<BN, EPI>;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES) != cudaSuccess)
+      return HB_ERR_CUDA;
+    configured = true;
+  }
+  const int m_tiles = (a.M + BM - 1) / BM;
+  const int n_tiles = (a.N + BN - 1) / BN;
+  int grid = m_tiles * n_tiles;
+  if (grid > num_sms) grid = num_sms;
+  if (grid < 1) return HB_OK;
+  kern<<<grid, NUM_THREADS, T::SMEM_BYTES, s>>>(tmA, tmB, a);
+  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+}
+
+template <int BN>
+int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, int epi, const GemmArgs& a, int num_sms,
+              cudaStream_t s) {
+  switch (epi) {
+    case HB_EPI_BF16: return launch_one<BN, HB_EPI_BF16>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU>(tmA, tmB, a, num_sms, s);
+    default: return HB_ERR_BAD_ARG;
+  }
+}
+
+}  // namespace
+
+int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return HB_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || (cols & 7u) || rows == 0 || cols == 0) return HB_ERR_BAD_ARG;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? HB_OK : HB_ERR_CUDA;
+}
+
+// Tile width: 256 columns halves the shared-memory traffic per flop; 128 gives more tiles
+// when the problem has too few to fill the SMs or the last wave would be mostly idle.
+int hb_gemm_pick_bn(int M, int N, int num_sms) {
+  const int m_tiles = (M + BM - 1) / BM;
+  const long t256 = static_cast<long>(m_tiles) * ((N + 255) / 256);
+  const long t128 = static_cast<long>(m_tiles) * ((N + 127) / 128);
+  if (t256 < num_sms) return 128;
+  const double e256 = static_cast<double>(t256) / (((t256 + num_sms - 1) / num_sms) * num_sms);
+  const double e128 = static_cast<double>(t128) / (((t128 + num_sms - 1) / num_sms) * num_sms);
+  return (e128 * 0.92 > e256) ? 128 : 256;
+}
+
+int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi, const GemmArgs& a,
+                   int num_sms, cudaStream_t s) {
+  if (bn == 256) return launch_bn<256>(tmA, tmB, epi, a, num_sms, s);
+  if (bn == 128) return launch_bn<128>(tmA, tmB, epi, a, num_sms, s);
+  return HB_ERR_BAD_ARG;
+}

@@ -1,0 +1,151 @@
+// Internal declarations shared by the translation units of libhb.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/hb.h"
+
+// Device status codes (OR-ed into the context's status word).
+enum : uint32_t {
+  HB_DEV_GEMM_WAIT_EXPIRED = 1u << 0,
+  HB_DEV_ATTN_BAD_INDEX = 1u << 1,
+  HB_DEV_APPEND_BAD_INDEX = 1u << 2,
+  HB_DEV_POOL_BAD_INDEX = 1u << 3,
+  HB_DEV_ATTN_WAIT_EXPIRED = 1u << 4,
+};
+
+// Attention work item: one (segment, kv head, row tile, key split).
+struct AttnItem {
+  int32_t seg;        // segment index
+  int32_t kv_head;
+  int32_t row0;       // first row of the tile inside the segment
+  int32_t n_rows;     // rows in the tile
+  int32_t key0;       // first key of this split
+  int32_t key1;       // one past the last key this split may touch
+  int32_t split;      // split index, n_splits
+  int32_t n_splits;
+  int32_t part_base;  // first partial-result record of this (seg, kv_head, row tile)
+  int32_t pad[3];
+};
+
+// Pool work item: rows [row0, row0 + n_rows) of an embedding segment.
+struct PoolItem {
+  int32_t seg;
+  int32_t row0;       // absolute token row
+  int32_t n_rows;
+  int32_t block;      // block index inside the segment
+  int32_t n_blocks;
+  int32_t part_base;  // first partial-sum record of the segment
+  int32_t pad[2];
+};
+
+struct DeviceDesc {
+  // all device pointers into the context's descriptor buffer
+  const int32_t* tok;       // [T]
+  const int32_t* row_seg;   // [T]
+  const int32_t* row_pos;   // [T]
+  const hb_seg* segs;       // [R]
+  const int32_t* pages;     // [n_page_ids]
+  const int32_t* logit_src; // [n_logit_rows] token row feeding logits row i
+  const AttnItem* attn_items;
+  const PoolItem* pool_items;
+  int32_t T, R, n_logit, n_attn_items, n_pool_items;
+};
+
+struct KvGeom {
+  __nv_bfloat16* arena;
+  int64_t layer_stride;  // elements
+  int64_t page_stride;   // elements: 2 * Hkv * P * Dh
+  int32_t n_pages, Hkv, P, Dh;
+};
+
+struct hb_kv {
+  hb_model_cfg cfg;
+  void* arena;
+  size_t arena_bytes;
+  int32_t n_pages;
+  std::vector<uint8_t> used;
+  int32_t n_free;
+};
+
+struct hb_pool {
+  hb_model_cfg cfg;
+  void* arena;
+  size_t arena_bytes;
+  int32_t n_slots;
+  std::vector<uint8_t> used;
+  int32_t n_free;
+};
+
+// ---- GEMM -------------------------------------------------------------------
+struct GemmArgs {
+  void* C;
+  int32_t M, N, K;      // K = columns of A; B has K >> b_kshift columns
+  int32_t ldc;          // elements
+  int32_t b_kshift;     // B k-block index = A k-block index >> b_kshift
+  uint32_t* status;
+};
+
+int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
+                    uint32_t box_rows);
+int hb_gemm_pick_bn(int M, int N, int num_sms);
+int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
+                   const GemmArgs& a, int num_sms, cudaStream_t s);
+
+// ---- elementwise / attention launchers ---------------------------------------
+struct hb_ctx;
+int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s);
+int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
+int hb_launch_rope_append(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s);
+int hb_launch_attention(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s);
+int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
+                    int n_slots, float* out_emb, cudaStream_t s);
+int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s);
+
+struct hb_ctx {
+  hb_model_cfg cfg;
+  int32_t max_tokens, max_segs, max_page_ids;
+  int num_sms;
+  int device;
+  bool owns_ws;
+  uint8_t* ws;
+  size_t ws_bytes;
+  // workspace carve-up (device)
+  float* x;                 // [max_tokens, d] residual stream, fp32
+  __nv_bfloat16* h;         // [max_tokens, d] normed activations
+  float* qkv;               // [max_tokens, n_qkv] projection output, fp32
+  __nv_bfloat16* q;         // [max_tokens, Hq*Dh] rotated queries
+  __nv_bfloat16* attn_out;  // [max_tokens, Hq*Dh]
+  __nv_bfloat16* act;       // [max_tokens, F]
+  __nv_bfloat16* logit_in;  // [max_logit_rows, 2d] hi/lo split of final hidden rows
+  float* rope_cos;          // [max_pos, Dh/2]
+  float* rope_sin;
+  float* attn_part;         // split-KV partial results
+  float* pool_part;         // pooling partial sums
+  uint32_t* counters;       // arrival counters (attention merge, pooling merge)
+  uint32_t* status;         // device status word
+  uint8_t* desc_dev;        // packed descriptor
+  size_t desc_cap;
+  void* extra;              // host-side state (pinned descriptor staging ring, layout)
+  size_t attn_part_floats, pool_part_floats;
+  int32_t n_counters;
+  int32_t max_logit_rows;
+  DeviceDesc dd;
+  // tensor maps over the activation buffers (A operands)
+  CUtensorMap tm_h, tm_attn_out, tm_act, tm_logit_in;
+  // cached weight tensor maps
+  struct WMaps {
+    const void* key[4];
+    CUtensorMap qkv, o, gu, down;
+    int bn_qkv, bn_o, bn_gu, bn_down;
+  };
+  std::vector<WMaps> wmaps;
+  const void* lm_key;
+  CUtensorMap tm_lm;
+  int32_t last_launches;
+};

@@ -1,0 +1,650 @@
+// Host side of libhb: context, workspace carve-up, page / slot free lists, descriptor
+// validation and packing, and the launch sequence of one mixed step (the Forward, IncPooler
+// and logits part of the paper's inference loop, Algorithm 1).
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "hb_internal.h"
+
+namespace {
+
+constexpr int POOL_ROWS = 32;   // rows per pooling work item
+constexpr int N_STAGING = 4;    // pinned descriptor staging ring
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool cfg_ok(const hb_model_cfg* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->d_model < 64 || c->n_heads < 1 || c->n_kv_heads < 1 || c->d_ffn < 64 || c->vocab < 8)
+    return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_heads % c->n_kv_heads) return false;
+  if (c->d_model % 64 || (c->n_heads * c->head_dim) % 64 || c->d_ffn % 64 || c->vocab % 8) return false;
+  if (c->d_model > 8192) return false;
+  if (c->page_size != 16) return false;
+  if (c->max_pos < 1 || !(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return false;
+  return true;
+}
+
+struct Carve {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  }
+};
+
+struct Layout {
+  size_t x, h, qkv, q, attn_out, act, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, status, desc;
+  size_t total, desc_cap, attn_part_floats, pool_part_floats;
+  int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items;
+};
+
+Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids) {
+  Layout L{};
+  Carve cv;
+  const size_t rows = align_up(static_cast<size_t>(max_tokens), 128);
+  const size_t lrows = align_up(static_cast<size_t>(max_segs), 128);
+  const size_t n_qkv = static_cast<size_t>(c.n_heads + 2 * c.n_kv_heads) * c.head_dim;
+  const size_t n_q = static_cast<size_t>(c.n_heads) * c.head_dim;
+  L.rows_pad = static_cast<int32_t>(rows);
+  L.logit_rows_pad = static_cast<int32_t>(lrows);
+  L.x = cv.take(rows * c.d_model * 4);
+  L.h = cv.take(rows * c.d_model * 2);
+  L.qkv = cv.take(rows * n_qkv * 4);
+  L.q = cv.take(rows * n_q * 2);
+  L.attn_out = cv.take(rows * n_q * 2);
+  L.act = cv.take(rows * c.d_ffn * 2);
+  L.logit_in = cv.take(lrows * 2 * c.d_model * 2);
+  L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
+  L.rope_sin = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
+  L.max_pool_items = max_tokens / POOL_ROWS + max_segs + 1;
+  L.max_attn_items = 0;
+  L.attn_part_floats = 4;
+  L.pool_part_floats = static_cast<size_t>(L.max_pool_items) * c.d_model;
+  L.attn_part = cv.take(L.attn_part_floats * 4);
+  L.pool_part = cv.take(L.pool_part_floats * 4);
+  L.n_counters = max_segs + 1;
+  L.counters = cv.take(static_cast<size_t>(L.n_counters) * 4);
+  L.status = cv.take(256);
+  size_t dc = 0;
+  dc += align_up(static_cast<size_t>(max_tokens) * 4, 16) * 3;          // tok, row_seg, row_pos
+  dc += align_up(static_cast<size_t>(max_segs) * sizeof(hb_seg), 16);
+  dc += align_up(static_cast<size_t>(max_page_ids) * 4, 16);
+  dc += align_up(static_cast<size_t>(max_segs) * 4, 16);                // logit_src
+  dc += align_up(static_cast<size_t>(L.max_attn_items) * sizeof(AttnItem), 16);
+  dc += align_up(static_cast<size_t>(L.max_pool_items) * sizeof(PoolItem), 16);
+  L.desc_cap = dc + 64;
+  L.desc = cv.take(L.desc_cap);
+  L.total = cv.off;
+  return L;
+}
+
+int validate(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids, int32_t n_pages,
+             int32_t n_slots, const hb_batch_desc* d) {
+  if (!d) return HB_ERR_BAD_ARG;
+  if (d->n_tokens < 0 || d->n_segs < 0 || d->n_page_ids < 0 || d->n_logit_rows < 0 || d->n_emb_rows < 0)
+    return HB_ERR_BAD_DESC;
+  if (d->n_tokens > max_tokens || d->n_segs > max_segs || d->n_page_ids > max_page_ids) return HB_ERR_TOO_LARGE;
+  if ((d->n_tokens > 0 && !d->token_ids) || (d->n_segs > 0 && !d->segs) || (d->n_page_ids > 0 && !d->page_ids))
+    return HB_ERR_BAD_ARG;
+  if ((d->n_tokens == 0) != (d->n_segs == 0)) return HB_ERR_BAD_DESC;
+  for (int32_t t = 0; t < d->n_tokens; ++t)
+    if (d->token_ids[t] < 0 || d->token_ids[t] >= c.vocab) return HB_ERR_BAD_DESC;
+  for (int32_t i = 0; i < d->n_page_ids; ++i)
+    if (d->page_ids[i] < 0 || d->page_ids[i] >= n_pages) return HB_ERR_BAD_DESC;
+  const int P = c.page_size;
+  std::vector<uint8_t> page_written(static_cast<size_t>(std::max(n_pages, 1)), 0);
+  std::vector<uint8_t> slot_used(static_cast<size_t>(std::max(n_slots, 1)), 0);
+  std::vector<uint8_t> lrow(static_cast<size_t>(std::max(d->n_logit_rows, 1)), 0);
+  std::vector<uint8_t> erow(static_cast<size_t>(std::max(d->n_emb_rows, 1)), 0);
+  int32_t at = 0, prev_kind = 0, n_l = 0, n_e = 0;
+  for (int32_t r = 0; r < d->n_segs; ++r) {
+    const hb_seg& s = d->segs[r];
+    if (s.kind < HB_KIND_DECODE || s.kind > HB_KIND_EMBED_CHUNK || s.kind < prev_kind) return HB_ERR_BAD_DESC;
+    prev_kind = s.kind;
+    if (s.q_start != at || s.q_len < 1 || (s.kind == HB_KIND_DECODE && s.q_len != 1)) return HB_ERR_BAD_DESC;
+    if (s.q_len > d->n_tokens - at) return HB_ERR_BAD_DESC;
+    at += s.q_len;
+    if (s.pos_start < 0 || s.pos_start > c.max_pos - s.q_len) return HB_ERR_BAD_DESC;
+    const int32_t need = (s.pos_start + s.q_len + P - 1) / P;
+    if (s.pt_start < 0 || s.pt_len < need || s.pt_start > d->n_page_ids - s.pt_len) return HB_ERR_BAD_DESC;
+    // pages this segment writes must not be listed by any other segment, nor twice by this one
+    for (int32_t b = s.pos_start / P; b < need; ++b) {
+      const int32_t pg = d->page_ids[s.pt_start + b];
+      if (page_written[pg]) return HB_ERR_BAD_DESC;
+      page_written[pg] = static_cast<uint8_t>(1);
+    }
+    const bool embed = (s.kind == HB_KIND_EMBED_CHUNK);
+    if (embed) {
+      if (s.pool_mode != HB_POOL_MEAN && s.pool_mode != HB_POOL_LAST) return HB_ERR_BAD_DESC;
+      if (s.pool_slot < 0 || s.pool_slot >= n_slots || slot_used[s.pool_slot]) return HB_ERR_BAD_DESC;
+      slot_used[s.pool_slot] = 1;
+      if (s.logits_row != -1) return HB_ERR_BAD_DESC;
+      if (s.is_final) {
+        if (s.emb_row < 0 || s.emb_row >= d->n_emb_rows || erow[s.emb_row]) return HB_ERR_BAD_DESC;
+        erow[s.emb_row] = 1;
+        ++n_e;
+      } else if (s.emb_row != -1) {
+        return HB_ERR_BAD_DESC;
+      }
+    } else {
+      if (s.pool_mode != HB_POOL_NONE || s.pool_slot != -1 || s.emb_row != -1) return HB_ERR_BAD_DESC;
+      const bool wants = (s.kind == HB_KIND_DECODE) || (s.is_final != 0);
+      if (wants) {
+        if (s.logits_row < 0 || s.logits_row >= d->n_logit_rows || lrow[s.logits_row]) return HB_ERR_BAD_DESC;
+        lrow[s.logits_row] = 1;
+        ++n_l;
+      } else if (s.logits_row != -1) {
+        return HB_ERR_BAD_DESC;
+      }
+    }
+  }
+  if (at != d->n_tokens || n_l != d->n_logit_rows || n_e != d->n_emb_rows) return HB_ERR_BAD_DESC;
+  // a page read by one segment and written by another: reject (read-only sharing is allowed)
+  for (int32_t r = 0; r < d->n_segs; ++r) {
+    const hb_seg& s = d->segs[r];
+    const int32_t first_w = s.pos_start / P;
+    for (int32_t b = 0; b < first_w && b < s.pt_len; ++b)
+      if (page_written[d->page_ids[s.pt_start + b]]) return HB_ERR_BAD_DESC;
+  }
+  return HB_OK;
+}
+
+struct Staging {
+  uint8_t* host = nullptr;
+  cudaEvent_t ev = nullptr;
+  bool pending = false;
+};
+
+struct CtxExtra {
+  Staging ring[N_STAGING];
+  int next = 0;
+  Layout lay;
+};
+
+CtxExtra* extra_of(hb_ctx* c) { return static_cast<CtxExtra*>(c->extra); }
+
+}  // namespace
+
+extern "C" {
+
+int hb_workspace_bytes(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids,
+                       size_t* out_bytes) {
+  if (!cfg_ok(cfg) || !out_bytes || max_tokens < 1 || max_segs < 1 || max_page_ids < 1) return HB_ERR_BAD_ARG;
+  *out_bytes = make_layout(*cfg, max_tokens, max_segs, max_page_ids).total;
+  return HB_OK;
+}
+
+int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids, void* workspace,
+              size_t workspace_bytes, hb_ctx** out) {
+  if (!out) return HB_ERR_BAD_ARG;
+  *out = nullptr;
+  if (!cfg) return HB_ERR_BAD_ARG;
+  if (!cfg_ok(cfg)) return HB_ERR_UNSUPPORTED;
+  if (max_tokens < 1 || max_segs < 1 || max_page_ids < 1) return HB_ERR_BAD_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HB_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HB_ERR_CUDA;
+  if (prop.major != 10) return HB_ERR_UNSUPPORTED;  // tcgen05 / TMEM kernels: sm_100 only
+  const Layout lay = make_layout(*cfg, max_tokens, max_segs, max_page_ids);
+  hb_ctx* c = new (std::nothrow) hb_ctx();
+  CtxExtra* ex = new (std::nothrow) CtxExtra();
+  if (!c || !ex) { delete c; delete ex; return HB_ERR_BAD_ARG; }
+  ex->lay = lay;
+  c->cfg = *cfg;
+  c->max_tokens = max_tokens;
+  c->max_segs = max_segs;
+  c->max_page_ids = max_page_ids;
+  c->num_sms = prop.multiProcessorCount;
+  c->device = dev;
+  c->extra = ex;
+  c->lm_key = nullptr;
+  c->last_launches = 0;
+  if (workspace) {
+    if (workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255u)) {
+      delete c; delete ex;
+      return HB_ERR_BAD_ARG;
+    }
+    c->ws = static_cast<uint8_t*>(workspace);
+    c->owns_ws = false;
+  } else {
+    void* p = nullptr;
+    if (cudaMalloc(&p, lay.total) != cudaSuccess) { delete c; delete ex; return HB_ERR_CUDA; }
+    c->ws = static_cast<uint8_t*>(p);
+    c->owns_ws = true;
+  }
+  c->ws_bytes = lay.total;
+  c->x = reinterpret_cast<float*>(c->ws + lay.x);
+  c->h = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.h);
+  c->qkv = reinterpret_cast<float*>(c->ws + lay.qkv);
+  c->q = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.q);
+  c->attn_out = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.attn_out);
+  c->act = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.act);
+  c->logit_in = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.logit_in);
+  c->rope_cos = reinterpret_cast<float*>(c->ws + lay.rope_cos);
+  c->rope_sin = reinterpret_cast<float*>(c->ws + lay.rope_sin);
+  c->attn_part = reinterpret_cast<float*>(c->ws + lay.attn_part);
+  c->pool_part = reinterpret_cast<float*>(c->ws + lay.pool_part);
+  c->counters = reinterpret_cast<uint32_t*>(c->ws + lay.counters);
+  c->status = reinterpret_cast<uint32_t*>(c->ws + lay.status);
+  c->desc_dev = c->ws + lay.desc;
+  c->desc_cap = lay.desc_cap;
+  c->attn_part_floats = lay.attn_part_floats;
+  c->pool_part_floats = lay.pool_part_floats;
+  c->n_counters = lay.n_counters;
+  c->max_logit_rows = lay.logit_rows_pad;
+  c->wmaps.resize(cfg->n_layers);
+  for (auto& w : c->wmaps) w.key[0] = w.key[1] = w.key[2] = w.key[3] = nullptr;
+
+  int rc = HB_OK;
+  bool cuda_ok = true;
+  // zero the activation buffers once (rows past the batch feed unused accumulator rows)
+  cuda_ok &= cudaMemset(c->ws, 0, lay.total) == cudaSuccess;
+  // rotary table: angle(p, i) = p * theta^(-2i/Dh), computed in double, stored as float
+  {
+    const int half = cfg->head_dim / 2;
+    std::vector<float> hc(static_cast<size_t>(cfg->max_pos) * half), hs(hc.size());
+    for (int i = 0; i < half; ++i) {
+      const double inv_freq = pow(static_cast<double>(cfg->rope_theta), -2.0 * i / cfg->head_dim);
+      for (int p = 0; p < cfg->max_pos; ++p) {
+        const double a = static_cast<double>(p) * inv_freq;
+        hc[static_cast<size_t>(p) * half + i] = static_cast<float>(cos(a));
+        hs[static_cast<size_t>(p) * half + i] = static_cast<float>(sin(a));
+      }
+    }
+    cuda_ok &= cudaMemcpy(c->rope_cos, hc.data(), hc.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+    cuda_ok &= cudaMemcpy(c->rope_sin, hs.data(), hs.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  }
+  for (int i = 0; i < N_STAGING; ++i) {
+    cuda_ok &= cudaMallocHost(reinterpret_cast<void**>(&ex->ring[i].host), lay.desc_cap) == cudaSuccess;
+    cuda_ok &= cudaEventCreateWithFlags(&ex->ring[i].ev, cudaEventDisableTiming) == cudaSuccess;
+  }
+  if (cuda_ok) {
+    const uint64_t n_q = static_cast<uint64_t>(cfg->n_heads) * cfg->head_dim;
+    rc = hb_tmap_2d_bf16(&c->tm_h, c->h, lay.rows_pad, cfg->d_model, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_attn_out, c->attn_out, lay.rows_pad, n_q, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_act, c->act, lay.rows_pad, cfg->d_ffn, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_logit_in, c->logit_in, lay.logit_rows_pad, 2ull * cfg->d_model, 128);
+  }
+  cuda_ok &= cudaDeviceSynchronize() == cudaSuccess;
+  if (!cuda_ok || rc != HB_OK) {
+    hb_destroy(c);
+    return cuda_ok ? rc : HB_ERR_CUDA;
+  }
+  *out = c;
+  return HB_OK;
+}
+
+int hb_destroy(hb_ctx* c) {
+  if (!c) return HB_ERR_BAD_ARG;
+  cudaDeviceSynchronize();
+  CtxExtra* ex = extra_of(c);
+  if (ex) {
+    for (int i = 0; i < N_STAGING; ++i) {
+      if (ex->ring[i].host) cudaFreeHost(ex->ring[i].host);
+      if (ex->ring[i].ev) cudaEventDestroy(ex->ring[i].ev);
+    }
+    delete ex;
+  }
+  if (c->owns_ws && c->ws) cudaFree(c->ws);
+  delete c;
+  return HB_OK;
+}
+
+// ---- KV pages ----------------------------------------------------------------
+
+int hb_kv_arena_bytes(const hb_model_cfg* cfg, int32_t n_pages, size_t* out_bytes) {
+  if (!cfg_ok(cfg) || n_pages < 1 || !out_bytes) return HB_ERR_BAD_ARG;
+  *out_bytes = static_cast<size_t>(cfg->n_layers) * n_pages * 2 * cfg->n_kv_heads * cfg->page_size * cfg->head_dim * 2;
+  return HB_OK;
+}
+
+int hb_kv_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32_t n_pages, hb_kv** out) {
+  if (!out) return HB_ERR_BAD_ARG;
+  *out = nullptr;
+  size_t need = 0;
+  if (hb_kv_arena_bytes(cfg, n_pages, &need) != HB_OK) return HB_ERR_BAD_ARG;
+  if (arena && (arena_bytes < need || (reinterpret_cast<uintptr_t>(arena) & 255u))) return HB_ERR_BAD_ARG;
+  hb_kv* kv = new (std::nothrow) hb_kv();
+  if (!kv) return HB_ERR_BAD_ARG;
+  kv->cfg = *cfg;
+  kv->arena = arena;
+  kv->arena_bytes = arena_bytes;
+  kv->n_pages = n_pages;
+  kv->used.assign(n_pages, 0);
+  kv->n_free = n_pages;
+  *out = kv;
+  return HB_OK;
+}
+
+int hb_kv_destroy(hb_kv* kv) {
+  if (!kv) return HB_ERR_BAD_ARG;
+  delete kv;
+  return HB_OK;
+}
+
+int hb_kv_alloc_pages(hb_kv* kv, int32_t n, int32_t* out_ids) {
+  if (!kv || n < 0 || (n > 0 && !out_ids)) return HB_ERR_BAD_ARG;
+  if (n > kv->n_free) return HB_ERR_OOM_PAGES;
+  int32_t got = 0;
+  for (int32_t p = 0; p < kv->n_pages && got < n; ++p)
+    if (!kv->used[p]) {
+      kv->used[p] = 1;
+      out_ids[got++] = p;
+    }
+  kv->n_free -= n;
+  return HB_OK;
+}
+
+int hb_kv_free_pages(hb_kv* kv, int32_t n, const int32_t* ids) {
+  if (!kv || n < 0 || (n > 0 && !ids)) return HB_ERR_BAD_ARG;
+  for (int32_t i = 0; i < n; ++i) {
+    if (ids[i] < 0 || ids[i] >= kv->n_pages || !kv->used[ids[i]]) return HB_ERR_BAD_ARG;
+    for (int32_t j = 0; j < i; ++j)
+      if (ids[j] == ids[i]) return HB_ERR_BAD_ARG;
+  }
+  for (int32_t i = 0; i < n; ++i) kv->used[ids[i]] = 0;
+  kv->n_free += n;
+  return HB_OK;
+}
+
+int hb_kv_free_count(const hb_kv* kv, int32_t* out_free) {
+  if (!kv || !out_free) return HB_ERR_BAD_ARG;
+  *out_free = kv->n_free;
+  return HB_OK;
+}
+
+// ---- pool slots ----------------------------------------------------------------
+
+int hb_pool_arena_bytes(const hb_model_cfg* cfg, int32_t n_slots, size_t* out_bytes) {
+  if (!cfg_ok(cfg) || n_slots < 1 || !out_bytes) return HB_ERR_BAD_ARG;
+  *out_bytes = static_cast<size_t>(n_slots) * cfg->d_model * 4 + static_cast<size_t>(n_slots) * 16;
+  return HB_OK;
+}
+
+int hb_pool_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32_t n_slots, hb_pool** out) {
+  if (!out) return HB_ERR_BAD_ARG;
+  *out = nullptr;
+  size_t need = 0;
+  if (hb_pool_arena_bytes(cfg, n_slots, &need) != HB_OK) return HB_ERR_BAD_ARG;
+  if (arena && (arena_bytes < need || (reinterpret_cast<uintptr_t>(arena) & 255u))) return HB_ERR_BAD_ARG;
+  hb_pool* p = new (std::nothrow) hb_pool();
+  if (!p) return HB_ERR_BAD_ARG;
+  p->cfg = *cfg;
+  p->arena = arena;
+  p->arena_bytes = arena_bytes;
+  p->n_slots = n_slots;
+  p->used.assign(n_slots, 0);
+  p->n_free = n_slots;
+  *out = p;
+  return HB_OK;
+}
+
+int hb_pool_destroy(hb_pool* p) {
+  if (!p) return HB_ERR_BAD_ARG;
+  delete p;
+  return HB_OK;
+}
+
+int hb_pool_alloc_slot(hb_pool* p, int32_t* out_slot) {
+  if (!p || !out_slot) return HB_ERR_BAD_ARG;
+  if (p->n_free == 0) return HB_ERR_OOM_SLOTS;
+  for (int32_t s = 0; s < p->n_slots; ++s)
+    if (!p->used[s]) {
+      p->used[s] = 1;
+      --p->n_free;
+      *out_slot = s;
+      return HB_OK;
+    }
+  return HB_ERR_OOM_SLOTS;
+}
+
+int hb_pool_free_slot(hb_pool* p, int32_t slot) {
+  if (!p || slot < 0 || slot >= p->n_slots || !p->used[slot]) return HB_ERR_BAD_ARG;
+  p->used[slot] = 0;
+  ++p->n_free;
+  return HB_OK;
+}
+
+// ---- the step --------------------------------------------------------------------
+
+int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids,
+                     int32_t n_pages, int32_t n_slots, const hb_batch_desc* desc) {
+  if (!cfg_ok(cfg)) return HB_ERR_BAD_ARG;
+  return validate(*cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, desc);
+}
+
+int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv* kv, hb_pool* pool,
+                  float* out_logits, float* out_emb, void* stream) {
+  if (!c || !d || !w || !kv || !w->layers || !w->tok_emb || !w->final_norm) return HB_ERR_BAD_ARG;
+  if (!kv->arena) return HB_ERR_BAD_ARG;
+  if (memcmp(&kv->cfg, &c->cfg, sizeof(hb_model_cfg)) != 0) return HB_ERR_BAD_ARG;
+  const int32_t n_slots = pool ? pool->n_slots : 0;
+  int rc = validate(c->cfg, c->max_tokens, c->max_segs, c->max_page_ids, kv->n_pages, n_slots, d);
+  if (rc != HB_OK) return rc;
+  if (d->n_logit_rows > 0 && (!out_logits || !w->lm_head)) return HB_ERR_BAD_ARG;
+  if (d->n_emb_rows > 0 && !out_emb) return HB_ERR_BAD_ARG;
+  bool any_embed = false;
+  for (int32_t r = 0; r < d->n_segs; ++r) any_embed |= (d->segs[r].kind == HB_KIND_EMBED_CHUNK);
+  if (any_embed && (!pool || !pool->arena)) return HB_ERR_BAD_ARG;
+  c->last_launches = 0;
+  if (d->n_tokens == 0) return HB_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const hb_model_cfg& cfg = c->cfg;
+  CtxExtra* ex = extra_of(c);
+
+  // ---- pack the descriptor into pinned staging, one H2D copy ----
+  Staging& st = ex->ring[ex->next];
+  ex->next = (ex->next + 1) % N_STAGING;
+  if (st.pending) {
+    if (cudaEventSynchronize(st.ev) != cudaSuccess) return HB_ERR_CUDA;
+    st.pending = false;
+  }
+  const int32_t T = d->n_tokens, R = d->n_segs;
+  size_t off = 0;
+  auto place = [&](size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes, 16);
+    return o;
+  };
+  const size_t o_tok = place(static_cast<size_t>(T) * 4), o_rseg = place(static_cast<size_t>(T) * 4),
+               o_rpos = place(static_cast<size_t>(T) * 4), o_segs = place(static_cast<size_t>(R) * sizeof(hb_seg)),
+               o_pages = place(static_cast<size_t>(d->n_page_ids) * 4),
+               o_lsrc = place(static_cast<size_t>(d->n_logit_rows) * 4);
+  int32_t* tok = reinterpret_cast<int32_t*>(st.host + o_tok);
+  int32_t* rseg = reinterpret_cast<int32_t*>(st.host + o_rseg);
+  int32_t* rpos = reinterpret_cast<int32_t*>(st.host + o_rpos);
+  hb_seg* segs = reinterpret_cast<hb_seg*>(st.host + o_segs);
+  int32_t* pages = reinterpret_cast<int32_t*>(st.host + o_pages);
+  int32_t* lsrc = reinterpret_cast<int32_t*>(st.host + o_lsrc);
+  memcpy(tok, d->token_ids, static_cast<size_t>(T) * 4);
+  memcpy(segs, d->segs, static_cast<size_t>(R) * sizeof(hb_seg));
+  if (d->n_page_ids) memcpy(pages, d->page_ids, static_cast<size_t>(d->n_page_ids) * 4);
+  std::vector<PoolItem> pitems;
+  int32_t part_at = 0;
+  for (int32_t r = 0; r < R; ++r) {
+    const hb_seg& sg = d->segs[r];
+    for (int32_t j = 0; j < sg.q_len; ++j) {
+      rseg[sg.q_start + j] = r;
+      rpos[sg.q_start + j] = sg.pos_start + j;
+    }
+    if (sg.logits_row >= 0) lsrc[sg.logits_row] = sg.q_start + sg.q_len - 1;
+    if (sg.kind == HB_KIND_EMBED_CHUNK) {
+      if (sg.pool_mode == HB_POOL_MEAN) {
+        const int32_t nb = (sg.q_len + POOL_ROWS - 1) / POOL_ROWS;
+        for (int32_t b = 0; b < nb; ++b) {
+          PoolItem it{};
+          it.seg = r;
+          it.row0 = sg.q_start + b * POOL_ROWS;
+          it.n_rows = std::min(POOL_ROWS, sg.q_len - b * POOL_ROWS);
+          it.block = b;
+          it.n_blocks = nb;
+          it.part_base = part_at;
+          pitems.push_back(it);
+        }
+        part_at += nb;
+      } else {  // last-token head: only the final chunk's last row is read
+        PoolItem it{};
+        it.seg = r;
+        it.row0 = sg.q_start + sg.q_len - 1;
+        it.n_rows = sg.is_final ? 1 : 0;
+        it.block = 0;
+        it.n_blocks = 1;
+        it.part_base = part_at;
+        pitems.push_back(it);
+        part_at += 1;
+      }
+    }
+  }
+  if (static_cast<int32_t>(pitems.size()) > ex->lay.max_pool_items) return HB_ERR_TOO_LARGE;
+  const size_t o_pitems = place(pitems.size() * sizeof(PoolItem));
+  if (off > c->desc_cap) return HB_ERR_TOO_LARGE;
+  if (!pitems.empty()) memcpy(st.host + o_pitems, pitems.data(), pitems.size() * sizeof(PoolItem));
+  if (cudaMemcpyAsync(c->desc_dev, st.host, off, cudaMemcpyHostToDevice, s) != cudaSuccess) return HB_ERR_CUDA;
+  if (cudaEventRecord(st.ev, s) != cudaSuccess) return HB_ERR_CUDA;
+  st.pending = true;
+
+  DeviceDesc& dd = c->dd;
+  dd.tok = reinterpret_cast<const int32_t*>(c->desc_dev + o_tok);
+  dd.row_seg = reinterpret_cast<const int32_t*>(c->desc_dev + o_rseg);
+  dd.row_pos = reinterpret_cast<const int32_t*>(c->desc_dev + o_rpos);
+  dd.segs = reinterpret_cast<const hb_seg*>(c->desc_dev + o_segs);
+  dd.pages = reinterpret_cast<const int32_t*>(c->desc_dev + o_pages);
+  dd.logit_src = reinterpret_cast<const int32_t*>(c->desc_dev + o_lsrc);
+  dd.attn_items = nullptr;
+  dd.pool_items = reinterpret_cast<const PoolItem*>(c->desc_dev + o_pitems);
+  dd.T = T;
+  dd.R = R;
+  dd.n_logit = d->n_logit_rows;
+  dd.n_attn_items = 0;
+  dd.n_pool_items = static_cast<int32_t>(pitems.size());
+
+  KvGeom kg;
+  kg.arena = static_cast<__nv_bfloat16*>(kv->arena);
+  kg.Hkv = cfg.n_kv_heads;
+  kg.P = cfg.page_size;
+  kg.Dh = cfg.head_dim;
+  kg.n_pages = kv->n_pages;
+  kg.page_stride = 2ll * cfg.n_kv_heads * cfg.page_size * cfg.head_dim;
+  kg.layer_stride = kg.page_stride * kv->n_pages;
+
+  const int n_qkv = (cfg.n_heads + 2 * cfg.n_kv_heads) * cfg.head_dim;
+  const int n_q = cfg.n_heads * cfg.head_dim;
+  int launches = 0;
+#define HB_TRY(expr)                  \
+  do {                                \
+    const int rc__ = (expr);          \
+    if (rc__ != HB_OK) return rc__;   \
+    ++launches;                       \
+  } while (0)
+
+  for (int l = 0; l < cfg.n_layers; ++l) {
+    const hb_layer_weights& lw = w->layers[l];
+    if (!lw.attn_norm || !lw.wqkv || !lw.wo || !lw.ffn_norm || !lw.w_gate_up || !lw.w_down) return HB_ERR_BAD_ARG;
+    hb_ctx::WMaps& wm = c->wmaps[l];
+    if (wm.key[0] != lw.wqkv || wm.key[1] != lw.wo || wm.key[2] != lw.w_gate_up || wm.key[3] != lw.w_down) {
+      wm.bn_qkv = hb_gemm_pick_bn(c->max_tokens, n_qkv, c->num_sms);
+      wm.bn_o = hb_gemm_pick_bn(c->max_tokens, cfg.d_model, c->num_sms);
+      wm.bn_gu = hb_gemm_pick_bn(c->max_tokens, 2 * cfg.d_ffn, c->num_sms);
+      wm.bn_down = wm.bn_o;
+      if ((rc = hb_tmap_2d_bf16(&wm.qkv, lw.wqkv, n_qkv, cfg.d_model, wm.bn_qkv)) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.o, lw.wo, cfg.d_model, n_q, wm.bn_o)) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.gu, lw.w_gate_up, 2ull * cfg.d_ffn, cfg.d_model, wm.bn_gu)) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, wm.bn_down)) != HB_OK) return rc;
+      wm.key[0] = lw.wqkv; wm.key[1] = lw.wo; wm.key[2] = lw.w_gate_up; wm.key[3] = lw.w_down;
+    }
+    if (l == 0) HB_TRY(hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
+    else HB_TRY(hb_launch_rmsnorm(c, lw.attn_norm, s));
+    GemmArgs ga;
+    ga.status = c->status;
+    ga.b_kshift = 0;
+    ga.M = T;
+    // QKV projection (fp32 out, rotated and appended next)
+    ga.C = c->qkv; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
+    HB_TRY(hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
+    HB_TRY(hb_launch_rope_append(c, kg, l, s));
+    HB_TRY(hb_launch_attention(c, kg, l, s));
+    // O projection, added to the residual stream
+    ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
+    HB_TRY(hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s));
+    HB_TRY(hb_launch_rmsnorm(c, lw.ffn_norm, s));
+    // gate/up projection with SwiGLU
+    ga.C = c->act; ga.N = 2 * cfg.d_ffn; ga.K = cfg.d_model; ga.ldc = cfg.d_ffn;
+    HB_TRY(hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s));
+    // down projection, added to the residual stream
+    ga.C = c->x; ga.N = cfg.d_model; ga.K = cfg.d_ffn; ga.ldc = cfg.d_model;
+    HB_TRY(hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s));
+  }
+  float* pool_sum = pool ? static_cast<float*>(pool->arena) : nullptr;
+  uint32_t* pool_meta = pool ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(pool->arena) +
+                                                           static_cast<size_t>(pool->n_slots) * cfg.d_model * 4)
+                             : nullptr;
+  rc = hb_launch_final(c, w->final_norm, pool_sum, pool_meta, n_slots, out_emb, s);
+  if (rc != HB_OK) return rc;
+  launches += (dd.n_logit > 0) + (dd.n_pool_items > 0);
+  if (dd.n_logit > 0) {
+    if (c->lm_key != w->lm_head) {
+      if ((rc = hb_tmap_2d_bf16(&c->tm_lm, w->lm_head, cfg.vocab, cfg.d_model, 128)) != HB_OK) return rc;
+      c->lm_key = w->lm_head;
+    }
+    GemmArgs ga;
+    ga.status = c->status;
+    ga.b_kshift = 1;  // A holds (hi, lo) 64-column blocks: each weight k-block is used twice
+    ga.M = dd.n_logit; ga.N = cfg.vocab; ga.K = 2 * cfg.d_model; ga.ldc = cfg.vocab; ga.C = out_logits;
+    HB_TRY(hb_gemm_launch(c->tm_logit_in, c->tm_lm, 128, HB_EPI_F32, ga, c->num_sms, s));
+  }
+#undef HB_TRY
+  c->last_launches = launches;
+  return HB_OK;
+}
+
+int hb_argmax(hb_ctx* c, const float* logits, int32_t n_rows, int32_t* out_tokens, void* stream) {
+  if (!c || n_rows < 0 || (n_rows > 0 && (!logits || !out_tokens))) return HB_ERR_BAD_ARG;
+  return hb_launch_argmax(logits, n_rows, c->cfg.vocab, out_tokens, static_cast<cudaStream_t>(stream));
+}
+
+int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
+  if (!c) return HB_ERR_BAD_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint32_t code = 0;
+  if (cudaMemcpyAsync(&code, c->status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return HB_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;
+  if (code != 0) {
+    if (cudaMemsetAsync(c->status, 0, 4, s) != cudaSuccess) return HB_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;
+  }
+  if (out_code) *out_code = code;
+  return code ? HB_ERR_DEVICE_STATUS : HB_OK;
+}
+
+int hb_last_launch_count(const hb_ctx* c, int32_t* out_count) {
+  if (!c || !out_count) return HB_ERR_BAD_ARG;
+  *out_count = c->last_launches;
+  return HB_OK;
+}
+
+int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+            void* stream) {
+  if (!c || !A || !B || !C || M < 1 || N < 8 || K < 8 || (N & 7) || (K & 7)) return HB_ERR_BAD_ARG;
+  if (epilogue < HB_EPI_BF16 || epilogue > HB_EPI_SWIGLU) return HB_ERR_BAD_ARG;
+  if (epilogue == HB_EPI_SWIGLU && (N & 15)) return HB_ERR_BAD_ARG;
+  if (reinterpret_cast<uintptr_t>(C) & 15u) return HB_ERR_BAD_ARG;
+  const int bn = hb_gemm_pick_bn(M, N, c->num_sms);
+  CUtensorMap ta, tb;
+  int rc = hb_tmap_2d_bf16(&ta, A, M, K, 128);
+  if (rc != HB_OK) return rc;
+  rc = hb_tmap_2d_bf16(&tb, B, N, K, bn);
+  if (rc != HB_OK) return rc;
+  GemmArgs ga;
+  ga.C = C; ga.M = M; ga.N = N; ga.K = K; ga.b_kshift = 0; ga.status = c->status;
+  ga.ldc = (epilogue == HB_EPI_SWIGLU) ? N / 2 : N;
+  return hb_gemm_launch(ta, tb, bn, epilogue, ga, c->num_sms, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

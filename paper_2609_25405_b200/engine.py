@@ -1,0 +1,141 @@
+"""Host-side glue around hb_mixed_step: request state, page / slot ownership and the
+batch unit of Section 3.2 (rows sorted by type: decode, prefill chunks, embedding chunks).
+
+This is bookkeeping only.  The batch-composition policy is the caller's: `Engine.step`
+takes the list of (request, rows) the scheduler chose for this iteration.
+"""
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class Request:
+    """One embedding or generation request as it moves through iterations."""
+
+    def __init__(self, kind, tokens, pool_mode=B.POOL_NONE):
+        assert kind in ("gen", "embed")
+        self.kind = kind
+        self.tokens = [int(t) for t in tokens]   # prompt / text; generated tokens are appended
+        self.n_prompt = len(self.tokens)
+        self.n_done = 0                          # tokens whose K/V is in the cache
+        self.pages = []
+        self.slot = -1
+        self.pool_mode = pool_mode
+        self.finished = False
+
+    @property
+    def in_decode(self):
+        return self.kind == "gen" and self.n_done >= self.n_prompt
+
+    def remaining(self):
+        return len(self.tokens) - self.n_done
+
+
+def build_batch(entries, page_size):
+    """entries: list of dicts(kind, tokens, pos_start, pages, pool_slot, pool_mode, is_final,
+    wants_logits).  Returns (Batch, order) with segments sorted by kind (stable) and
+    logits / embedding rows numbered in segment order; order[i] = index into `entries`."""
+    order = sorted(range(len(entries)), key=lambda i: entries[i]["kind"])
+    segs = np.zeros(len(entries), dtype=B.SEG_DTYPE)
+    toks, pages = [], []
+    n_l = n_e = 0
+    at = 0
+    for si, ei in enumerate(order):
+        e = entries[ei]
+        q = len(e["tokens"])
+        s = segs[si]
+        s["kind"] = e["kind"]
+        s["q_start"] = at
+        s["q_len"] = q
+        s["pos_start"] = e["pos_start"]
+        s["pt_start"] = len(pages)
+        s["pt_len"] = len(e["pages"])
+        s["pool_slot"] = e.get("pool_slot", -1)
+        s["pool_mode"] = e.get("pool_mode", B.POOL_NONE)
+        s["is_final"] = 1 if e.get("is_final") else 0
+        s["logits_row"] = -1
+        s["emb_row"] = -1
+        if e["kind"] == B.KIND_EMBED_CHUNK:
+            if e.get("is_final"):
+                s["emb_row"] = n_e
+                n_e += 1
+        elif e["kind"] == B.KIND_DECODE or e.get("is_final"):
+            s["logits_row"] = n_l
+            n_l += 1
+        toks.extend(int(t) for t in e["tokens"])
+        pages.extend(int(p) for p in e["pages"])
+        at += q
+    return B.Batch(toks, segs, pages, n_l, n_e), order
+
+
+class Engine:
+    def __init__(self, shape, weights, n_pages, n_slots, max_tokens, max_segs, max_pos,
+                 kv_fill=None, pool_fill=None, device="cuda"):
+        self.shape = shape
+        self.cfg = B.model_cfg(shape, max_pos)
+        self.weights = weights
+        self.max_tokens, self.max_segs = max_tokens, max_segs
+        max_page_ids = max_segs * ((max_pos + shape.page_size - 1) // shape.page_size)
+        self.ctx = B.Context(self.cfg, max_tokens, max_segs, max_page_ids)
+        self.kv = B.KvCache(self.cfg, n_pages, device, fill=kv_fill)
+        self.pool = B.Pool(self.cfg, n_slots, device, fill=pool_fill)
+        self.out_logits = torch.zeros((max_segs, shape.V), dtype=torch.float32, device=device)
+        self.out_emb = torch.zeros((max_segs, shape.d), dtype=torch.float32, device=device)
+
+    def _ensure_pages(self, req, n_tokens):
+        P = self.shape.page_size
+        need = (n_tokens + P - 1) // P - len(req.pages)
+        if need > 0:
+            req.pages.extend(self.kv.alloc(need))
+
+    def entry_for(self, req, rows):
+        """Descriptor entry for `rows` new rows of `req` (and reserve pages / slot)."""
+        assert rows >= 1 and rows <= req.remaining()
+        self._ensure_pages(req, req.n_done + rows)
+        toks = req.tokens[req.n_done:req.n_done + rows]
+        e = dict(tokens=toks, pos_start=req.n_done, pages=list(req.pages))
+        last = (req.n_done + rows == len(req.tokens))
+        if req.kind == "embed":
+            if req.slot < 0:
+                req.slot = self.pool.alloc()
+            e.update(kind=B.KIND_EMBED_CHUNK, pool_slot=req.slot, pool_mode=req.pool_mode, is_final=last)
+        elif req.in_decode:
+            assert rows == 1
+            e.update(kind=B.KIND_DECODE, is_final=True)
+        else:
+            e.update(kind=B.KIND_PREFILL_CHUNK, is_final=last)
+        return e
+
+    def step(self, work, stream=None):
+        """work: list of (Request, rows).  Enqueues one mixed step.  Returns
+        (batch, logits_rows {req: row}, emb_rows {req: row}); outputs land in
+        self.out_logits / self.out_emb once the stream is synchronised."""
+        entries = [self.entry_for(r, n) for r, n in work]
+        batch, order = build_batch(entries, self.shape.page_size)
+        self.ctx.mixed_step(batch, self.weights, self.kv, self.pool, self.out_logits, self.out_emb, stream)
+        lrows, erows = {}, {}
+        for si, ei in enumerate(order):
+            req, n = work[ei]
+            req.n_done += n
+            s = batch.segs[si]
+            if s["logits_row"] >= 0:
+                lrows[req] = int(s["logits_row"])
+            if s["emb_row"] >= 0:
+                erows[req] = int(s["emb_row"])
+                req.finished = True
+        return batch, lrows, erows
+
+    def release(self, req):
+        """Return a finished request's pages and pool slot."""
+        if req.pages:
+            self.kv.free(req.pages)
+            req.pages = []
+        if req.slot >= 0:
+            self.pool.free(req.slot)
+            req.slot = -1
+
+    def close(self):
+        self.ctx.close()
+        self.kv.close()
+        self.pool.close()

@@ -1,0 +1,74 @@
+"""Parity of the tcgen05 projection GEMM (through the C-ABI) with the oracle's definition."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ops
+from paper_2609_25405_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2609_25405_b200 import binding as B
+    c = B.Context(B.model_cfg(synth.SHAPES["tiny"], 64), 128, 8, 64)
+    yield c
+    c.close()
+
+
+def _bf16_exact(rng, shape, std):
+    a = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
+    return synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(a)).reshape(shape)
+
+
+# (M, N, K): several tiles, ragged M tail, N not a multiple of the tile, K not a multiple of 64,
+# a single row, more tiles than SMs (persistent loop + both TMEM accumulators), long K (ring wraps)
+SHAPES = [(128, 256, 64), (68, 768, 256), (300, 328, 200), (1, 1024, 256), (4, 1024, 512),
+          (515, 2048, 1024), (2500, 3072, 256), (256, 256, 4096), (4096, 1536, 512)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("epi", ["f32", "bf16", "resid", "swiglu"])
+def test_gemm_matches_oracle(ctx, M, N, K, epi):
+    from paper_2609_25405_b200 import binding as B
+    if epi == "swiglu" and N % 16:
+        pytest.skip("swiglu needs N % 16 == 0")
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    A = _bf16_exact(rng, (M, K), 1.0)
+    Bm = _bf16_exact(rng, (N, K), 0.05)
+    dA, dB = B.bf16_from_f32(A), B.bf16_from_f32(Bm)
+    scale = 0.05 * np.sqrt(K)
+    if epi == "f32":
+        out = torch.full((M + 1, N), 777.0, dtype=torch.float32, device="cuda")
+        ctx.gemm(dA, dB, out, M, N, K, B.EPI_F32)
+        ref = ops.projection(A, Bm, "plain")
+        tol = 2e-5 * scale * np.sqrt(K) + 1e-6
+    elif epi == "bf16":
+        out = torch.full((M + 1, N), 777.0, dtype=torch.bfloat16, device="cuda")
+        ctx.gemm(dA, dB, out, M, N, K, B.EPI_BF16)
+        ref = ops.projection(A, Bm, "plain")
+        tol = None
+    elif epi == "resid":
+        C0 = rng.standard_normal((M + 1, N), dtype=np.float32)
+        out = torch.from_numpy(C0.copy()).cuda()
+        ctx.gemm(dA, dB, out, M, N, K, B.EPI_RESID_F32)
+        ref = ops.projection(A, Bm, "resid", C0[:M])
+        tol = 2e-5 * scale * np.sqrt(K) + 1e-5
+    else:
+        out = torch.full((M + 1, N // 2), 777.0, dtype=torch.bfloat16, device="cuda")
+        ctx.gemm(dA, dB, out, M, N, K, B.EPI_SWIGLU)
+        ref = ops.projection(A, Bm, "swiglu")
+        tol = None
+    assert ctx.status_poll() == 0
+    got = out.float().cpu().numpy().astype(np.float64)
+    if tol is None:   # bf16 output: one rounding of the fp32 result (2^-9 relative) + accumulation noise
+        err = np.abs(got[:M] - ref)
+        assert np.all(err <= np.abs(ref) * 2.0 ** -8 + 2e-5 * scale * np.sqrt(K) + 1e-6), err.max()
+    else:
+        assert np.max(np.abs(got[:M] - ref)) <= tol
+    # the row after the last one is never touched
+    if epi == "resid":
+        assert np.array_equal(got[M], C0[M].astype(np.float64))
+    else:
+        assert np.all(got[M] == 777.0)
