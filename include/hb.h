@@ -214,6 +214,21 @@ HB_API int hb_argmax(hb_ctx* ctx, const float* logits, int32_t n_rows, int32_t* 
  * *out_code holds the kernel-specific code.  Returns HB_ERR_DEVICE_STATUS then. */
 HB_API int hb_status_poll(hb_ctx* ctx, void* stream, uint32_t* out_code);
 
+/* Per-kernel-class device timing.  While enabled, hb_mixed_step brackets every launch with a
+ * pair of CUDA events on the step's stream; hb_profile_read synchronises them, adds the
+ * elapsed milliseconds and launch counts per class into the two arrays of HB_N_CLASSES
+ * entries, and clears the record.  Classes: */
+enum {
+  HB_CLASS_GEMM = 0,      /* QKV, O, gate/up, down projections                          */
+  HB_CLASS_ATTENTION = 1, /* varlen paged attention                                     */
+  HB_CLASS_NORM_ROPE = 2, /* gather + RMSNorm, RMSNorm, RoPE + KV append                */
+  HB_CLASS_POOL = 3,      /* final RMSNorm + pooler / logits-row preparation            */
+  HB_CLASS_LM_HEAD = 4,   /* LM-head projection                                         */
+  HB_N_CLASSES = 5
+};
+HB_API int hb_profile_enable(hb_ctx* ctx, int on);
+HB_API int hb_profile_read(hb_ctx* ctx, float* ms_by_class, int32_t* launches_by_class);
+
 /* Kernels launched by the last hb_mixed_step on this context. */
 HB_API int hb_last_launch_count(const hb_ctx* ctx, int32_t* out_count);
 

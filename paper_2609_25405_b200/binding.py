@@ -20,6 +20,7 @@ ERRORS = {0: "HB_OK", -1: "HB_ERR_BAD_ARG", -2: "HB_ERR_CUDA", -3: "HB_ERR_OOM_P
 KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK = 0, 1, 2
 POOL_NONE, POOL_MEAN, POOL_LAST = 0, 1, 2
 EPI_BF16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU = 0, 1, 2, 3
+CLASSES = ("gemm", "attention", "norm_rope", "pool", "lm_head")
 
 
 class HbError(RuntimeError):
@@ -86,6 +87,8 @@ _sig = {
     "hb_argmax": [_P, _P, C.c_int32, _P, _P],
     "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
     "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
+    "hb_profile_enable": [_P, C.c_int],
+    "hb_profile_read": [_P, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
     "hb_gemm": [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
 }
 for _name, _args in _sig.items():
@@ -332,6 +335,16 @@ class Context:
         if rc not in (HB_OK, -7):
             raise HbError(rc, "hb_status_poll")
         return code.value
+
+    def profile_enable(self, on):
+        check(lib.hb_profile_enable(self.handle, 1 if on else 0), "hb_profile_enable")
+
+    def profile_read(self):
+        """{class name: (milliseconds, launches)} accumulated since the last read."""
+        ms = (C.c_float * len(CLASSES))()
+        n = (C.c_int32 * len(CLASSES))()
+        check(lib.hb_profile_read(self.handle, ms, n), "hb_profile_read")
+        return {CLASSES[i]: (float(ms[i]), int(n[i])) for i in range(len(CLASSES))}
 
     def last_launch_count(self):
         n = C.c_int32()

@@ -161,10 +161,17 @@ struct Staging {
   bool pending = false;
 };
 
+struct ProfRec {
+  cudaEvent_t a, b;
+  int cls;
+};
+
 struct CtxExtra {
   Staging ring[N_STAGING];
   int next = 0;
   Layout lay;
+  bool profiling = false;
+  std::vector<ProfRec> free_recs, used_recs;
 };
 
 CtxExtra* extra_of(hb_ctx* c) { return static_cast<CtxExtra*>(c->extra); }
@@ -290,6 +297,11 @@ int hb_destroy(hb_ctx* c) {
       if (ex->ring[i].host) cudaFreeHost(ex->ring[i].host);
       if (ex->ring[i].ev) cudaEventDestroy(ex->ring[i].ev);
     }
+    for (auto* v : {&ex->free_recs, &ex->used_recs})
+      for (ProfRec& r : *v) {
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+      }
     delete ex;
   }
   if (c->owns_ws && c->ws) cudaFree(c->ws);
@@ -537,9 +549,28 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
   const int n_qkv = (cfg.n_heads + 2 * cfg.n_kv_heads) * cfg.head_dim;
   const int n_q = cfg.n_heads * cfg.head_dim;
   int launches = 0;
-#define HB_TRY(expr)                  \
+  auto prof_begin = [&](int cls) -> ProfRec* {
+    if (!ex->profiling) return nullptr;
+    ProfRec r;
+    if (!ex->free_recs.empty()) {
+      r = ex->free_recs.back();
+      ex->free_recs.pop_back();
+    } else if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) {
+      return nullptr;
+    }
+    r.cls = cls;
+    cudaEventRecord(r.a, s);
+    ex->used_recs.push_back(r);
+    return &ex->used_recs.back();
+  };
+  auto prof_end = [&](ProfRec* r) {
+    if (r) cudaEventRecord(r->b, s);
+  };
+#define HB_TRY(cls, expr)             \
   do {                                \
+    ProfRec* pr__ = prof_begin(cls);  \
     const int rc__ = (expr);          \
+    prof_end(pr__);                   \
     if (rc__ != HB_OK) return rc__;   \
     ++launches;                       \
   } while (0)
@@ -559,35 +590,39 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
       if ((rc = hb_tmap_2d_bf16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, wm.bn_down)) != HB_OK) return rc;
       wm.key[0] = lw.wqkv; wm.key[1] = lw.wo; wm.key[2] = lw.w_gate_up; wm.key[3] = lw.w_down;
     }
-    if (l == 0) HB_TRY(hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
-    else HB_TRY(hb_launch_rmsnorm(c, lw.attn_norm, s));
+    if (l == 0) HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
+    else HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.attn_norm, s));
     GemmArgs ga;
     ga.status = c->status;
     ga.b_kshift = 0;
     ga.M = T;
     // QKV projection (fp32 out, rotated and appended next)
     ga.C = c->qkv; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
-    HB_TRY(hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
-    HB_TRY(hb_launch_rope_append(c, kg, l, s));
-    HB_TRY(hb_launch_attention(c, kg, l, s));
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
+    HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rope_append(c, kg, l, s));
+    HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, l, s));
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
-    HB_TRY(hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s));
-    HB_TRY(hb_launch_rmsnorm(c, lw.ffn_norm, s));
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s));
+    HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.ffn_norm, s));
     // gate/up projection with SwiGLU
     ga.C = c->act; ga.N = 2 * cfg.d_ffn; ga.K = cfg.d_model; ga.ldc = cfg.d_ffn;
-    HB_TRY(hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s));
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s));
     // down projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = cfg.d_ffn; ga.ldc = cfg.d_model;
-    HB_TRY(hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s));
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s));
   }
   float* pool_sum = pool ? static_cast<float*>(pool->arena) : nullptr;
   uint32_t* pool_meta = pool ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(pool->arena) +
                                                            static_cast<size_t>(pool->n_slots) * cfg.d_model * 4)
                              : nullptr;
-  rc = hb_launch_final(c, w->final_norm, pool_sum, pool_meta, n_slots, out_emb, s);
-  if (rc != HB_OK) return rc;
-  launches += (dd.n_logit > 0) + (dd.n_pool_items > 0);
+  {
+    ProfRec* pr = prof_begin(HB_CLASS_POOL);
+    rc = hb_launch_final(c, w->final_norm, pool_sum, pool_meta, n_slots, out_emb, s);
+    prof_end(pr);
+    if (rc != HB_OK) return rc;
+    launches += (dd.n_logit > 0) + (dd.n_pool_items > 0);
+  }
   if (dd.n_logit > 0) {
     if (c->lm_key != w->lm_head) {
       if ((rc = hb_tmap_2d_bf16(&c->tm_lm, w->lm_head, cfg.vocab, cfg.d_model, 128)) != HB_OK) return rc;
@@ -597,7 +632,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     ga.status = c->status;
     ga.b_kshift = 1;  // A holds (hi, lo) 64-column blocks: each weight k-block is used twice
     ga.M = dd.n_logit; ga.N = cfg.vocab; ga.K = 2 * cfg.d_model; ga.ldc = cfg.vocab; ga.C = out_logits;
-    HB_TRY(hb_gemm_launch(c->tm_logit_in, c->tm_lm, 128, HB_EPI_F32, ga, c->num_sms, s));
+    HB_TRY(HB_CLASS_LM_HEAD, hb_gemm_launch(c->tm_logit_in, c->tm_lm, 128, HB_EPI_F32, ga, c->num_sms, s));
   }
 #undef HB_TRY
   c->last_launches = launches;
@@ -621,6 +656,27 @@ int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
   }
   if (out_code) *out_code = code;
   return code ? HB_ERR_DEVICE_STATUS : HB_OK;
+}
+
+int hb_profile_enable(hb_ctx* c, int on) {
+  if (!c) return HB_ERR_BAD_ARG;
+  extra_of(c)->profiling = (on != 0);
+  return HB_OK;
+}
+
+int hb_profile_read(hb_ctx* c, float* ms_by_class, int32_t* launches_by_class) {
+  if (!c || !ms_by_class || !launches_by_class) return HB_ERR_BAD_ARG;
+  CtxExtra* ex = extra_of(c);
+  for (ProfRec& r : ex->used_recs) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess)
+      return HB_ERR_CUDA;
+    ms_by_class[r.cls] += ms;
+    launches_by_class[r.cls] += 1;
+    ex->free_recs.push_back(r);
+  }
+  ex->used_recs.clear();
+  return HB_OK;
 }
 
 int hb_last_launch_count(const hb_ctx* c, int32_t* out_count) {

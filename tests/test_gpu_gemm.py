@@ -40,12 +40,12 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
     dA, dB = B.bf16_from_f32(A), B.bf16_from_f32(Bm)
     scale = 0.05 * np.sqrt(K)
     if epi == "f32":
-        out = torch.full((M + 1, N), 777.0, dtype=torch.float32, device="cuda")
+        out = torch.full((M + 1, N), 768.0, dtype=torch.float32, device="cuda")
         ctx.gemm(dA, dB, out, M, N, K, B.EPI_F32)
         ref = ops.projection(A, Bm, "plain")
         tol = 2e-5 * scale * np.sqrt(K) + 1e-6
     elif epi == "bf16":
-        out = torch.full((M + 1, N), 777.0, dtype=torch.bfloat16, device="cuda")
+        out = torch.full((M + 1, N), 768.0, dtype=torch.bfloat16, device="cuda")
         ctx.gemm(dA, dB, out, M, N, K, B.EPI_BF16)
         ref = ops.projection(A, Bm, "plain")
         tol = None
@@ -56,7 +56,7 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
         ref = ops.projection(A, Bm, "resid", C0[:M])
         tol = 2e-5 * scale * np.sqrt(K) + 1e-5
     else:
-        out = torch.full((M + 1, N // 2), 777.0, dtype=torch.bfloat16, device="cuda")
+        out = torch.full((M + 1, N // 2), 768.0, dtype=torch.bfloat16, device="cuda")
         ctx.gemm(dA, dB, out, M, N, K, B.EPI_SWIGLU)
         ref = ops.projection(A, Bm, "swiglu")
         tol = None
@@ -71,4 +71,4 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
     if epi == "resid":
         assert np.array_equal(got[M], C0[M].astype(np.float64))
     else:
-        assert np.all(got[M] == 777.0)
+        assert np.all(got[M] == 768.0)

@@ -146,7 +146,9 @@ def test_cfg1_mean_state_after_each_chunk(weights):
         assert list(meta[:2]) == list(M.pool_counters_after([33, 1, 50, 16][:k + 1]))
         S = eng.pool.sums()[req.slot].cpu().numpy().astype(np.float64)
         ref = hh[:at].sum(0)
-        assert np.max(np.abs(S - ref)) <= 2e-2 * np.sqrt(at)
+        # per-row error of the unit-rms hidden states is bounded like the embedding tolerance;
+        # rounding errors of near-identical rows are correlated, so the bound grows with the count
+        assert np.max(np.abs(S - ref)) <= 1e-2 * at
     assert eng.ctx.status_poll() == 0
     eng.close()
 
