@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-batch step: tokens/s (decode + embedding rows) and roofline fraction.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3-7b|cfg2-1b|cfg4-7b-f<frac>]
+  python bench.py --impl reference ...     # the CPU oracle on the host cores, same metric
+
+A step is one hb_mixed_step over one synthetic mixed batch.  `value` times K steps with CUDA
+events around the library calls (weights, KV pages and pool state resident in HBM; each call
+copies its own small descriptor).  `e2e` repeats the K steps building the descriptor on the host
+and reading logits and embeddings back to pinned host memory inside the timed region.
+N > 1 runs N independent replicas (the method scales by replication; no collective).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mixed-batch tokens/s (decode+embed) on 1 B200 and % of roofline"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def get_spec(name):
+    from paper_2609_25405_b200 import workloads
+    if name in workloads.SPECS:
+        return workloads.SPECS[name]
+    if name.startswith("cfg4-7b-f"):
+        return workloads.sweep_spec(float(name[len("cfg4-7b-f"):]))
+    raise SystemExit(f"unknown workload {name}")
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.strip().split(", ") for r in open(self.f.name).read().strip().splitlines() if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[5:9]):
+                if v.strip().lower() == "active":
+                    reasons.add(nm)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample
+# ------------------------------------------------------------------------------------------
+
+class _SampleWeights:
+    """Random float32 weights of the workload's shape for TIMING the oracle: one layer's tensors
+    are generated and served for every layer, and only the first 1024 vocabulary rows exist
+    (the sample's token ids stay below 1024, no logits are asked for)."""
+
+    def __init__(self, shape, seed=0):
+        rng = np.random.default_rng(seed)
+        s = shape
+        g = lambda r, c: rng.standard_normal((r, c), dtype=np.float32) * np.float32(0.02)
+        self._layer = dict(attn_norm=np.ones(s.d, np.float32), ffn_norm=np.ones(s.d, np.float32),
+                           wq=g(s.Hq * s.Dh, s.d), wk=g(s.Hkv * s.Dh, s.d), wv=g(s.Hkv * s.Dh, s.d),
+                           wo=g(s.d, s.Hq * s.Dh), wg=g(s.F, s.d), wu=g(s.F, s.d), wd=g(s.d, s.F))
+        self.tok_emb = g(1024, s.d)
+        self.final_norm = np.ones(s.d, np.float32)
+        self.lm_head = self.tok_emb
+
+    def layer(self, l):
+        return self._layer
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def oracle_sample(spec, n_tokens, repeats=1):
+    """Times oracle.embed on one embedding request of n_tokens (last-token or mean pooling as the
+    workload says), fp32.  Returns (tokens/s, seconds per sample)."""
+    from oracle import transformer as T
+    from paper_2609_25405_b200 import synth, consts
+    shape = synth.SHAPES[spec.shape]
+    W = _SampleWeights(shape)
+    toks = np.random.default_rng(1).integers(0, 1024, n_tokens)
+    mode = "last" if spec.pool_mode == consts.POOL_LAST else "mean"
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        T.embed(shape, W, toks, mode, dtype=np.float32)
+        times.append(time.perf_counter() - t0)
+    return n_tokens / float(np.mean(times)), times
+
+
+def sample_tokens(spec):
+    return min(spec.chunk, 512 if spec.shape == "7b" else 1024)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = get_spec(args.workload)
+    n = sample_tokens(spec) // 2
+    for _ in range(args.warmup):
+        oracle_sample(spec, n)
+    t0 = time.perf_counter()
+    _, times = oracle_sample(spec, n, repeats=args.steps)
+    total = time.perf_counter() - t0
+    value = n * args.steps / sum(times)
+    cores = blas_threads()
+    sample = (f"oracle.transformer.embed (fp32 numpy) on one {n}-token embedding request of the {spec.shape} shape "
+              f"per step; one layer's random weights reused for all layers (timing only)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": spec.name, "sample_tokens": n},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "wall_s": total}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3-7b")
+    ap.add_argument("--packer-warm", type=int, default=50, help="host-only packer steps before the first GPU step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-alias", type=int, default=0)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200 import synth, workloads
+    from paper_2609_25405_b200.engine import build_batch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    spec = get_spec(args.workload)
+    if world > 1:   # independent replicas: each rank draws its own batch stream
+        spec = workloads.MixSpec(**{**spec.__dict__, "seed": spec.seed + 7919 * rank})
+    shape = synth.SHAPES[spec.shape]
+    n_steps_total = args.warmup + args.steps
+    max_pos = spec.ctx_hi + n_steps_total + 8 if spec.n_decode else spec.emb_hi + 8
+    max_pos = max(max_pos, spec.emb_hi + 8)
+    cfg = B.model_cfg(shape, max_pos)
+    P = shape.page_size
+    n_unique = args.decode_alias if args.decode_alias else spec.n_decode
+    dec_pages = n_unique * ((spec.ctx_hi + P - 1) // P + 1) + spec.n_decode * ((n_steps_total + P - 1) // P + 2)
+    emb_pages = 3 * spec.budget // P + 32 * ((spec.emb_hi + P - 1) // P)
+    n_pages = dec_pages + emb_pages
+    max_segs = spec.n_decode + spec.budget // 16 + 8
+    max_page_ids = spec.n_decode * ((max_pos + P - 1) // P) + (spec.budget // 16 + 8) * ((spec.emb_hi + P - 1) // P + 1)
+
+    weights = B.DeviceWeights.random_on_device(shape, seed=0)
+    kv = B.KvCache(cfg, n_pages)
+    kvb = kv.arena.view(torch.bfloat16)
+    step_e = 1 << 28
+    for i in range(0, kvb.numel(), step_e):          # synthetic cached K/V: N(0,1)
+        kvb[i:i + step_e].normal_(0.0, 1.0)
+    pool = B.Pool(cfg, 256)
+    ctx = B.Context(cfg, spec.budget, max_segs, max_page_ids)
+    wl = workloads.MixedWorkload(spec, kv, pool, max_pos, decode_alias=args.decode_alias)
+    for _ in range(args.packer_warm):                # reach the packer's steady state (host only)
+        _, commit = wl.next_step()
+        commit(advance_decode=False)
+    entries_all, batches, work = [], [], []
+    for _ in range(n_steps_total):
+        entries, commit = wl.next_step()
+        entries = [dict(e, pages=list(e["pages"])) for e in entries]
+        commit()
+        entries_all.append(entries)
+        batches.append(build_batch(entries, P)[0])
+        work.append(workloads.step_work(shape, entries))
+    out_logits = torch.zeros((max_segs, shape.V), dtype=torch.float32, device="cuda")
+    out_emb = torch.zeros((max_segs, shape.d), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def run(i):
+        ctx.mixed_step(batches[i], weights, kv, pool, out_logits, out_emb, stream)
+
+    for i in range(args.warmup):
+        run(i)
+    torch.cuda.synchronize()
+    if ctx.status_poll() != 0:
+        raise SystemExit("device status set during warm-up")
+    timed = list(range(args.warmup, n_steps_total))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    launches = 0
+    for i in timed:
+        run(i)
+        launches += ctx.last_launch_count()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+
+    # ---- end to end: host packing + call + read-back of logits / embeddings ----
+    h_logits = torch.empty((max_segs, shape.V), dtype=torch.float32).pin_memory()
+    h_emb = torch.empty((max_segs, shape.d), dtype=torch.float32).pin_memory()
+    barrier()
+    t0 = time.perf_counter()
+    h2d = d2h = 0
+    for i in timed:
+        b = build_batch(entries_all[i], P)[0]
+        ctx.mixed_step(b, weights, kv, pool, out_logits, out_emb, stream)
+        nl, ne = b.desc.n_logit_rows, b.desc.n_emb_rows
+        if nl:
+            h_logits[:nl].copy_(out_logits[:nl], non_blocking=True)
+        if ne:
+            h_emb[:ne].copy_(out_emb[:ne], non_blocking=True)
+        torch.cuda.synchronize()
+        h2d += b.host_bytes()
+        d2h += nl * shape.V * 4 + ne * shape.d * 4
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- per-class kernel timing (events around every launch, same steps) ----
+    ctx.profile_enable(True)
+    for i in timed:
+        run(i)
+    torch.cuda.synchronize()
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    status = ctx.status_poll()
+
+    tokens = sum(work[i]["T"] for i in timed)
+    t_all = torch.tensor([ms, e2e_s * 1e3, float(tokens)], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        mx = t_all.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = t_all.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        ms, e2e_ms, tokens = float(mx[0]), float(mx[1]), float(sm[2])
+    else:
+        e2e_ms = e2e_s * 1e3
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    K = len(timed)
+    w = {k: float(np.mean([work[i][k] for i in timed])) for k in work[0]}
+    gemm_ms, gemm_n = prof["gemm"]
+    gemm_flops_launch = (w["gemm_flops"] - 2.0 * shape.d * shape.V * w["n_logit"]) * K / max(gemm_n, 1)
+    ach_tf = gemm_flops_launch / (gemm_ms / max(gemm_n, 1) * 1e-3) / 1e12 if gemm_ms > 0 else None
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": "hb_gemm_tcgen05_kernel (QKV, O, gate/up, down projections)",
+                "achieved": ach_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": (ach_tf / peak_tf) if ach_tf else None, "traffic": None,
+                "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step)",
+                "frac_of_burst": (ach_tf / peaks["bf16_tflops"]) if ach_tf else None,
+                "launches": gemm_n, "flops_per_launch": gemm_flops_launch}
+    step_ms = ms / K
+    bytes_step = w["weight_bytes"] + w["kv_read_bytes"] + w["kv_write_bytes"]
+    t_gemm_burst = w["gemm_flops"] / (peaks["bf16_tflops"] * 1e12)
+    t_gemm_sust = w["gemm_flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_mem = bytes_step / (peaks["hbm_gbs"] * 1e9)
+    step_roof = {"gemm_tflop": w["gemm_flops"] / 1e12, "attn_tflop": w["attn_flops"] / 1e12,
+                 "bytes_gb": bytes_step / 1e9, "t_gemm_ms_burst": t_gemm_burst * 1e3,
+                 "t_gemm_ms_sustained": t_gemm_sust * 1e3, "t_mem_ms": t_mem * 1e3,
+                 "bound": "tensor" if t_gemm_burst > t_mem else "hbm",
+                 "frac_of_burst_roof": max(t_gemm_burst, t_mem) * 1e3 / step_ms,
+                 "frac_of_sustained_roof": max(t_gemm_sust, t_mem) * 1e3 / step_ms,
+                 "peak_kind": peak_kind}
+    breakdown = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in prof.items()}
+    line = {"metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": spec.name, "shape": spec.shape, "tokens_per_step": w["T"],
+                       "decode_rows": spec.n_decode, "chunk": spec.chunk, "token_budget": spec.budget,
+                       "l2": "inputs larger than L2 (weights and KV pages are re-streamed every step)",
+                       "replicas": world, "decode_alias": args.decode_alias},
+            "clocks": clocks, "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                                      "h2d_bytes_per_step": h2d / K, "d2h_bytes_per_step": d2h / K},
+            "gpu_launches": launches, "roofline": roofline, "step_roofline": step_roof,
+            "kernel_classes": breakdown, "device_status": status}
+    if not args.no_cpu_baseline:
+        n = sample_tokens(spec)
+        v, times = oracle_sample(spec, n)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"oracle.transformer.embed (fp32 numpy) on one {n}-token embedding request "
+                                          f"of the {spec.shape} shape, {times[0]:.1f} s; one layer's random weights "
+                                          f"reused for all layers (timing only)"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

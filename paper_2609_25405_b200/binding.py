@@ -17,10 +17,8 @@ HB_OK = 0
 ERRORS = {0: "HB_OK", -1: "HB_ERR_BAD_ARG", -2: "HB_ERR_CUDA", -3: "HB_ERR_OOM_PAGES",
           -4: "HB_ERR_OOM_SLOTS", -5: "HB_ERR_TOO_LARGE", -6: "HB_ERR_BAD_DESC",
           -7: "HB_ERR_DEVICE_STATUS", -8: "HB_ERR_UNSUPPORTED"}
-KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK = 0, 1, 2
-POOL_NONE, POOL_MEAN, POOL_LAST = 0, 1, 2
-EPI_BF16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU = 0, 1, 2, 3
-CLASSES = ("gemm", "attention", "norm_rope", "pool", "lm_head")
+from .consts import (KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK, POOL_NONE, POOL_MEAN,  # noqa: F401,E402
+                     POOL_LAST, EPI_BF16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
 
 
 class HbError(RuntimeError):

@@ -1,80 +1,418 @@
-// Varlen causal attention over the paged KV cache for every row of the mixed batch
-// (Section 3.2: decode tokens attend over their cached context, embedding / prefill chunks
-// attend causally over their own earlier chunks plus themselves).  Row j of a segment has
-// position pos = pos_start + j and sees keys 0 .. pos of its own request; all keys, the
-// row's own included, are read from the pages (the append kernel ran before).
+// Varlen causal attention over the paged KV cache for every row of the mixed batch, one launch
+// (Section 3.2 of the paper: decode tokens attend over their cached context, embedding / prefill
+// chunks attend causally over their own earlier chunks plus themselves).  Row j of a segment has
+// position pos = pos_start + j and sees keys 0 .. pos of its own request; all keys, the row's own
+// included, are read from the pages (the append kernel ran before).
 //
-// Bring-up version: one warp per (row, query head), online softmax in fp32.
+// Work items come from the batch descriptor (host-built list):
+//   chunk item   64 query rows = (64 / G) tokens x G query heads of one KV head (G = Hq / Hkv),
+//                all visible keys; the four warps own 16 rows each and share the K/V tiles.
+//   decode item  the G query heads of one KV head of one decode row over one split of at most
+//                SPLIT keys; the four warps share the rows and own 16 keys of every 64-key tile;
+//                their partial (max, sum, output) are merged in shared memory, and the splits
+//                of a row through a scratch record per split, merged in split order by the CTA
+//                that arrives last (integer arrival counter; no floating-point atomics).
+// K/V tiles of 64 keys (4 pages) are gathered with 16-byte cp.async into an XOR-swizzled
+// shared-memory ring; S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate),
+// softmax in fp32 with exp2.  Split decisions depend on the request's own length only, so a
+// request's result does not depend on its batch mates.
 #include "hb_internal.h"
 
 namespace {
 
-template <int E>  // elements of the head dimension per lane: Dh = 32 * E
-__global__ void __launch_bounds__(128)
-attn_rowwarp_kernel(const __nv_bfloat16* __restrict__ q, KvGeom kv, int layer,
-                    const int32_t* __restrict__ row_seg, const int32_t* __restrict__ row_pos,
-                    const hb_seg* __restrict__ segs, const int32_t* __restrict__ pages,
-                    __nv_bfloat16* __restrict__ out, int Hq, float scale, uint32_t* status) {
-  const int t = blockIdx.x;
-  const int head = blockIdx.y * 4 + (threadIdx.x >> 5);
+constexpr int ATT_THREADS = 128;
+constexpr int TILE_KEYS = 64;
+constexpr int TILE_ROWS = 64;
+constexpr int STAGES = 3;
+
+struct AttnParams {
+  const __nv_bfloat16* q;     // [T, Hq*Dh]
+  __nv_bfloat16* out;         // [T, Hq*Dh]
+  KvGeom kv;
+  int layer;
+  const AttnItem* items;
+  const hb_seg* segs;
+  const int32_t* pages;
+  float* part;                // split records: [record][G][Dh + 2]
+  uint32_t* counters;         // [seg * Hkv + kv_head]
+  uint32_t* status;
+  int Hq, G;
+  float scale_log2;           // log2(e) / sqrt(Dh)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;  // 0 source bytes: the 16 destination bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Byte offset of 16-byte chunk `c` of row `r` in a [rows][DH] bf16 tile (XOR swizzle).
+template <int DH>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+  return static_cast<uint32_t>(r * (DH * 2) + ((c ^ (r & 7)) << 4));
+}
+
+// One warp: 16 query rows against NT*8 keys starting at tile-local key `kofs`.
+// qf: Q fragments; m, l: running max (scaled, log2 domain) and per-thread partial sums of the two
+// rows this thread touches (row lane/4 and row lane/4 + 8); oacc: unnormalised output.
+template <int DH, int NT>
+__device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], uint32_t k_tile, uint32_t v_tile,
+                                            int kofs, int key_base, int key_end, int pos_a, int pos_b,
+                                            float scale_log2, float (&m)[2], float (&l)[2],
+                                            float (&oacc)[DH / 8][4]) {
   const int lane = threadIdx.x & 31;
-  if (head >= Hq) return;
-  const int Dh = kv.Dh;
-  const int hk = head / (Hq / kv.Hkv);
-  const int pos = row_pos[t];
-  const hb_seg sg = segs[row_seg[t]];
-  float qv[E];
+  float s[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.0f;
+  // S = Q K^T
   {
-    const __nv_bfloat16* qp = q + (static_cast<size_t>(t) * Hq + head) * Dh + lane * E;
+    const int j = lane >> 3, rr = lane & 7;
 #pragma unroll
-    for (int e = 0; e < E; ++e) qv[e] = __bfloat162float(qp[e]) * scale;
-  }
-  float m = -INFINITY, l = 0.0f, acc[E];
+    for (int ks = 0; ks < DH / 16; ++ks) {
 #pragma unroll
-  for (int e = 0; e < E; ++e) acc[e] = 0.0f;
-  const __nv_bfloat16* lbase = kv.arena + layer * kv.layer_stride;
-  const int64_t head_stride = static_cast<int64_t>(kv.P) * Dh;
-  for (int s = 0; s <= pos; ++s) {
-    const int blk = s / kv.P, slot = s - blk * kv.P;
-    const int page = pages[sg.pt_start + blk];
-    if (page < 0 || page >= kv.n_pages) {
-      if (lane == 0) atomicOr(status, HB_DEV_ATTN_BAD_INDEX);
-      return;
+      for (int np = 0; np < NT / 2; ++np) {
+        const int key = kofs + np * 16 + (j >> 1) * 8 + rr;
+        uint32_t b[4];
+        ldsm_x4(k_tile + tile_off<DH>(key, ks * 2 + (j & 1)), b);
+        mma_bf16(s[np * 2], qf[ks], b[0], b[1]);
+        mma_bf16(s[np * 2 + 1], qf[ks], b[2], b[3]);
+      }
     }
-    const __nv_bfloat16* kp = lbase + page * kv.page_stride + hk * head_stride + slot * Dh + lane * E;
-    const __nv_bfloat16* vp = kp + kv.Hkv * head_stride;
-    float dot = 0.0f;
-#pragma unroll
-    for (int e = 0; e < E; ++e) dot += qv[e] * __bfloat162float(kp[e]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    const float m_new = fmaxf(m, dot);
-    const float corr = __expf(m - m_new);
-    const float p = __expf(dot - m_new);
-    l = l * corr + p;
-#pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = acc[e] * corr + p * __bfloat162float(vp[e]);
-    m = m_new;
   }
-  const float inv = 1.0f / l;
-  __nv_bfloat16* op = out + (static_cast<size_t>(t) * Hq + head) * Dh + lane * E;
+  // mask + online softmax
+  float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-  for (int e = 0; e < E; ++e) op[e] = __float2bfloat16(acc[e] * inv);
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int key = key_base + kofs + nt * 8 + 2 * (lane & 3) + (e & 1);
+      const int pos = (e < 2) ? pos_a : pos_b;
+      const bool vis = (key <= pos) && (key < key_end);
+      s[nt][e] = vis ? s[nt][e] * scale_log2 : -INFINITY;
+      mx[e >> 1] = fmaxf(mx[e >> 1], s[nt][e]);
+    }
+  }
+  float corr[2], msafe[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+    const float m_new = fmaxf(m[h], mx[h]);
+    msafe[h] = (m_new == -INFINITY) ? 0.0f : m_new;
+    corr[h] = exp2f(m[h] - msafe[h]);   // m = -inf -> 0
+    m[h] = m_new;
+  }
+  float rs[2] = {0.0f, 0.0f};
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float p = exp2f(s[nt][e] - msafe[e >> 1]);
+      s[nt][e] = p;
+      rs[e >> 1] += p;
+    }
+  }
+  l[0] = l[0] * corr[0] + rs[0];
+  l[1] = l[1] * corr[1] + rs[1];
+#pragma unroll
+  for (int dn = 0; dn < DH / 8; ++dn) {
+    oacc[dn][0] *= corr[0]; oacc[dn][1] *= corr[0];
+    oacc[dn][2] *= corr[1]; oacc[dn][3] *= corr[1];
+  }
+  // O += P V
+  {
+    const int j = lane >> 3, rr = lane & 7;
+#pragma unroll
+    for (int kp = 0; kp < NT / 2; ++kp) {
+      uint32_t a[4];
+      a[0] = pack2(s[kp * 2][0], s[kp * 2][1]);
+      a[1] = pack2(s[kp * 2][2], s[kp * 2][3]);
+      a[2] = pack2(s[kp * 2 + 1][0], s[kp * 2 + 1][1]);
+      a[3] = pack2(s[kp * 2 + 1][2], s[kp * 2 + 1][3]);
+      const int key = kofs + kp * 16 + (j & 1) * 8 + rr;
+#pragma unroll
+      for (int dp = 0; dp < DH / 16; ++dp) {
+        uint32_t b[4];
+        ldsm_x4_trans(v_tile + tile_off<DH>(key, dp * 2 + (j >> 1)), b);
+        mma_bf16(oacc[dp * 2], a, b[0], b[1]);
+        mma_bf16(oacc[dp * 2 + 1], a, b[2], b[3]);
+      }
+    }
+  }
+}
+
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS)
+attn_kernel(const AttnParams p) {
+  constexpr int CH = DH / 8;                          // 16-byte chunks per row
+  constexpr int TILE_BYTES = TILE_KEYS * DH * 2;
+  constexpr int REC = DH + 2;                         // floats per row of a partial record
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint32_t is_last_s;
+  const uint32_t q_s = smem_u32(smem);
+  const uint32_t kv_s = q_s + TILE_BYTES;             // stage st: K at kv_s + st*2*TILE_BYTES, V after it
+
+  const AttnItem it = p.items[blockIdx.x];
+  const hb_seg sg = p.segs[it.seg];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = p.G, Hq = p.Hq;
+  const bool decode = (it.mode != 0);
+  const int hk = it.kv_head;
+  const __nv_bfloat16* kv_layer = p.kv.arena + static_cast<int64_t>(p.layer) * p.kv.layer_stride;
+  const int64_t head_off = static_cast<int64_t>(hk) * p.kv.P * DH;
+  const int64_t v_off = static_cast<int64_t>(p.kv.Hkv) * p.kv.P * DH;
+
+  // ---- Q tile -> shared memory (rows past n_rows are zero) ----
+  for (int u = tid; u < TILE_ROWS * CH; u += ATT_THREADS) {
+    const int rr = u / CH, c = u - rr * CH;
+    const int r = it.row0 + rr;
+    const bool valid = rr < it.n_rows;
+    const int tok = sg.q_start + (valid ? r / G : 0), head = hk * G + (valid ? r % G : 0);
+    const __nv_bfloat16* src = p.q + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8;
+    cp_async16(q_s + tile_off<DH>(rr, c), src, valid);
+  }
+  cp_async_commit();
+
+  const int n_tiles = (it.key1 - it.key0 + TILE_KEYS - 1) / TILE_KEYS;
+  auto load_tile = [&](int kt) {
+    if (kt < n_tiles) {
+      const uint32_t k_dst = kv_s + (kt % STAGES) * 2 * TILE_BYTES;
+      const int kb = it.key0 + kt * TILE_KEYS;
+      for (int u = tid; u < TILE_KEYS * CH; u += ATT_THREADS) {
+        const int rr = u / CH, c = u - rr * CH;
+        const int key = kb + rr;
+        bool valid = key < it.key1;
+        const __nv_bfloat16* src = kv_layer;
+        if (valid) {
+          const int blk = key / p.kv.P, slot = key - blk * p.kv.P;
+          const int page = p.pages[sg.pt_start + blk];
+          if (page < 0 || page >= p.kv.n_pages) {
+            atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
+            valid = false;
+          } else {
+            src = kv_layer + static_cast<int64_t>(page) * p.kv.page_stride + head_off + slot * DH + c * 8;
+          }
+        }
+        const uint32_t off = tile_off<DH>(rr, c);
+        cp_async16(k_dst + off, src, valid);
+        cp_async16(k_dst + TILE_BYTES + off, valid ? src + v_off : src, valid);
+      }
+    }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int st = 0; st < STAGES - 1; ++st) load_tile(st);
+
+  // rows of this thread: chunk items: warp-private rows; decode items: rows 0..15 for every warp
+  const int row_base = decode ? 0 : warp * 16;
+  const int ra = row_base + (lane >> 2), rb = ra + 8;
+  // position of the rows (rows past n_rows get -1: nothing visible)
+  const int pos_a = (ra < it.n_rows) ? sg.pos_start + (it.row0 + ra) / G : -1;
+  const int pos_b = (rb < it.n_rows) ? sg.pos_start + (it.row0 + rb) / G : -1;
+  // last position any row of this warp can see (skip tiles past it)
+  int warp_last = -1;
+  {
+    const int last_row = min(row_base + 15, it.n_rows - 1);
+    if (last_row >= row_base) warp_last = sg.pos_start + (it.row0 + last_row) / G;
+  }
+
+  uint32_t qf[DH / 16][4];
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.0f, 0.0f};
+  float oacc[DH / 8][4];
+#pragma unroll
+  for (int dn = 0; dn < DH / 8; ++dn) oacc[dn][0] = oacc[dn][1] = oacc[dn][2] = oacc[dn][3] = 0.0f;
+
+  for (int kt = 0; kt < n_tiles; ++kt) {
+    cp_async_wait<STAGES - 2>();
+    __syncthreads();
+    load_tile(kt + STAGES - 1);
+    if (kt == 0) {
+      const int j = lane >> 3, rr = lane & 7;
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks)
+        ldsm_x4(q_s + tile_off<DH>(row_base + (j & 1) * 8 + rr, ks * 2 + (j >> 1)), qf[ks]);
+    }
+    const uint32_t k_tile = kv_s + (kt % STAGES) * 2 * TILE_BYTES;
+    const int key_base = it.key0 + kt * TILE_KEYS;
+    if (decode) {
+      if (key_base + warp * 16 < it.key1)
+        warp_attend<DH, 2>(qf, k_tile, k_tile + TILE_BYTES, warp * 16, key_base, it.key1, pos_a, pos_b,
+                           p.scale_log2, m, l, oacc);
+    } else {
+      if (key_base <= warp_last)
+        warp_attend<DH, 8>(qf, k_tile, k_tile + TILE_BYTES, 0, key_base, it.key1, pos_a, pos_b, p.scale_log2, m,
+                           l, oacc);
+    }
+  }
+  cp_async_wait<0>();
+  // row sums: add the four threads of a quad
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
+    l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
+  }
+
+  if (!decode) {
+    // ---- chunk item: normalise, stage the warp's 16 rows in shared memory, store 16-byte vectors ----
+    const float inv_a = (l[0] > 0.0f) ? 1.0f / l[0] : 0.0f, inv_b = (l[1] > 0.0f) ? 1.0f / l[1] : 0.0f;
+    uint8_t* stage = smem;  // Q tile region; this warp touches its own 16 rows only
+#pragma unroll
+    for (int dn = 0; dn < DH / 8; ++dn) {
+      const uint32_t va = pack2(oacc[dn][0] * inv_a, oacc[dn][1] * inv_a);
+      const uint32_t vb = pack2(oacc[dn][2] * inv_b, oacc[dn][3] * inv_b);
+      *reinterpret_cast<uint32_t*>(stage + tile_off<DH>(ra, dn) + (lane & 3) * 4) = va;
+      *reinterpret_cast<uint32_t*>(stage + tile_off<DH>(rb, dn) + (lane & 3) * 4) = vb;
+    }
+    __syncwarp();
+    for (int u = lane; u < 16 * CH; u += 32) {
+      const int rr = row_base + u / CH, c = u % CH;
+      if (rr < it.n_rows) {
+        const int r = it.row0 + rr;
+        const int tok = sg.q_start + r / G, head = hk * G + r % G;
+        const uint4 v = *reinterpret_cast<const uint4*>(stage + tile_off<DH>(rr, c));
+        *reinterpret_cast<uint4*>(p.out + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8) = v;
+      }
+    }
+    return;
+  }
+
+  // ---- decode item: merge the four warps' partials in shared memory ----
+  __syncthreads();  // every warp is done reading the K/V ring
+  float* mbuf = reinterpret_cast<float*>(smem + TILE_BYTES);  // [4 warps][16 rows][REC]
+  {
+    float* mine = mbuf + warp * 16 * REC;
+#pragma unroll
+    for (int dn = 0; dn < DH / 8; ++dn) {
+      const int col = dn * 8 + 2 * (lane & 3);
+      mine[(lane >> 2) * REC + col] = oacc[dn][0];
+      mine[(lane >> 2) * REC + col + 1] = oacc[dn][1];
+      mine[((lane >> 2) + 8) * REC + col] = oacc[dn][2];
+      mine[((lane >> 2) + 8) * REC + col + 1] = oacc[dn][3];
+    }
+    if ((lane & 3) == 0) {
+      mine[(lane >> 2) * REC + DH] = m[0];
+      mine[(lane >> 2) * REC + DH + 1] = l[0];
+      mine[((lane >> 2) + 8) * REC + DH] = m[1];
+      mine[((lane >> 2) + 8) * REC + DH + 1] = l[1];
+    }
+  }
+  __syncthreads();
+  const int tok = sg.q_start;  // a decode segment has one row
+  float* rec = p.part + static_cast<size_t>(it.part_base + it.split) * G * REC;
+  for (int idx = tid; idx < G * DH; idx += ATT_THREADS) {
+    const int g = idx / DH, d = idx - g * DH;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) M = fmaxf(M, mbuf[(w * 16 + g) * REC + DH]);
+    const float Ms = (M == -INFINITY) ? 0.0f : M;
+    float L = 0.0f, o = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float f = exp2f(mbuf[(w * 16 + g) * REC + DH] - Ms);
+      L += mbuf[(w * 16 + g) * REC + DH + 1] * f;
+      o += mbuf[(w * 16 + g) * REC + d] * f;
+    }
+    if (it.n_splits == 1) {
+      p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
+    } else {
+      rec[g * REC + d] = o;
+      if (d == 0) {
+        rec[g * REC + DH] = M;
+        rec[g * REC + DH + 1] = L;
+      }
+    }
+  }
+  if (it.n_splits == 1) return;
+  // ---- splits of this (row, kv head): the CTA that arrives last merges them in split order ----
+  __threadfence();
+  __syncthreads();
+  uint32_t* counter = p.counters + it.seg * p.kv.Hkv + hk;
+  if (tid == 0) {
+    const uint32_t prev = atomicAdd(counter, 1u);
+    is_last_s = (prev + 1u == static_cast<uint32_t>(it.n_splits)) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!is_last_s) return;
+  __threadfence();
+  const float* recs = p.part + static_cast<size_t>(it.part_base) * G * REC;
+  for (int idx = tid; idx < G * DH; idx += ATT_THREADS) {
+    const int g = idx / DH, d = idx - g * DH;
+    float M = -INFINITY;
+    for (int sp = 0; sp < it.n_splits; ++sp) M = fmaxf(M, __ldcg(recs + (static_cast<size_t>(sp) * G + g) * REC + DH));
+    const float Ms = (M == -INFINITY) ? 0.0f : M;
+    float L = 0.0f, o = 0.0f;
+    for (int sp = 0; sp < it.n_splits; ++sp) {
+      const float* r = recs + (static_cast<size_t>(sp) * G + g) * REC;
+      const float f = exp2f(__ldcg(r + DH) - Ms);
+      L += __ldcg(r + DH + 1) * f;
+      o += __ldcg(r + d) * f;
+    }
+    p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
+  }
+  if (tid == 0) *counter = 0u;  // ready for the next launch
+}
+
+template <int DH>
+int launch(const AttnParams& p, int n_items, cudaStream_t s) {
+  constexpr int SMEM = TILE_KEYS * DH * 2 * (1 + 2 * STAGES);
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+      return HB_ERR_CUDA;
+    configured = true;
+  }
+  attn_kernel<DH><<<n_items, ATT_THREADS, SMEM, s>>>(p);
+  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
 }
 
 }  // namespace
 
 int hb_launch_attention(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s) {
-  const int Hq = c->cfg.n_heads;
-  const dim3 grid(c->dd.T, (Hq + 3) / 4);
-  const float scale = 1.0f / sqrtf(static_cast<float>(c->cfg.head_dim));
-  if (c->cfg.head_dim == 64)
-    attn_rowwarp_kernel<2><<<grid, 128, 0, s>>>(c->q, kv, layer, c->dd.row_seg, c->dd.row_pos, c->dd.segs,
-                                                 c->dd.pages, c->attn_out, Hq, scale, c->status);
-  else if (c->cfg.head_dim == 128)
-    attn_rowwarp_kernel<4><<<grid, 128, 0, s>>>(c->q, kv, layer, c->dd.row_seg, c->dd.row_pos, c->dd.segs,
-                                                 c->dd.pages, c->attn_out, Hq, scale, c->status);
-  else
-    return HB_ERR_UNSUPPORTED;
-  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+  if (c->dd.n_attn_items <= 0) return HB_OK;
+  AttnParams p;
+  p.q = c->q;
+  p.out = c->attn_out;
+  p.kv = kv;
+  p.layer = layer;
+  p.items = c->dd.attn_items;
+  p.segs = c->dd.segs;
+  p.pages = c->dd.pages;
+  p.part = c->attn_part;
+  p.counters = c->attn_counters;
+  p.status = c->status;
+  p.Hq = c->cfg.n_heads;
+  p.G = c->cfg.n_heads / c->cfg.n_kv_heads;
+  p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));
+  if (c->cfg.head_dim == 64) return launch<64>(p, c->dd.n_attn_items, s);
+  if (c->cfg.head_dim == 128) return launch<128>(p, c->dd.n_attn_items, s);
+  return HB_ERR_UNSUPPORTED;
 }

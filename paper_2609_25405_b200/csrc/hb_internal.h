@@ -29,8 +29,9 @@ struct AttnItem {
   int32_t key1;       // one past the last key this split may touch
   int32_t split;      // split index, n_splits
   int32_t n_splits;
-  int32_t part_base;  // first partial-result record of this (seg, kv_head, row tile)
-  int32_t pad[3];
+  int32_t part_base;  // first partial-result record of this (seg, kv_head)
+  int32_t mode;       // 0 = chunk item (64 query rows, all keys), 1 = decode item (one split)
+  int32_t pad[2];
 };
 
 // Pool work item: rows [row0, row0 + n_rows) of an embedding segment.
@@ -127,7 +128,8 @@ struct hb_ctx {
   float* rope_sin;
   float* attn_part;         // split-KV partial results
   float* pool_part;         // pooling partial sums
-  uint32_t* counters;       // arrival counters (attention merge, pooling merge)
+  uint32_t* counters;       // arrival counters of the pooling merge, one per segment
+  uint32_t* attn_counters;  // arrival counters of the split-KV merge, one per (segment, kv head)
   uint32_t* status;         // device status word
   uint8_t* desc_dev;        // packed descriptor
   size_t desc_cap;

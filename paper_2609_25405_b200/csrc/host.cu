@@ -12,6 +12,8 @@
 namespace {
 
 constexpr int POOL_ROWS = 32;   // rows per pooling work item
+constexpr int ATT_TILE_ROWS = 64;   // query rows (tokens x grouped heads) per chunk attention item
+constexpr int ATT_SPLIT_KEYS = 512; // keys per decode attention item; depends on nothing but this constant
 constexpr int N_STAGING = 4;    // pinned descriptor staging ring
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -22,6 +24,8 @@ bool cfg_ok(const hb_model_cfg* c) {
     return false;
   if (c->head_dim != 64 && c->head_dim != 128) return false;
   if (c->n_heads % c->n_kv_heads) return false;
+  const int g = c->n_heads / c->n_kv_heads;
+  if (g > 16 || (64 % g)) return false;  // attention tiles: 64 rows = (64/g) tokens x g heads
   if (c->d_model % 64 || (c->n_heads * c->head_dim) % 64 || c->d_ffn % 64 || c->vocab % 8) return false;
   if (c->d_model > 8192) return false;
   if (c->page_size != 16) return false;
@@ -39,7 +43,8 @@ struct Carve {
 };
 
 struct Layout {
-  size_t x, h, qkv, q, attn_out, act, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, status, desc;
+  size_t x, h, qkv, q, attn_out, act, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
+      status, desc;
   size_t total, desc_cap, attn_part_floats, pool_part_floats;
   int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items;
 };
@@ -63,13 +68,16 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
   L.rope_sin = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
   L.max_pool_items = max_tokens / POOL_ROWS + max_segs + 1;
-  L.max_attn_items = 0;
-  L.attn_part_floats = 4;
+  const int G = c.n_heads / c.n_kv_heads;
+  const int max_splits = (c.max_pos + ATT_SPLIT_KEYS - 1) / ATT_SPLIT_KEYS;
+  L.max_attn_items = c.n_kv_heads * (max_tokens * G / ATT_TILE_ROWS + max_segs + max_segs * max_splits);
+  L.attn_part_floats = static_cast<size_t>(max_segs) * c.n_kv_heads * max_splits * G * (c.head_dim + 2);
   L.pool_part_floats = static_cast<size_t>(L.max_pool_items) * c.d_model;
   L.attn_part = cv.take(L.attn_part_floats * 4);
   L.pool_part = cv.take(L.pool_part_floats * 4);
   L.n_counters = max_segs + 1;
   L.counters = cv.take(static_cast<size_t>(L.n_counters) * 4);
+  L.attn_counters = cv.take(static_cast<size_t>(max_segs) * c.n_kv_heads * 4);
   L.status = cv.take(256);
   size_t dc = 0;
   dc += align_up(static_cast<size_t>(max_tokens) * 4, 16) * 3;          // tok, row_seg, row_pos
@@ -239,6 +247,7 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->attn_part = reinterpret_cast<float*>(c->ws + lay.attn_part);
   c->pool_part = reinterpret_cast<float*>(c->ws + lay.pool_part);
   c->counters = reinterpret_cast<uint32_t*>(c->ws + lay.counters);
+  c->attn_counters = reinterpret_cast<uint32_t*>(c->ws + lay.attn_counters);
   c->status = reinterpret_cast<uint32_t*>(c->ws + lay.status);
   c->desc_dev = c->ws + lay.desc;
   c->desc_cap = lay.desc_cap;
@@ -515,9 +524,53 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     }
   }
   if (static_cast<int32_t>(pitems.size()) > ex->lay.max_pool_items) return HB_ERR_TOO_LARGE;
+  // attention work list: chunk items (64 query rows x all visible keys) and decode items (one
+  // split of ATT_SPLIT_KEYS keys); sorted by cost, largest first, so the tail of the launch is short
+  std::vector<AttnItem> aitems;
+  {
+    const int G = cfg.n_heads / cfg.n_kv_heads;
+    int32_t rec_at = 0;
+    for (int32_t r = 0; r < R; ++r) {
+      const hb_seg& sg = d->segs[r];
+      for (int32_t hk = 0; hk < cfg.n_kv_heads; ++hk) {
+        if (sg.kind == HB_KIND_DECODE) {
+          const int32_t n_keys = sg.pos_start + 1;
+          const int32_t ns = (n_keys + ATT_SPLIT_KEYS - 1) / ATT_SPLIT_KEYS;
+          for (int32_t sp = 0; sp < ns; ++sp) {
+            AttnItem it{};
+            it.seg = r; it.kv_head = hk; it.row0 = 0; it.n_rows = G;
+            it.key0 = sp * ATT_SPLIT_KEYS;
+            it.key1 = std::min(n_keys, it.key0 + ATT_SPLIT_KEYS);
+            it.split = sp; it.n_splits = ns; it.part_base = rec_at; it.mode = 1;
+            aitems.push_back(it);
+          }
+          rec_at += ns;
+        } else {
+          const int32_t rows = sg.q_len * G;
+          for (int32_t row0 = 0; row0 < rows; row0 += ATT_TILE_ROWS) {
+            AttnItem it{};
+            it.seg = r; it.kv_head = hk; it.row0 = row0; it.n_rows = std::min(ATT_TILE_ROWS, rows - row0);
+            it.key0 = 0;
+            it.key1 = sg.pos_start + (row0 + it.n_rows - 1) / G + 1;
+            it.split = 0; it.n_splits = 1; it.part_base = 0; it.mode = 0;
+            aitems.push_back(it);
+          }
+        }
+      }
+    }
+    auto cost = [](const AttnItem& a) {
+      return static_cast<int64_t>(a.key1 - a.key0) * (a.mode ? 16 : a.n_rows);
+    };
+    std::stable_sort(aitems.begin(), aitems.end(),
+                     [&](const AttnItem& a, const AttnItem& b) { return cost(a) > cost(b); });
+    if (static_cast<int32_t>(aitems.size()) > ex->lay.max_attn_items) return HB_ERR_TOO_LARGE;
+    if (static_cast<size_t>(rec_at) * G * (cfg.head_dim + 2) > c->attn_part_floats) return HB_ERR_TOO_LARGE;
+  }
+  const size_t o_aitems = place(aitems.size() * sizeof(AttnItem));
   const size_t o_pitems = place(pitems.size() * sizeof(PoolItem));
   if (off > c->desc_cap) return HB_ERR_TOO_LARGE;
   if (!pitems.empty()) memcpy(st.host + o_pitems, pitems.data(), pitems.size() * sizeof(PoolItem));
+  if (!aitems.empty()) memcpy(st.host + o_aitems, aitems.data(), aitems.size() * sizeof(AttnItem));
   if (cudaMemcpyAsync(c->desc_dev, st.host, off, cudaMemcpyHostToDevice, s) != cudaSuccess) return HB_ERR_CUDA;
   if (cudaEventRecord(st.ev, s) != cudaSuccess) return HB_ERR_CUDA;
   st.pending = true;
@@ -529,12 +582,12 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
   dd.segs = reinterpret_cast<const hb_seg*>(c->desc_dev + o_segs);
   dd.pages = reinterpret_cast<const int32_t*>(c->desc_dev + o_pages);
   dd.logit_src = reinterpret_cast<const int32_t*>(c->desc_dev + o_lsrc);
-  dd.attn_items = nullptr;
+  dd.attn_items = reinterpret_cast<const AttnItem*>(c->desc_dev + o_aitems);
   dd.pool_items = reinterpret_cast<const PoolItem*>(c->desc_dev + o_pitems);
   dd.T = T;
   dd.R = R;
   dd.n_logit = d->n_logit_rows;
-  dd.n_attn_items = 0;
+  dd.n_attn_items = static_cast<int32_t>(aitems.size());
   dd.n_pool_items = static_cast<int32_t>(pitems.size());
 
   KvGeom kg;

@@ -10,7 +10,7 @@ from dataclasses import dataclass
 
 import numpy as np
 
-from . import binding as B
+from . import consts as B
 from . import synth
 
 
@@ -131,8 +131,10 @@ class MixedWorkload:
             left -= q
         self.inflight = queue[idx:] + nxt        # requests the budget did not reach stay first in line
 
-        def commit():
+        def commit(advance_decode=True):
             for r, q in plan:
+                if r.kind == "gen" and not advance_decode:
+                    continue
                 r.done += q
                 if r.kind == "embed" and r.done == r.n:
                     self.kv.free(r.pages)
