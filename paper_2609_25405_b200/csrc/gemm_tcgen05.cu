@@ -13,6 +13,11 @@
 //            releases stages and publishes finished accumulators
 //   warps 2-5 epilogue: tcgen05.ld the accumulator (each warp owns 32 TMEM lanes), apply
 //            the epilogue, store with 16-byte vectors; overlaps the next tile's main loop
+// Two variants share the code.  CG = 1: one CTA per 128 x BN tile.  CG = 2: a cluster of two CTAs
+// works on one 256 x 256 tile with tcgen05 cta_group::2: each CTA loads its own 128 rows of A and
+// its own 128 rows of B (no multicast), the leader CTA issues MMAs that read both CTAs' shared
+// memory, and each CTA's TMEM receives its 128 accumulator rows.  This halves the B traffic per SM
+// and leaves room for six pipeline stages.
 // Every mbarrier wait is bounded in time; on expiry the CTA raises a status bit, stops
 // issuing work, lets outstanding copies land, frees its TMEM and returns.
 #include "hb_internal.h"
@@ -25,11 +30,12 @@ constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
-template <int BN>
+template <int BN, int CG>
 struct Tile {
-  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int B_ROWS = BN / CG;            // rows of B this CTA loads per stage
+  static constexpr int STAGES = (B_ROWS == 256) ? 4 : 6;
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = B_ROWS * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulators; 256 or 512 (powers of two)
   static constexpr int BAR_BYTES = 256;
@@ -95,6 +101,39 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_2d_cg2(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                int c_inner, int c_outer) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
+      : "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// The same shared-memory offset in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
 __device__ __forceinline__ void tcgen05_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -114,11 +153,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
   return d;
 }
 
-// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = BN.
-template <int BN>
+// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128 * CG, N = BN.
+template <int BN, int CG>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
-         (static_cast<uint32_t>(BM >> 4) << 24);
+         (static_cast<uint32_t>((BM * CG) >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
@@ -128,6 +167,25 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16_cg2(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+                                              uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Arrive (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs.
+__device__ __forceinline__ void umma_commit_cg2(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"(mask)
       : "memory");
 }
 
@@ -210,11 +268,11 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
   }
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const GemmArgs g) {
-  using T = Tile<BN>;
+  using T = Tile<BN, CG>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -229,8 +287,14 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // CG = 2: the two CTAs of a cluster share every tile; rank 0 leads (issues the MMAs and owns
+  // the full / tmem-empty barriers).  CG = 1: every CTA is its own leader.
+  const uint32_t rank = (CG == 2) ? cluster_ctarank() : 0u;
+  const bool leader = (rank == 0u);
+  const int worker = (CG == 2) ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int n_workers = (CG == 2) ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
-  const int m_tiles = (g.M + BM - 1) / BM;
+  const int m_tiles = (g.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (g.N + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
   const int k_blocks = (g.K + BK - 1) / BK;
@@ -242,21 +306,35 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tempty_bar(a), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(static_cast<uint32_t>(T::TMEM_COLS))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(static_cast<uint32_t>(T::TMEM_COLS))
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(static_cast<uint32_t>(T::TMEM_COLS))
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tcgen05_fence_before();
   __syncthreads();
+  if constexpr (CG == 2) cluster_sync();  // the peer's barriers are initialised before anything signals them
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+
+  // Give up: raise the flag here and in the peer CTA so that every role of the group leaves its loop.
+  auto give_up = [&]() {
+    *abort_flag = 1u;
+    if constexpr (CG == 2) st_cluster_u32(map_to_rank(smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u), 1u);
+  };
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -264,16 +342,24 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const int m0 = (tile % m_tiles) * BM;
-        const int n0 = (tile / m_tiles) * BN;
+      // the data of both CTAs of a group is accounted on the leader's barrier
+      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+        const int m0 = (tile % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
+        const int n0 = (tile / m_tiles) * BN + static_cast<int>(rank) * T::B_ROWS;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; give_up(); break; }
           const uint32_t a_dst = smem_base + stage * T::STAGE_BYTES;
           const uint32_t b_dst = a_dst + T::A_BYTES;
-          mbar_arrive_expect_tx(full_bar(stage), T::STAGE_BYTES);
-          tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, m0);
-          tma_load_2d(b_dst, &tmB, full_bar(stage), (kb >> g.b_kshift) * BK, n0);
+          if constexpr (CG == 2) {
+            const uint32_t bar = map_to_rank(full_bar(stage), 0u);
+            if (leader) mbar_arrive_expect_tx(full_bar(stage), 2u * T::STAGE_BYTES);
+            tma_load_2d_cg2(a_dst, &tmA, bar, kb * BK, m0);
+            tma_load_2d_cg2(b_dst, &tmB, bar, (kb >> g.b_kshift) * BK, n0);
+          } else {
+            mbar_arrive_expect_tx(full_bar(stage), T::STAGE_BYTES);
+            tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, m0);
+            tma_load_2d(b_dst, &tmB, full_bar(stage), (kb >> g.b_kshift) * BK, n0);
+          }
           if (++stage == T::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -284,20 +370,20 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc<BN>();
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = make_idesc<BN, CG>();
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; give_up(); break; }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; give_up(); break; }
           tcgen05_fence_after();
           const uint32_t a_addr = smem_base + stage * T::STAGE_BYTES;
           const uint64_t adesc = make_smem_desc(a_addr);
@@ -305,13 +391,18 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 elements along K inside the 128-byte swizzle row = +32 B = +2 in the address field
-            umma_bf16(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
+            if constexpr (CG == 2) umma_bf16_cg2(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
+            else umma_bf16(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
           }
-          umma_commit(empty_bar(stage));  // stage is free once these MMAs have read it
+          // the stage is free (in every CTA of the group) once these MMAs have read it
+          if constexpr (CG == 2) umma_commit_cg2(empty_bar(stage));
+          else umma_commit(empty_bar(stage));
           if (++stage == T::STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(tfull_bar(acc));      // accumulator complete
+        if constexpr (CG == 2) umma_commit_cg2(tfull_bar(acc));  // accumulator complete (both CTAs)
+        else umma_commit(tfull_bar(acc));
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -322,10 +413,10 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const int m0 = (tile % m_tiles) * BM;
+    for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+      const int m0 = (tile % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
       const int n0 = (tile / m_tiles) * BN;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; give_up(); break; }
       tcgen05_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
@@ -337,19 +428,29 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       }
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if constexpr (CG == 2) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));
+        else mbar_arrive(tempty_bar(acc));
+      }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
   tcgen05_fence_before();
   __syncthreads();
+  // no CTA of a group leaves (or frees TMEM) while its peer may still read its shared memory or signal it
+  if constexpr (CG == 2) cluster_sync();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(g.status, HB_DEV_GEMM_WAIT_EXPIRED);
   if (warp == 1) {
     tcgen05_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"(static_cast<uint32_t>(T::TMEM_COLS))
-                 : "memory");
+    if constexpr (CG == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(static_cast<uint32_t>(T::TMEM_COLS))
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(static_cast<uint32_t>(T::TMEM_COLS))
+                   : "memory");
   }
 }
 
@@ -371,33 +472,44 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CG>
 int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& a, int num_sms, cudaStream_t s) {
-  using T = Tile<BN>;
+  using T = Tile<BN, CG>;
   static bool configured = false;
-  auto kern = hb_gemm_tcgen05_kernel<BN, EPI>;
+  auto kern = hb_gemm_tcgen05_kernel<BN, EPI, CG>;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES) != cudaSuccess)
       return HB_ERR_CUDA;
     configured = true;
   }
-  const int m_tiles = (a.M + BM - 1) / BM;
+  const int m_tiles = (a.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (a.N + BN - 1) / BN;
-  int grid = m_tiles * n_tiles;
-  if (grid > num_sms) grid = num_sms;
-  if (grid < 1) return HB_OK;
-  kern<<<grid, NUM_THREADS, T::SMEM_BYTES, s>>>(tmA, tmB, a);
-  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+  int workers = m_tiles * n_tiles;
+  if (workers > num_sms / CG) workers = num_sms / CG;
+  if (workers < 1) return HB_OK;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(workers * CG));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = T::SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, a) == cudaSuccess ? HB_OK : HB_ERR_CUDA;
 }
 
-template <int BN>
+template <int BN, int CG>
 int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, int epi, const GemmArgs& a, int num_sms,
               cudaStream_t s) {
   switch (epi) {
-    case HB_EPI_BF16: return launch_one<BN, HB_EPI_BF16>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_BF16: return launch_one<BN, HB_EPI_BF16, CG>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, a, num_sms, s);
     default: return HB_ERR_BAD_ARG;
   }
 }
@@ -421,6 +533,8 @@ int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t 
 // Tile width: 256 columns halves the shared-memory traffic per flop; 128 gives more tiles
 // when the problem has too few to fill the SMs or the last wave would be mostly idle.
 int hb_gemm_pick_bn(int M, int N, int num_sms) {
+  // enough rows and columns for 256 x 256 pair tiles to fill the machine: use CTA pairs
+  if (M > 128 && static_cast<long>((M + 255) / 256) * ((N + 255) / 256) >= num_sms / 2) return HB_GEMM_PAIR256;
   const int m_tiles = (M + BM - 1) / BM;
   const long t256 = static_cast<long>(m_tiles) * ((N + 255) / 256);
   const long t128 = static_cast<long>(m_tiles) * ((N + 127) / 128);
@@ -430,9 +544,12 @@ int hb_gemm_pick_bn(int M, int N, int num_sms) {
   return (e128 * 0.92 > e256) ? 128 : 256;
 }
 
-int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi, const GemmArgs& a,
+int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : variant; }
+
+int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,
                    int num_sms, cudaStream_t s) {
-  if (bn == 256) return launch_bn<256>(tmA, tmB, epi, a, num_sms, s);
-  if (bn == 128) return launch_bn<128>(tmA, tmB, epi, a, num_sms, s);
+  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, epi, a, num_sms, s);
+  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, epi, a, num_sms, s);
+  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, epi, a, num_sms, s);
   return HB_ERR_BAD_ARG;
 }

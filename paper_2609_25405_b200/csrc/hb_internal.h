@@ -94,7 +94,11 @@ struct GemmArgs {
 
 int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
                     uint32_t box_rows);
+// GEMM variants: 128 / 256 = one CTA per 128 x BN tile; HB_GEMM_PAIR256 = a CTA pair per 256 x 256 tile.
+// The B tensor map's box must have hb_gemm_box_rows(variant) rows.
+constexpr int HB_GEMM_PAIR256 = 512;
 int hb_gemm_pick_bn(int M, int N, int num_sms);
+int hb_gemm_box_rows(int variant);
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s);
 

@@ -637,10 +637,10 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
       wm.bn_o = hb_gemm_pick_bn(c->max_tokens, cfg.d_model, c->num_sms);
       wm.bn_gu = hb_gemm_pick_bn(c->max_tokens, 2 * cfg.d_ffn, c->num_sms);
       wm.bn_down = wm.bn_o;
-      if ((rc = hb_tmap_2d_bf16(&wm.qkv, lw.wqkv, n_qkv, cfg.d_model, wm.bn_qkv)) != HB_OK) return rc;
-      if ((rc = hb_tmap_2d_bf16(&wm.o, lw.wo, cfg.d_model, n_q, wm.bn_o)) != HB_OK) return rc;
-      if ((rc = hb_tmap_2d_bf16(&wm.gu, lw.w_gate_up, 2ull * cfg.d_ffn, cfg.d_model, wm.bn_gu)) != HB_OK) return rc;
-      if ((rc = hb_tmap_2d_bf16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, wm.bn_down)) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.qkv, lw.wqkv, n_qkv, cfg.d_model, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.o, lw.wo, cfg.d_model, n_q, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.gu, lw.w_gate_up, 2ull * cfg.d_ffn, cfg.d_model, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_bf16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
       wm.key[0] = lw.wqkv; wm.key[1] = lw.wo; wm.key[2] = lw.w_gate_up; wm.key[3] = lw.w_down;
     }
     if (l == 0) HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
@@ -748,7 +748,7 @@ int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t
   CUtensorMap ta, tb;
   int rc = hb_tmap_2d_bf16(&ta, A, M, K, 128);
   if (rc != HB_OK) return rc;
-  rc = hb_tmap_2d_bf16(&tb, B, N, K, bn);
+  rc = hb_tmap_2d_bf16(&tb, B, N, K, hb_gemm_box_rows(bn));
   if (rc != HB_OK) return rc;
   GemmArgs ga;
   ga.C = C; ga.M = M; ga.N = N; ga.K = K; ga.b_kshift = 0; ga.status = c->status;
