@@ -12,9 +12,10 @@
 //                their partial (max, sum, output) are merged in shared memory, and the splits
 //                of a row through a scratch record per split, merged in split order by the CTA
 //                that arrives last (integer arrival counter; no floating-point atomics).
-// K/V tiles of 64 keys (4 pages) are gathered with 16-byte cp.async into an XOR-swizzled
-// shared-memory ring; S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate),
-// softmax in fp32 with exp2.  Split decisions depend on the request's own length only, so a
+// K/V tiles of 64 keys (4 pages) are gathered by TMA: one thread issues a 2-D tensor copy per
+// (page, 64-column half) into a 128-byte-swizzled shared-memory ring and the CTA waits on the
+// stage's mbarrier (bounded).  S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32
+// accumulate), softmax in fp32 with exp2.  Split decisions depend on the request's own length only, so a
 // request's result does not depend on its batch mates.
 #include "hb_internal.h"
 
@@ -54,6 +55,43 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait (1 s).  Returns false if it expired.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u && global_ns() - t0 > 1000000000ull) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c_inner,
+                                            int c_outer) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
+      : "memory");
+}
+
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -75,10 +113,11 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Byte offset of 16-byte chunk `c` of row `r` in a [rows][DH] bf16 tile (XOR swizzle).
+// Byte offset of 16-byte chunk `c` of row `r` in a 64-row tile stored as [DH/64 halves][64 rows][64]
+// bf16 with the 128-byte swizzle TMA applies (chunk index XOR row mod 8 inside each 128-byte row).
 template <int DH>
 __device__ __forceinline__ uint32_t tile_off(int r, int c) {
-  return static_cast<uint32_t>(r * (DH * 2) + ((c ^ (r & 7)) << 4));
+  return static_cast<uint32_t>((c >> 3) * (64 * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
 // One warp: 16 query rows against NT*8 keys starting at tile-local key `kofs`.
@@ -172,14 +211,20 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
 
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS)
-attn_kernel(const AttnParams p) {
+attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   constexpr int CH = DH / 8;                          // 16-byte chunks per row
   constexpr int TILE_BYTES = TILE_KEYS * DH * 2;
+  constexpr int PAGE_HALF_BYTES = 16 * 128;           // one page of one 64-column half
   constexpr int REC = DH + 2;                         // floats per row of a partial record
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint32_t is_last_s;
-  const uint32_t q_s = smem_u32(smem);
-  const uint32_t kv_s = q_s + TILE_BYTES;             // stage st: K at kv_s + st*2*TILE_BYTES, V after it
+  extern __shared__ uint8_t smem_raw[];
+  // carve-up (1024-byte aligned for the TMA swizzle): STAGES x (K tile, V tile) | barriers, flag | page ids.
+  // The Q tile borrows the K half of the last stage until the fragments are in registers.
+  const uint32_t kv_s = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (kv_s - smem_u32(smem_raw));
+  const uint32_t q_s = kv_s + (STAGES - 1) * 2 * TILE_BYTES;
+  const uint32_t bar_s = kv_s + STAGES * 2 * TILE_BYTES;
+  uint32_t& is_last_s = *reinterpret_cast<uint32_t*>(smem + STAGES * 2 * TILE_BYTES + 32);
+  int32_t* pg_s = reinterpret_cast<int32_t*>(smem + STAGES * 2 * TILE_BYTES + 64);
 
   const AttnItem it = p.items[blockIdx.x];
   const hb_seg sg = p.segs[it.seg];
@@ -187,10 +232,21 @@ attn_kernel(const AttnParams p) {
   const int G = p.G, Hq = p.Hq;
   const bool decode = (it.mode != 0);
   const int hk = it.kv_head;
-  const __nv_bfloat16* kv_layer = p.kv.arena + static_cast<int64_t>(p.layer) * p.kv.layer_stride;
-  const int64_t head_off = static_cast<int64_t>(hk) * p.kv.P * DH;
-  const int64_t v_off = static_cast<int64_t>(p.kv.Hkv) * p.kv.P * DH;
 
+  if (tid == 0) {
+    for (int st = 0; st < STAGES; ++st) mbar_init(bar_s + 8u * st, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // page ids of the keys this item reads -> shared memory (checked once)
+  const int first_blk = it.key0 / p.kv.P;
+  const int n_blk = (it.key1 + p.kv.P - 1) / p.kv.P - first_blk;
+  int bad = 0;
+  for (int i = tid; i < n_blk; i += ATT_THREADS) {
+    const int blk = first_blk + i;
+    const int pg = (blk < sg.pt_len) ? p.pages[sg.pt_start + blk] : -1;
+    bad |= (pg < 0 || pg >= p.kv.n_pages);
+    pg_s[i] = pg;
+  }
   // ---- Q tile -> shared memory (rows past n_rows are zero) ----
   for (int u = tid; u < TILE_ROWS * CH; u += ATT_THREADS) {
     const int rr = u / CH, c = u - rr * CH;
@@ -201,36 +257,36 @@ attn_kernel(const AttnParams p) {
     cp_async16(q_s + tile_off<DH>(rr, c), src, valid);
   }
   cp_async_commit();
+  if (__syncthreads_or(bad)) {  // also publishes the barrier initialisation and the page ids
+    if (tid == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
+    cp_async_wait<0>();
+    return;                     // nothing was requested from TMA yet
+  }
 
   const int n_tiles = (it.key1 - it.key0 + TILE_KEYS - 1) / TILE_KEYS;
-  auto load_tile = [&](int kt) {
-    if (kt < n_tiles) {
-      const uint32_t k_dst = kv_s + (kt % STAGES) * 2 * TILE_BYTES;
-      const int kb = it.key0 + kt * TILE_KEYS;
-      for (int u = tid; u < TILE_KEYS * CH; u += ATT_THREADS) {
-        const int rr = u / CH, c = u - rr * CH;
-        const int key = kb + rr;
-        bool valid = key < it.key1;
-        const __nv_bfloat16* src = kv_layer;
-        if (valid) {
-          const int blk = key / p.kv.P, slot = key - blk * p.kv.P;
-          const int page = p.pages[sg.pt_start + blk];
-          if (page < 0 || page >= p.kv.n_pages) {
-            atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
-            valid = false;
-          } else {
-            src = kv_layer + static_cast<int64_t>(page) * p.kv.page_stride + head_off + slot * DH + c * 8;
-          }
-        }
-        const uint32_t off = tile_off<DH>(rr, c);
-        cp_async16(k_dst + off, src, valid);
-        cp_async16(k_dst + TILE_BYTES + off, valid ? src + v_off : src, valid);
+  // one thread: request the pages of tile kt from TMA (K and V, every 64-column half)
+  auto issue_tile = [&](int kt) {
+    const int st = kt % STAGES;
+    const uint32_t k_dst = kv_s + st * 2 * TILE_BYTES, bar = bar_s + 8u * st;
+    const int kb = it.key0 + kt * TILE_KEYS;
+    const int n_pg = min(TILE_KEYS / 16, (it.key1 - kb + 15) / 16);
+    const int pi0 = kb / 16 - first_blk;
+    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n_pg) * 2u * (DH / 64) * PAGE_HALF_BYTES);
+    for (int pi = 0; pi < n_pg; ++pi) {
+      const int64_t page = pg_s[pi0 + pi];
+      const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.kv.n_pages + page) * 2) * p.kv.Hkv + hk) * 16);
+      const int row_v = row_k + p.kv.Hkv * 16;
+#pragma unroll
+      for (int h = 0; h < DH / 64; ++h) {
+        tma_load_2d(k_dst + h * (64 * 128) + pi * PAGE_HALF_BYTES, &kv_map, bar, h * 64, row_k);
+        tma_load_2d(k_dst + TILE_BYTES + h * (64 * 128) + pi * PAGE_HALF_BYTES, &kv_map, bar, h * 64, row_v);
       }
     }
-    cp_async_commit();
   };
-#pragma unroll
-  for (int st = 0; st < STAGES - 1; ++st) load_tile(st);
+  int issued = 0;
+  if (tid == 0) {
+    for (; issued < STAGES - 1 && issued < n_tiles; ++issued) issue_tile(issued);
+  }
 
   // rows of this thread: chunk items: warp-private rows; decode items: rows 0..15 for every warp
   const int row_base = decode ? 0 : warp * 16;
@@ -251,10 +307,16 @@ attn_kernel(const AttnParams p) {
 #pragma unroll
   for (int dn = 0; dn < DH / 8; ++dn) oacc[dn][0] = oacc[dn][1] = oacc[dn][2] = oacc[dn][3] = 0.0f;
 
+  // A wait that expires is remembered; control flow stays uniform (every thread keeps meeting the
+  // block barriers) and the CTA leaves at the next loop head without storing anything.
+  int failed = 0;
+  cp_async_wait<0>();
   for (int kt = 0; kt < n_tiles; ++kt) {
-    cp_async_wait<STAGES - 2>();
-    __syncthreads();
-    load_tile(kt + STAGES - 1);
+    if (__syncthreads_or(failed)) { failed = 1; break; }   // everyone is done with tile kt - 1 (and Q landed)
+    if (tid == 0 && kt > 0) {   // at kt = 0 the last stage still holds Q
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // stages were read / patched by generic accesses
+      for (; issued < n_tiles && issued < kt + STAGES; ++issued) issue_tile(issued);
+    }
     if (kt == 0) {
       const int j = lane >> 3, rr = lane & 7;
 #pragma unroll
@@ -263,6 +325,18 @@ attn_kernel(const AttnParams p) {
     }
     const uint32_t k_tile = kv_s + (kt % STAGES) * 2 * TILE_BYTES;
     const int key_base = it.key0 + kt * TILE_KEYS;
+    if (!mbar_wait(bar_s + 8u * (kt % STAGES), static_cast<uint32_t>((kt / STAGES) & 1))) failed = 1;
+    const int valid_rows = it.key1 - key_base;
+    if (valid_rows < TILE_KEYS) {
+      // rows past the last key hold stale bytes (rest of the last page, pages not requested): zero the
+      // V rows so that a zero probability times garbage cannot produce NaN (K rows are masked anyway)
+      uint8_t* v_gen = smem + (kt % STAGES) * 2 * TILE_BYTES + TILE_BYTES;
+      for (int u = tid; u < (TILE_KEYS - valid_rows) * CH; u += ATT_THREADS) {
+        const int rr = valid_rows + u / CH, c = u % CH;
+        *reinterpret_cast<uint4*>(v_gen + tile_off<DH>(rr, c)) = make_uint4(0u, 0u, 0u, 0u);
+      }
+      __syncthreads();
+    }
     if (decode) {
       if (key_base + warp * 16 < it.key1)
         warp_attend<DH, 2>(qf, k_tile, k_tile + TILE_BYTES, warp * 16, key_base, it.key1, pos_a, pos_b,
@@ -273,7 +347,14 @@ attn_kernel(const AttnParams p) {
                            l, oacc);
     }
   }
-  cp_async_wait<0>();
+  if (__syncthreads_or(failed)) {
+    if (tid == 0) {
+      atomicOr(p.status, HB_DEV_ATTN_WAIT_EXPIRED);
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block retires
+    }
+    __syncthreads();
+    return;
+  }
   // row sums: add the four threads of a quad
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
@@ -284,7 +365,7 @@ attn_kernel(const AttnParams p) {
   if (!decode) {
     // ---- chunk item: normalise, stage the warp's 16 rows in shared memory, store 16-byte vectors ----
     const float inv_a = (l[0] > 0.0f) ? 1.0f / l[0] : 0.0f, inv_b = (l[1] > 0.0f) ? 1.0f / l[1] : 0.0f;
-    uint8_t* stage = smem;  // Q tile region; this warp touches its own 16 rows only
+    uint8_t* stage = smem;  // the ring is idle now; this warp touches its own 16 rows of the first tile only
 #pragma unroll
     for (int dn = 0; dn < DH / 8; ++dn) {
       const uint32_t va = pack2(oacc[dn][0] * inv_a, oacc[dn][1] * inv_a);
@@ -307,7 +388,7 @@ attn_kernel(const AttnParams p) {
 
   // ---- decode item: merge the four warps' partials in shared memory ----
   __syncthreads();  // every warp is done reading the K/V ring
-  float* mbuf = reinterpret_cast<float*>(smem + TILE_BYTES);  // [4 warps][16 rows][REC]
+  float* mbuf = reinterpret_cast<float*>(smem);  // [4 warps][16 rows][REC], over the idle ring
   {
     float* mine = mbuf + warp * 16 * REC;
 #pragma unroll
@@ -382,21 +463,23 @@ attn_kernel(const AttnParams p) {
 }
 
 template <int DH>
-int launch(const AttnParams& p, int n_items, cudaStream_t s) {
-  constexpr int SMEM = TILE_KEYS * DH * 2 * (1 + 2 * STAGES);
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+int launch(const CUtensorMap& kv_map, const AttnParams& p, int n_items, int max_pos, cudaStream_t s) {
+  // ring + barriers + page ids of one item (at most every page of a request) + alignment slack
+  const int smem = TILE_KEYS * DH * 2 * (2 * STAGES) + 64 + (max_pos / 16 + 2) * 4 + 1024;
+  static int configured = 0;
+  if (smem > 227 * 1024) return HB_ERR_UNSUPPORTED;
+  if (configured < smem) {
+    if (cudaFuncSetAttribute(attn_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return HB_ERR_CUDA;
-    configured = true;
+    configured = smem;
   }
-  attn_kernel<DH><<<n_items, ATT_THREADS, SMEM, s>>>(p);
+  attn_kernel<DH><<<n_items, ATT_THREADS, smem, s>>>(kv_map, p);
   return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
 }
 
 }  // namespace
 
-int hb_launch_attention(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s) {
+int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s) {
   if (c->dd.n_attn_items <= 0) return HB_OK;
   AttnParams p;
   p.q = c->q;
@@ -412,7 +495,7 @@ int hb_launch_attention(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s) 
   p.Hq = c->cfg.n_heads;
   p.G = c->cfg.n_heads / c->cfg.n_kv_heads;
   p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));
-  if (c->cfg.head_dim == 64) return launch<64>(p, c->dd.n_attn_items, s);
-  if (c->cfg.head_dim == 128) return launch<128>(p, c->dd.n_attn_items, s);
+  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_attn_items, c->cfg.max_pos, s);
+  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_attn_items, c->cfg.max_pos, s);
   return HB_ERR_UNSUPPORTED;
 }

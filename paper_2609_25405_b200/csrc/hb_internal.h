@@ -67,6 +67,8 @@ struct KvGeom {
 
 struct hb_kv {
   hb_model_cfg cfg;
+  CUtensorMap map;      // arena as a 2-D bf16 tensor [rows of head_dim], box = one page x 64 columns
+  bool has_map;
   void* arena;
   size_t arena_bytes;
   int32_t n_pages;
@@ -107,7 +109,7 @@ struct hb_ctx;
 int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s);
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
 int hb_launch_rope_append(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s);
-int hb_launch_attention(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s);
+int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
                     int n_slots, float* out_emb, cudaStream_t s);
 int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s);

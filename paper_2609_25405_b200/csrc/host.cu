@@ -335,6 +335,15 @@ int hb_kv_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32
   hb_kv* kv = new (std::nothrow) hb_kv();
   if (!kv) return HB_ERR_BAD_ARG;
   kv->cfg = *cfg;
+  kv->has_map = false;
+  if (arena) {
+    const uint64_t rows = static_cast<uint64_t>(cfg->n_layers) * n_pages * 2 * cfg->n_kv_heads * cfg->page_size;
+    if (rows > 0x7fffffffull || hb_tmap_2d_bf16(&kv->map, arena, rows, cfg->head_dim, 16) != HB_OK) {
+      delete kv;
+      return rows > 0x7fffffffull ? HB_ERR_TOO_LARGE : HB_ERR_CUDA;
+    }
+    kv->has_map = true;
+  }
   kv->arena = arena;
   kv->arena_bytes = arena_bytes;
   kv->n_pages = n_pages;
@@ -444,7 +453,7 @@ int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_se
 int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv* kv, hb_pool* pool,
                   float* out_logits, float* out_emb, void* stream) {
   if (!c || !d || !w || !kv || !w->layers || !w->tok_emb || !w->final_norm) return HB_ERR_BAD_ARG;
-  if (!kv->arena) return HB_ERR_BAD_ARG;
+  if (!kv->arena || !kv->has_map) return HB_ERR_BAD_ARG;
   if (memcmp(&kv->cfg, &c->cfg, sizeof(hb_model_cfg)) != 0) return HB_ERR_BAD_ARG;
   const int32_t n_slots = pool ? pool->n_slots : 0;
   int rc = validate(c->cfg, c->max_tokens, c->max_segs, c->max_page_ids, kv->n_pages, n_slots, d);
@@ -535,12 +544,15 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
       for (int32_t hk = 0; hk < cfg.n_kv_heads; ++hk) {
         if (sg.kind == HB_KIND_DECODE) {
           const int32_t n_keys = sg.pos_start + 1;
-          const int32_t ns = (n_keys + ATT_SPLIT_KEYS - 1) / ATT_SPLIT_KEYS;
+          // about ATT_SPLIT_KEYS keys per split, equal parts rounded up to whole 64-key tiles
+          const int32_t ns0 = std::max(1, (n_keys + ATT_SPLIT_KEYS / 2) / ATT_SPLIT_KEYS);
+          const int32_t per = ((n_keys + ns0 - 1) / ns0 + 63) / 64 * 64;
+          const int32_t ns = (n_keys + per - 1) / per;
           for (int32_t sp = 0; sp < ns; ++sp) {
             AttnItem it{};
             it.seg = r; it.kv_head = hk; it.row0 = 0; it.n_rows = G;
-            it.key0 = sp * ATT_SPLIT_KEYS;
-            it.key1 = std::min(n_keys, it.key0 + ATT_SPLIT_KEYS);
+            it.key0 = sp * per;
+            it.key1 = std::min(n_keys, it.key0 + per);
             it.split = sp; it.n_splits = ns; it.part_base = rec_at; it.mode = 1;
             aitems.push_back(it);
           }
@@ -653,7 +665,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     ga.C = c->qkv; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rope_append(c, kg, l, s));
-    HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, l, s));
+    HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s));
@@ -704,6 +716,11 @@ int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
   if (cudaMemcpyAsync(&code, c->status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return HB_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;
   if (code != 0) {
+    // a block that gave up may have left arrival counters mid-count: clear them with the status word
+    if (cudaMemsetAsync(c->attn_counters, 0, static_cast<size_t>(c->max_segs) * c->cfg.n_kv_heads * 4, s) !=
+            cudaSuccess ||
+        cudaMemsetAsync(c->counters, 0, static_cast<size_t>(c->n_counters) * 4, s) != cudaSuccess)
+      return HB_ERR_CUDA;
     if (cudaMemsetAsync(c->status, 0, 4, s) != cudaSuccess) return HB_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;
   }
