@@ -230,7 +230,7 @@ def main():
 
     weights = B.DeviceWeights.random_on_device(shape, seed=0)
     kv = B.KvCache(cfg, n_pages)
-    kvb = kv.arena.view(torch.bfloat16)
+    kvb = kv.arena.view(torch.float16)
     step_e = 1 << 28
     for i in range(0, kvb.numel(), step_e):          # synthetic cached K/V: N(0,1)
         kvb[i:i + step_e].normal_(0.0, 1.0)
@@ -352,6 +352,8 @@ def main():
     line = {"metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "precision": "bf16 weights x fp16 activations / KV cache on the tensor cores, fp32 accumulation, "
+                         "fp32 residual stream, norms, softmax and pooling",
             "config": {"workload": spec.name, "shape": spec.shape, "tokens_per_step": w["T"],
                        "decode_rows": spec.n_decode, "chunk": spec.chunk, "token_budget": spec.budget,
                        "l2": "inputs larger than L2 (weights and KV pages are re-streamed every step)",

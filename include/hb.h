@@ -63,7 +63,10 @@ typedef struct hb_pool hb_pool;
 
 /* Decoder-only model: pre-norm RMSNorm, rotate-half RoPE, grouped-query causal
  * attention, SwiGLU FFN, no biases, untied LM head.  head_dim must be 64 or
- * 128; d_model, n_heads*head_dim, d_ffn multiples of 64; page_size 16. */
+ * 128; d_model, n_heads*head_dim, d_ffn multiples of 64; page_size 16.
+ * Precision: bf16 model weights, repacked to fp16 for the tensor cores;
+ * activations between kernels, the KV cache and the attention probabilities
+ * fp16; residual stream, norms, softmax, pooling and every accumulation fp32. */
 typedef struct {
   int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
   int32_t page_size;    /* tokens per KV page (16)                              */
@@ -72,14 +75,18 @@ typedef struct {
   float rms_eps;
 } hb_model_cfg;
 
-/* All weights are bf16, row-major [out, in] (y = x * W^T), device memory owned
- * by the caller.
- *   wqkv      [(n_heads + 2 n_kv_heads) * head_dim, d_model]: q rows, then k, then v
- *   wo        [d_model, n_heads * head_dim]
- *   w_gate_up [2 * d_ffn, d_model]: row 2j = gate row j, row 2j+1 = up row j
- *   w_down    [d_model, d_ffn]
- *   attn_norm, ffn_norm, final_norm [d_model] gains
- *   tok_emb, lm_head [vocab, d_model] */
+/* Weights are row-major [out, in] (y = x * W^T), device memory owned by the
+ * caller.  The projection matrices are fp16: the model's bf16 values repacked
+ * once with hb_weights_pack_f16 (the tensor cores take one 16-bit format for
+ * both operands, and activations are fp16).  Gains and the token embedding
+ * stay bf16.
+ *   wqkv      fp16 [(n_heads + 2 n_kv_heads) * head_dim, d_model]: q rows, then k, then v
+ *   wo        fp16 [d_model, n_heads * head_dim]
+ *   w_gate_up fp16 [2 * d_ffn, d_model]: row 2j = gate row j, row 2j+1 = up row j
+ *   w_down    fp16 [d_model, d_ffn]
+ *   lm_head   fp16 [vocab, d_model]
+ *   attn_norm, ffn_norm, final_norm bf16 [d_model] gains
+ *   tok_emb   bf16 [vocab, d_model] */
 typedef struct {
   const void* attn_norm;
   const void* wqkv;
@@ -146,9 +153,9 @@ HB_API int hb_destroy(hb_ctx* ctx);
 
 /* ---- paged KV cache ------------------------------------------------------- */
 
-/* Bytes of one page across all layers, and of an arena of n_pages.  Arena
- * layout (bf16): [layer][page][K|V][kv_head][slot 0..page_size)[head_dim], so
- * the K (or V) rows of one (layer, page, head) are contiguous.  Host only. */
+/* Bytes of an arena of n_pages.  Arena layout (fp16; post-rotary K and V):
+ * [layer][page][K|V][kv_head][slot 0..page_size)[head_dim], so the K (or V)
+ * rows of one (layer, page, head) are contiguous.  Host only. */
 HB_API int hb_kv_arena_bytes(const hb_model_cfg* cfg, int32_t n_pages, size_t* out_bytes);
 
 /* Wrap a caller-owned device arena.  Only the free list lives in the library
@@ -203,6 +210,12 @@ HB_API int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t
 HB_API int hb_mixed_step(hb_ctx* ctx, const hb_batch_desc* desc, const hb_weights* w, hb_kv* kv,
                   hb_pool* pool, float* out_logits, float* out_emb, void* stream);
 
+/* Repack bf16 values to fp16, element by element, on `stream` (device
+ * pointers, 16-byte aligned; dst may equal src for an in-place repack, partial
+ * overlap is rejected).  Exact for 2^-14 <= |w| <= 65504; smaller magnitudes
+ * round to the fp16 subnormal grid (absolute error <= 2^-25), larger saturate. */
+HB_API int hb_weights_pack_f16(const void* src_bf16, void* dst_f16, size_t n_elems, void* stream);
+
 /* Greedy sampler over logits rows (Algorithm 1 "Sampler", greedy case): lowest
  * index of the maximum of each row.  logits device float [n_rows, vocab],
  * out_tokens device int32 [n_rows]. */
@@ -237,15 +250,16 @@ HB_API int hb_last_launch_count(const hb_ctx* ctx, int32_t* out_count);
 /* Epilogues of the projection GEMM (the dense contractions of the forward,
  * Section 3.1 "attention and feed-forward layers"). */
 enum {
-  HB_EPI_BF16 = 0,      /* C bf16 [M,N] = A * B^T                               */
+  HB_EPI_F16 = 0,       /* C fp16 [M,N] = A * B^T                               */
   HB_EPI_F32 = 1,       /* C float [M,N] = A * B^T                              */
   HB_EPI_RESID_F32 = 2, /* C float [M,N] += A * B^T (residual stream update)    */
-  HB_EPI_SWIGLU = 3     /* C bf16 [M,N/2]: silu(acc[2j]) * acc[2j+1]            */
+  HB_EPI_SWIGLU = 3     /* C fp16 [M,N/2]: silu(acc[2j]) * acc[2j+1]            */
 };
 
-/* C = epilogue(A * B^T): A bf16 [M,K] row-major, B bf16 [N,K] row-major (both
- * K-major), fp32 accumulation on the tcgen05 tensor cores.  All device
- * pointers, 16-byte aligned; K and N multiples of 8.  M may be any value >= 1. */
+/* C = epilogue(A * B^T): A fp16 [M,K] row-major (activations), B fp16 [N,K]
+ * row-major (weights), both K-major, fp32 accumulation on the tcgen05 tensor
+ * cores; fp16 outputs saturate at +-65504.  All device pointers, 16-byte
+ * aligned; K and N multiples of 8.  M may be any value >= 1. */
 HB_API int hb_gemm(hb_ctx* ctx, const void* A, const void* B, void* C, int32_t M, int32_t N,
             int32_t K, int32_t epilogue, void* stream);
 

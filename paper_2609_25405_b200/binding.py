@@ -18,7 +18,7 @@ ERRORS = {0: "HB_OK", -1: "HB_ERR_BAD_ARG", -2: "HB_ERR_CUDA", -3: "HB_ERR_OOM_P
           -4: "HB_ERR_OOM_SLOTS", -5: "HB_ERR_TOO_LARGE", -6: "HB_ERR_BAD_DESC",
           -7: "HB_ERR_DEVICE_STATUS", -8: "HB_ERR_UNSUPPORTED"}
 from .consts import (KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK, POOL_NONE, POOL_MEAN,  # noqa: F401,E402
-                     POOL_LAST, EPI_BF16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
+                     POOL_LAST, EPI_F16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
 
 
 class HbError(RuntimeError):
@@ -82,6 +82,7 @@ _sig = {
     "hb_validate_desc": [C.POINTER(ModelCfg), C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                          C.POINTER(BatchDesc)],
     "hb_mixed_step": [_P, C.POINTER(BatchDesc), C.POINTER(Weights), _P, _P, _P, _P, _P],
+    "hb_weights_pack_f16": [_P, _P, C.c_size_t, _P],
     "hb_argmax": [_P, _P, C.c_int32, _P, _P],
     "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
     "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
@@ -119,8 +120,17 @@ def bf16_from_f32(a, device="cuda"):
     return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
 
 
+def pack_f16_(t, stream=None):
+    """Repack a bf16 tensor to fp16 in place (library kernel); returns the fp16 view."""
+    assert t.dtype == torch.bfloat16 and t.is_contiguous()
+    check(lib.hb_weights_pack_f16(C.c_void_p(t.data_ptr()), C.c_void_p(t.data_ptr()), t.numel(),
+                                  _stream_ptr(stream)), "hb_weights_pack_f16")
+    return t.view(torch.float16)
+
+
 class DeviceWeights:
-    """Weights resident in HBM in the library's layout, plus the hb_weights struct."""
+    """Weights resident in HBM in the library's layout (projection matrices repacked to fp16 in
+    place, gains and token embedding bf16), plus the hb_weights struct."""
 
     def __init__(self, n_layers):
         self.tensors = []          # keep-alive
@@ -138,21 +148,22 @@ class DeviceWeights:
         s = W.shape
         self = cls(s.L)
         up = lambda a: self._keep(bf16_from_f32(a, device))
+        upw = lambda a: self._keep(pack_f16_(bf16_from_f32(a, device)))
         self.struct.tok_emb = up(W.tok_emb)
-        self.struct.lm_head = up(W.lm_head)
+        self.struct.lm_head = upw(W.lm_head)
         self.struct.final_norm = up(W.final_norm)
         for l in range(s.L):
             w = W.layer(l)
             lw = self.layers[l]
             lw.attn_norm = up(w["attn_norm"])
             lw.ffn_norm = up(w["ffn_norm"])
-            lw.wqkv = up(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0))
-            lw.wo = up(w["wo"])
+            lw.wqkv = upw(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0))
+            lw.wo = upw(w["wo"])
             gu = np.empty((2 * s.F, s.d), dtype=np.float32)
             gu[0::2] = w["wg"]
             gu[1::2] = w["wu"]
-            lw.w_gate_up = up(gu)
-            lw.w_down = up(w["wd"])
+            lw.w_gate_up = upw(gu)
+            lw.w_down = upw(w["wd"])
         return self
 
     @classmethod
@@ -163,13 +174,13 @@ class DeviceWeights:
         g = torch.Generator(device=device)
         g.manual_seed(seed)
 
-        def rnd(r, c):
+        def rnd(r, c, pack=True):
             t = torch.empty((r, c), dtype=torch.bfloat16, device=device)
             t.normal_(0.0, std, generator=g)
-            return self._keep(t)
+            return self._keep(pack_f16_(t) if pack else t)
 
         ones = lambda: self._keep(torch.ones(shape.d, dtype=torch.bfloat16, device=device))
-        self.struct.tok_emb = rnd(shape.V, shape.d)
+        self.struct.tok_emb = rnd(shape.V, shape.d, pack=False)
         self.struct.lm_head = rnd(shape.V, shape.d)
         self.struct.final_norm = ones()
         for l in range(shape.L):
@@ -203,10 +214,10 @@ class KvCache:
                                C.byref(self.handle)), "hb_kv_create")
 
     def view(self):
-        """bf16 view [L, page, 2, Hkv, P, Dh]."""
+        """fp16 view [L, page, 2, Hkv, P, Dh]."""
         c = self.cfg
-        return self.arena.view(torch.bfloat16).view(c.n_layers, self.n_pages, 2, c.n_kv_heads,
-                                                    c.page_size, c.head_dim)
+        return self.arena.view(torch.float16).view(c.n_layers, self.n_pages, 2, c.n_kv_heads,
+                                                   c.page_size, c.head_dim)
 
     def alloc(self, n):
         ids = (C.c_int32 * max(n, 1))()

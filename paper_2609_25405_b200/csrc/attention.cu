@@ -14,7 +14,7 @@
 //                that arrives last (integer arrival counter; no floating-point atomics).
 // K/V tiles of 64 keys (4 pages) are gathered by TMA: one thread issues a 2-D tensor copy per
 // (page, 64-column half) into a 128-byte-swizzled shared-memory ring and the CTA waits on the
-// stage's mbarrier (bounded).  S = Q K^T and O += P V run on mma.sync m16n8k16 (bf16 in, fp32
+// stage's mbarrier (bounded).  S = Q K^T and O += P V run on mma.sync m16n8k16 (fp16 in, fp32
 // accumulate), softmax in fp32 with exp2.  Split decisions depend on the request's own length only, so a
 // request's result does not depend on its batch mates.
 #include "hb_internal.h"
@@ -27,8 +27,8 @@ constexpr int TILE_ROWS = 64;
 constexpr int STAGES = 3;
 
 struct AttnParams {
-  const __nv_bfloat16* q;     // [T, Hq*Dh]
-  __nv_bfloat16* out;         // [T, Hq*Dh]
+  const __half* q;            // [T, Hq*Dh] fp16
+  __half* out;                // [T, Hq*Dh] fp16
   KvGeom kv;
   int layer;
   const AttnItem* items;
@@ -101,15 +101,15 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
@@ -142,8 +142,8 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
         const int key = kofs + np * 16 + (j >> 1) * 8 + rr;
         uint32_t b[4];
         ldsm_x4(k_tile + tile_off<DH>(key, ks * 2 + (j & 1)), b);
-        mma_bf16(s[np * 2], qf[ks], b[0], b[1]);
-        mma_bf16(s[np * 2 + 1], qf[ks], b[2], b[3]);
+        mma_f16(s[np * 2], qf[ks], b[0], b[1]);
+        mma_f16(s[np * 2 + 1], qf[ks], b[2], b[3]);
       }
     }
   }
@@ -202,8 +202,8 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
       for (int dp = 0; dp < DH / 16; ++dp) {
         uint32_t b[4];
         ldsm_x4_trans(v_tile + tile_off<DH>(key, dp * 2 + (j >> 1)), b);
-        mma_bf16(oacc[dp * 2], a, b[0], b[1]);
-        mma_bf16(oacc[dp * 2 + 1], a, b[2], b[3]);
+        mma_f16(oacc[dp * 2], a, b[0], b[1]);
+        mma_f16(oacc[dp * 2 + 1], a, b[2], b[3]);
       }
     }
   }
@@ -253,7 +253,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     const int r = it.row0 + rr;
     const bool valid = rr < it.n_rows;
     const int tok = sg.q_start + (valid ? r / G : 0), head = hk * G + (valid ? r % G : 0);
-    const __nv_bfloat16* src = p.q + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8;
+    const __half* src = p.q + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8;
     cp_async16(q_s + tile_off<DH>(rr, c), src, valid);
   }
   cp_async_commit();
@@ -423,7 +423,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
       o += mbuf[(w * 16 + g) * REC + d] * f;
     }
     if (it.n_splits == 1) {
-      p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
+      p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2half_rn(L > 0.0f ? o / L : 0.0f);
     } else {
       rec[g * REC + d] = o;
       if (d == 0) {
@@ -457,7 +457,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
       L += __ldcg(r + DH + 1) * f;
       o += __ldcg(r + d) * f;
     }
-    p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2bfloat16(L > 0.0f ? o / L : 0.0f);
+    p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2half_rn(L > 0.0f ? o / L : 0.0f);
   }
   if (tid == 0) *counter = 0u;  // ready for the next launch
 }

@@ -1,0 +1,468 @@
+// Chunk-row attention on the tcgen05 tensor cores (Section 3.2 of the paper: embedding / prefill
+// chunks attend causally over their own earlier chunks plus themselves).
+//
+// One CTA handles 128 query rows = (128 / G) consecutive tokens x the G query heads of one KV head
+// (G = Hq / Hkv) of one chunk segment, against every key the rows may see, in tiles of 64 keys
+// (4 KV pages).  192 threads:
+//   warp 0    TMA: gathers the pages of each key tile (one 2-D copy per page and 64-column half)
+//             into a shared-memory ring in the 128-byte-swizzled layout the MMA descriptors expect
+//   warp 1    MMA: S_j = Q K_j^T (128 x 64, fp32 in TMEM, double buffered) and
+//             O += P_j V_j (128 x Dh, fp32 in TMEM), both tcgen05.mma kind::f16 from shared memory;
+//             S_{j+1} is issued before P_j V_j so the tensor pipe works while softmax runs
+//   warps 2-5 softmax: one thread per query row (TMEM lane): read its S row, mask, running max and
+//             sum in fp32 (exp2), write P (fp16) to shared memory.  O stays in TMEM and is
+//             rescaled only when a row's maximum grows by more than 2^8 since the maximum in use
+//             (probabilities stay below 256, exact in fp16/fp32); the final 1/sum absorbs it.
+// Every mbarrier wait is bounded; on expiry the CTA raises a status bit and leaves without
+// storing.  The work split depends on the segment's own lengths only.
+#include "hb_internal.h"
+
+namespace {
+
+constexpr int TC_THREADS = 192;
+constexpr int BM = 128;        // query rows per CTA
+constexpr int BN = 64;         // keys per tile
+constexpr uint64_t WAIT_NS = 1000000000ull;
+
+struct TcParams {
+  const __half* q;            // [T, Hq*Dh]
+  __half* out;                // [T, Hq*Dh]
+  int n_pages, Hkv, Hq, G, layer;
+  const AttnItem* items;
+  const hb_seg* segs;
+  const int32_t* pages;
+  uint32_t* status;
+  float scale_log2;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait; false if it expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > WAIT_NS) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c_inner,
+                                            int c_outer) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
+      : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major operand: rows 128 B apart, 8-row groups
+// `sbo` bytes apart (lbo unused).  MN-major operand: `lbo` = distance between 64-element column
+// groups, `sbo` = distance between groups of 8 K-rows.
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// D fp32, A and B fp16; b_mn: B operand is MN-major (V: head dimension contiguous).
+__device__ __forceinline__ constexpr uint32_t make_idesc(int n, bool b_mn) {
+  return (1u << 4) | (0u << 7) | (0u << 10) | ((b_mn ? 1u : 0u) << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int DH>
+struct TcCfg {
+  static constexpr int SUB = DH / 64;                    // 64-column sub-tiles
+  static constexpr int STAGES = (DH == 128) ? 2 : 4;
+  static constexpr int Q_BYTES = BM * DH * 2;
+  static constexpr int KV_HALF = BN * DH * 2;            // K (or V) tile of one stage
+  static constexpr int P_BYTES = BM * BN * 2;
+  static constexpr int RING = STAGES * 2 * KV_HALF;
+  static constexpr int BAR_OFF = Q_BYTES + RING + P_BYTES;
+  static constexpr int TMEM_COLS = 256;                  // S: 2 x 64 columns, O: DH columns
+  static constexpr int O_COL = 128;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(TC_THREADS, 2)
+attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams p, int max_blk) {
+  using C = TcCfg<DH>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_s = base, ring_s = base + C::Q_BYTES, p_s = ring_s + C::RING, bar_s = base + C::BAR_OFF;
+  auto kv_full = [&](int s) { return bar_s + 8u * s; };
+  auto kv_empty = [&](int s) { return bar_s + 8u * (C::STAGES + s); };
+  auto s_full = [&](int b) { return bar_s + 8u * (2 * C::STAGES + b); };
+  auto s_empty = [&](int b) { return bar_s + 8u * (2 * C::STAGES + 2 + b); };
+  const uint32_t p_ready = bar_s + 8u * (2 * C::STAGES + 4), pv_done = bar_s + 8u * (2 * C::STAGES + 5);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  int32_t* pg_s = reinterpret_cast<int32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16);
+
+  const AttnItem it = p.items[blockIdx.x];
+  const hb_seg sg = p.segs[it.seg];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = p.G, Hq = p.Hq, hk = it.kv_head;
+  const int n_tiles = (it.key1 + BN - 1) / BN;           // key0 is 0 for chunk items
+  const int n_blk = (it.key1 + 15) / 16;
+
+  if (tid == 0) {
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(s_empty(b), 4); }
+    mbar_init(p_ready, 4);
+    mbar_init(pv_done, 1);
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  int bad = 0;
+  for (int i = tid; i < n_blk; i += TC_THREADS) {
+    const int pg = (i < sg.pt_len && i < max_blk) ? p.pages[sg.pt_start + i] : -1;
+    bad |= (pg < 0 || pg >= p.n_pages);
+    if (i < max_blk) pg_s[i] = pg;
+  }
+  // Q tile -> shared memory in the K-major 128-byte-swizzled layout ([SUB][128 rows][64]); rows past
+  // n_rows are zero
+  for (int u = tid; u < BM * (DH / 8); u += TC_THREADS) {
+    const int rr = u / (DH / 8), c = u - rr * (DH / 8);
+    const int r = it.row0 + rr;
+    const bool valid = rr < it.n_rows;
+    const int tok = sg.q_start + (valid ? r / G : 0), head = hk * G + (valid ? r % G : 0);
+    const __half* src = p.q + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8;
+    const uint32_t off = static_cast<uint32_t>((c >> 3) * (BM * 128) + rr * 128 + (((c & 7) ^ (rr & 7)) << 4));
+    cp_async16(q_s + off, src, valid);
+  }
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+  fence_async_smem();   // Q was written through the generic proxy; the MMA reads it through the async proxy
+  if (__syncthreads_or(bad)) {
+    if (tid == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
+    return;             // nothing requested from TMA, no TMEM held
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(static_cast<uint32_t>(C::TMEM_COLS)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      for (int j = 0; j < n_tiles; ++j) {
+        const int st = j % C::STAGES;
+        if (!mbar_wait(kv_empty(st), static_cast<uint32_t>(((j / C::STAGES) & 1) ^ 1), abort_flag)) break;
+        const int kb = j * BN;
+        const int n_pg = min(BN / 16, (it.key1 - kb + 15) / 16);
+        const uint32_t k_dst = ring_s + st * 2 * C::KV_HALF;
+        mbar_arrive_expect_tx(kv_full(st), static_cast<uint32_t>(n_pg) * 2u * C::SUB * (16 * 128));
+        for (int pi = 0; pi < n_pg; ++pi) {
+          const int64_t page = pg_s[kb / 16 + pi];
+          const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.n_pages + page) * 2) * p.Hkv + hk) * 16);
+          const int row_v = row_k + p.Hkv * 16;
+#pragma unroll
+          for (int h = 0; h < C::SUB; ++h) {
+            tma_load_2d(k_dst + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_k);
+            tma_load_2d(k_dst + C::KV_HALF + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_v);
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(BN, false);
+      constexpr uint32_t idesc_o = make_idesc(DH, true);
+      auto issue_s = [&](int j) -> bool {
+        const int st = j % C::STAGES, b = j & 1;
+        if (!mbar_wait(kv_full(st), static_cast<uint32_t>((j / C::STAGES) & 1), abort_flag)) return false;
+        if (!mbar_wait(s_empty(b), static_cast<uint32_t>(((j >> 1) & 1) ^ 1), abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t k_tile = ring_s + st * 2 * C::KV_HALF;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint64_t ad = make_desc(q_s + (ks >> 2) * (BM * 128) + (ks & 3) * 32, 16, 1024);
+          const uint64_t bd = make_desc(k_tile + (ks >> 2) * (BN * 128) + (ks & 3) * 32, 16, 1024);
+          umma(tmem + static_cast<uint32_t>(b * BN), ad, bd, idesc_s, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(s_full(b));
+        return true;
+      };
+      bool ok = issue_s(0);
+      for (int j = 0; ok && j < n_tiles; ++j) {
+        if (j + 1 < n_tiles) ok = issue_s(j + 1);
+        if (!ok) break;
+        if (!mbar_wait(p_ready, static_cast<uint32_t>(j & 1), abort_flag)) break;
+        tc_fence_after();
+        const uint32_t v_tile = ring_s + (j % C::STAGES) * 2 * C::KV_HALF + C::KV_HALF;
+#pragma unroll
+        for (int ks = 0; ks < BN / 16; ++ks) {
+          const uint64_t ad = make_desc(p_s + ks * 32, 16, 1024);
+          const uint64_t bd = make_desc(v_tile + ks * 2048, BN * 128, 1024);
+          umma(tmem + static_cast<uint32_t>(C::O_COL), ad, bd, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+        }
+        umma_commit(kv_empty(j % C::STAGES));
+        umma_commit(pv_done);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------- softmax (one thread per query row) ----------------
+    const int quarter = warp & 3;
+    const int rr = quarter * 32 + lane;                     // row of the tile = TMEM lane
+    const bool row_valid = rr < it.n_rows;
+    const int r = it.row0 + rr;
+    const int pos = row_valid ? sg.pos_start + r / G : -1;
+    const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+    float m_used = -INFINITY, l = 0.0f;
+    bool ok = true;
+    // the lanes of a warp leave the loop together (warp-wide votes and tcgen05.ld/st follow)
+    auto wait_w = [&](uint32_t bar, uint32_t parity) {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag)) != 0;
+    };
+    for (int j = 0; j < n_tiles; ++j) {
+      const int b = j & 1, key_base = j * BN;
+      if (!wait_w(s_full(b), static_cast<uint32_t>((j >> 1) & 1))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t sr[2][32];
+      tmem_ld32(t_lane + static_cast<uint32_t>(b * BN), sr[0]);
+      tmem_ld32(t_lane + static_cast<uint32_t>(b * BN + 32), sr[1]);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_empty(b));
+      // scale, mask (only tiles that touch the diagonal or the end of the keys), row maximum
+      const bool need_mask = (key_base + BN - 1 > pos) || (key_base + BN > it.key1);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float v = __uint_as_float(sr[h][i]) * p.scale_log2;
+          if (need_mask) {
+            const int key = key_base + h * 32 + i;
+            if (key > pos || key >= it.key1) v = -INFINITY;
+          }
+          sr[h][i] = __float_as_uint(v);
+          mx = fmaxf(mx, v);
+        }
+      }
+      const float m_new = fmaxf(m_used, mx);
+      const bool grow = (m_new > m_used + 8.0f) || (m_used == -INFINITY && m_new > -INFINITY);
+      // P_{j-1} V_{j-1} must have completed before O is rescaled or P is overwritten
+      if (j > 0 && !wait_w(pv_done, static_cast<uint32_t>((j - 1) & 1))) { ok = false; break; }
+      if (__any_sync(0xffffffffu, grow)) {
+        const float f = grow ? exp2f(m_used - m_new) : 1.0f;   // m_used = -inf -> 0
+        if (j > 0) {
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < DH; c += 32) {
+            uint32_t o[32];
+            tmem_ld32(t_lane + static_cast<uint32_t>(C::O_COL + c), o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+            tmem_st32(t_lane + static_cast<uint32_t>(C::O_COL + c), o);
+          }
+          tmem_st_wait();
+        }
+        l *= f;
+        if (grow) m_used = m_new;
+      }
+      const float ms = (m_used == -INFINITY) ? 0.0f : m_used;
+      // probabilities -> fp16 P row in shared memory (K-major, 128-byte swizzle)
+      uint8_t* prow = smem + C::Q_BYTES + C::RING + rr * 128;
+      float sum = 0.0f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int i = c * 8 + e * 2;
+          const float p0 = exp2f(__uint_as_float(sr[i >> 5][i & 31]) - ms);
+          const float p1 = exp2f(__uint_as_float(sr[(i + 1) >> 5][(i + 1) & 31]) - ms);
+          sum += p0 + p1;
+          pk[e] = pack_h2(p0, p1);
+        }
+        *reinterpret_cast<uint4*>(prow + ((c ^ (rr & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+      l += sum;
+      // keys past the end of the request hold stale bytes: zero those V rows (0 * garbage must stay 0)
+      const int valid_keys = it.key1 - key_base;
+      if (valid_keys < BN) {
+        uint8_t* v_gen = smem + C::Q_BYTES + (j % C::STAGES) * 2 * C::KV_HALF + C::KV_HALF;
+        const int t4 = tid - 64;  // 0..127 over the four softmax warps
+        for (int u = t4; u < (BN - valid_keys) * (DH / 8); u += 128) {
+          const int kr = valid_keys + u / (DH / 8), c = u % (DH / 8);
+          *reinterpret_cast<uint4*>(v_gen + (c >> 3) * (BN * 128) + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) =
+              make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_ready);
+    }
+    // ---- epilogue: O / l -> fp16 ----
+    if (ok && n_tiles > 0 && wait_w(pv_done, static_cast<uint32_t>((n_tiles - 1) & 1))) {
+      tc_fence_after();
+      const float inv = (l > 0.0f) ? 1.0f / l : 0.0f;
+      const int tok = sg.q_start + (row_valid ? r / G : 0), head = hk * G + (row_valid ? r % G : 0);
+      __half* orow = p.out + (static_cast<size_t>(tok) * Hq + head) * DH;
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 32) {
+        uint32_t o[32];
+        tmem_ld32(t_lane + static_cast<uint32_t>(C::O_COL + c), o);
+        tmem_ld_wait();
+        if (row_valid) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 pk;
+            pk.x = pack_h2(__uint_as_float(o[v * 8 + 0]) * inv, __uint_as_float(o[v * 8 + 1]) * inv);
+            pk.y = pack_h2(__uint_as_float(o[v * 8 + 2]) * inv, __uint_as_float(o[v * 8 + 3]) * inv);
+            pk.z = pack_h2(__uint_as_float(o[v * 8 + 4]) * inv, __uint_as_float(o[v * 8 + 5]) * inv);
+            pk.w = pack_h2(__uint_as_float(o[v * 8 + 6]) * inv, __uint_as_float(o[v * 8 + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + c + v * 8) = pk;
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (tid == 0) {
+      atomicOr(p.status, HB_DEV_ATTN_WAIT_EXPIRED);
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block retires
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
+                 "r"(static_cast<uint32_t>(C::TMEM_COLS)) : "memory");
+  }
+}
+
+template <int DH>
+int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_pos, cudaStream_t s) {
+  using C = TcCfg<DH>;
+  const int max_blk = max_pos / 16 + 2;
+  const int smem = C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16 + max_blk * 4 + 1024;
+  static int configured = 0;
+  if (smem > 227 * 1024) return HB_ERR_UNSUPPORTED;
+  if (configured < smem) {
+    if (cudaFuncSetAttribute(attn_chunk_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return HB_ERR_CUDA;
+    configured = smem;
+  }
+  attn_chunk_tc_kernel<DH><<<n_items, TC_THREADS, smem, s>>>(kv_map, p, max_blk);
+  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+}
+
+}  // namespace
+
+int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s) {
+  if (c->dd.n_tc_items <= 0) return HB_OK;
+  TcParams p;
+  p.q = c->q;
+  p.out = c->attn_out;
+  p.n_pages = kv.n_pages;
+  p.Hkv = kv.Hkv;
+  p.Hq = c->cfg.n_heads;
+  p.G = c->cfg.n_heads / c->cfg.n_kv_heads;
+  p.layer = layer;
+  p.items = c->dd.tc_items;
+  p.segs = c->dd.segs;
+  p.pages = c->dd.pages;
+  p.status = c->status;
+  p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));
+  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s);
+  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s);
+  return HB_ERR_UNSUPPORTED;
+}

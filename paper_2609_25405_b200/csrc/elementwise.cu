@@ -35,20 +35,30 @@ __device__ __forceinline__ void bf16x4_to_float4(uint2 raw, float4& o) {
   o = make_float4(fa.x, fa.y, fb.x, fb.y);
 }
 
-__device__ __forceinline__ uint2 float4_to_bf16x4(float4 v) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+// Activations leave these kernels as fp16 (three more mantissa bits than bf16), saturating at
+// the largest finite half.
+__device__ __forceinline__ float sat_h(float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); }
+
+__device__ __forceinline__ uint2 float4_to_f16x4(float4 v) {
+  __half2 a = __floats2half2_rn(sat_h(v.x), sat_h(v.y)), b = __floats2half2_rn(sat_h(v.z), sat_h(v.w));
   uint2 r;
   r.x = *reinterpret_cast<uint32_t*>(&a);
   r.y = *reinterpret_cast<uint32_t*>(&b);
   return r;
 }
 
-// x[t,:] = E[tok[t],:] (kept in fp32 as the residual stream); h[t,:] = bf16(rmsnorm(x) * gain).
+__device__ __forceinline__ void f16x4_to_float4(uint2 raw, float4& o) {
+  const float2 fa = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+  const float2 fb = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+  o = make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+
+// x[t,:] = E[tok[t],:] (kept in fp32 as the residual stream); h[t,:] = fp16(rmsnorm(x) * gain).
 // GATHER = false: x is read instead.
 template <bool GATHER>
 __global__ void __launch_bounds__(NORM_THREADS)
 norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E,
-            const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __nv_bfloat16* __restrict__ h,
+            const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __half* __restrict__ h,
             int d, float eps) {
   __shared__ float red[32];
   const int t = blockIdx.x;
@@ -72,7 +82,7 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
   }
   const float tot = block_sum(ss, red);
   const float rstd = rsqrtf(tot / static_cast<float>(d) + eps);
-  __nv_bfloat16* hrow = h + static_cast<size_t>(t) * d;
+  __half* hrow = h + static_cast<size_t>(t) * d;
 #pragma unroll
   for (int i = 0; i < MAX_VEC; ++i) {
     const int v = threadIdx.x + i * NORM_THREADS;
@@ -81,7 +91,7 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
       bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
       float4 o = make_float4(buf[i].x * rstd * g.x, buf[i].y * rstd * g.y, buf[i].z * rstd * g.z,
                              buf[i].w * rstd * g.w);
-      *reinterpret_cast<uint2*>(hrow + 4 * v) = float4_to_bf16x4(o);
+      *reinterpret_cast<uint2*>(hrow + 4 * v) = float4_to_f16x4(o);
     }
   }
 }
@@ -90,7 +100,7 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
 // pos * theta^(-2i/Dh) from a host-built table) and append of k, v to the request's KV page:
 // position pos lives in page pages[pt_start + pos / P], slot pos % P.
 __global__ void __launch_bounds__(256)
-rope_append_kernel(const float* __restrict__ qkv, __nv_bfloat16* __restrict__ q_out, KvGeom kv, int layer,
+rope_append_kernel(const float* __restrict__ qkv, __half* __restrict__ q_out, KvGeom kv, int layer,
                    const int32_t* __restrict__ row_seg, const int32_t* __restrict__ row_pos,
                    const hb_seg* __restrict__ segs, const int32_t* __restrict__ pages,
                    const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int Hq, int max_pos,
@@ -107,7 +117,7 @@ rope_append_kernel(const float* __restrict__ qkv, __nv_bfloat16* __restrict__ q_
   }
   const int n_qkv = (Hq + 2 * Hkv) * Dh;
   const float* row = qkv + static_cast<size_t>(t) * n_qkv;
-  __nv_bfloat16* kbase = kv.arena + layer * kv.layer_stride + page * kv.page_stride + slot * Dh;
+  __half* kbase = kv.arena + layer * kv.layer_stride + page * kv.page_stride + slot * Dh;
   const int64_t head_stride = static_cast<int64_t>(kv.P) * Dh;
   const float* cs = rope_cos + static_cast<size_t>(pos) * half;
   const float* sn = rope_sin + static_cast<size_t>(pos) * half;
@@ -126,27 +136,27 @@ rope_append_kernel(const float* __restrict__ qkv, __nv_bfloat16* __restrict__ q_
                                     a.w * c.w - b.w * s.w);
       const float4 hi = make_float4(b.x * c.x + a.x * s.x, b.y * c.y + a.y * s.y, b.z * c.z + a.z * s.z,
                                     b.w * c.w + a.w * s.w);
-      __nv_bfloat16* dst = (head < Hq) ? q_out + static_cast<size_t>(t) * Hq * Dh + head * Dh + i
+      __half* dst = (head < Hq) ? q_out + static_cast<size_t>(t) * Hq * Dh + head * Dh + i
                                        : kbase + (head - Hq) * head_stride + i;
-      *reinterpret_cast<uint2*>(dst) = float4_to_bf16x4(lo);
-      *reinterpret_cast<uint2*>(dst + half) = float4_to_bf16x4(hi);
+      *reinterpret_cast<uint2*>(dst) = float4_to_f16x4(lo);
+      *reinterpret_cast<uint2*>(dst + half) = float4_to_f16x4(hi);
     } else {
       const int w = u - rot_units;
       const int head = w / (Dh >> 2), i = (w - head * (Dh >> 2)) << 2;
       const float4 a = *reinterpret_cast<const float4*>(row + (Hq + Hkv + head) * Dh + i);
-      __nv_bfloat16* dst = kbase + (Hkv + head) * head_stride + i;
-      *reinterpret_cast<uint2*>(dst) = float4_to_bf16x4(a);
+      __half* dst = kbase + (Hkv + head) * head_stride + i;
+      *reinterpret_cast<uint2*>(dst) = float4_to_f16x4(a);
     }
   }
 }
 
-// Final RMSNorm of the rows that feed the LM head, written as a (hi, lo) bf16 pair:
-// hi = bf16(y), lo = bf16(y - hi), interleaved in blocks of 64 columns
+// Final RMSNorm of the rows that feed the LM head, written as a (hi, lo) fp16 pair:
+// hi = fp16(y), lo = fp16(y - hi), interleaved in blocks of 64 columns
 // ([hi 0..63 | lo 0..63 | hi 64..127 | ...]).  The LM-head GEMM runs over 2d columns with each
 // weight k-block used twice, which restores near-fp32 input precision for the logits.
 __global__ void __launch_bounds__(NORM_THREADS)
 final_logit_rows_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
-                        const int32_t* __restrict__ logit_src, __nv_bfloat16* __restrict__ out, int d, float eps) {
+                        const int32_t* __restrict__ logit_src, __half* __restrict__ out, int d, float eps) {
   __shared__ float red[32];
   const int i = blockIdx.x;
   const int t = logit_src[i];
@@ -163,7 +173,7 @@ final_logit_rows_kernel(const float* __restrict__ x, const __nv_bfloat16* __rest
     }
   }
   const float rstd = rsqrtf(block_sum(ss, red) / static_cast<float>(d) + eps);
-  __nv_bfloat16* orow = out + static_cast<size_t>(i) * 2 * d;
+  __half* orow = out + static_cast<size_t>(i) * 2 * d;
 #pragma unroll
   for (int k = 0; k < MAX_VEC; ++k) {
     const int v = threadIdx.x + k * NORM_THREADS;
@@ -172,12 +182,12 @@ final_logit_rows_kernel(const float* __restrict__ x, const __nv_bfloat16* __rest
       bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
       const float4 y = make_float4(buf[k].x * rstd * g.x, buf[k].y * rstd * g.y, buf[k].z * rstd * g.z,
                                    buf[k].w * rstd * g.w);
-      const uint2 hi = float4_to_bf16x4(y);
+      const uint2 hi = float4_to_f16x4(y);
       float4 hf;
-      bf16x4_to_float4(hi, hf);
-      const uint2 lo = float4_to_bf16x4(make_float4(y.x - hf.x, y.y - hf.y, y.z - hf.z, y.w - hf.w));
+      f16x4_to_float4(hi, hf);
+      const uint2 lo = float4_to_f16x4(make_float4(y.x - hf.x, y.y - hf.y, y.z - hf.z, y.w - hf.w));
       const int c = 4 * v;
-      __nv_bfloat16* dst = orow + (c >> 6) * 128 + (c & 63);
+      __half* dst = orow + (c >> 6) * 128 + (c & 63);
       *reinterpret_cast<uint2*>(dst) = hi;
       *reinterpret_cast<uint2*>(dst + 64) = lo;
     }
@@ -325,6 +335,24 @@ argmax_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out
   }
 }
 
+// Weight repack: bf16 -> fp16, element by element (in place allowed: each thread reads its 8 values
+// before it writes them).  Exact for 2^-14 <= |w| <= 65504; smaller magnitudes land on the fp16
+// subnormal grid (absolute error <= 2^-25), larger ones saturate.
+__global__ void __launch_bounds__(256)
+bf16_to_f16_kernel(const __nv_bfloat16* src, __half* dst, size_t n_vec, size_t n) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t v = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; v < n_vec; v += stride) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(src + v * 8);
+    float4 a, b;
+    bf16x4_to_float4(make_uint2(raw.x, raw.y), a);
+    bf16x4_to_float4(make_uint2(raw.z, raw.w), b);
+    const uint2 lo = float4_to_f16x4(a), hi = float4_to_f16x4(b);
+    *reinterpret_cast<uint4*>(dst + v * 8) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0)
+    for (size_t i = n_vec * 8; i < n; ++i) dst[i] = __float2half_rn(sat_h(__bfloat162float(src[i])));
+}
+
 int check_launch() { return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA; }
 
 }  // namespace
@@ -364,6 +392,17 @@ int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool
     if (check_launch() != HB_OK) return HB_ERR_CUDA;
   }
   return HB_OK;
+}
+
+int hb_launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s) {
+  if (n == 0) return HB_OK;
+  const size_t n_vec = n / 8;
+  size_t blocks = (n_vec + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  bf16_to_f16_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(src),
+                                                                   static_cast<__half*>(dst), n_vec, n);
+  return check_launch();
 }
 
 int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s) {

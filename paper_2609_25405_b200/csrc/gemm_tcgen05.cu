@@ -1,5 +1,6 @@
-// Projection GEMM for sm_100a: C = epilogue(A * B^T), A [M,K] and B [N,K] bf16 K-major,
-// fp32 accumulation in tensor memory.
+// Projection GEMM for sm_100a: C = epilogue(A * B^T), A [M,K] fp16 activations and B [N,K] fp16 weights
+// (the model's bf16 weights repacked once to fp16; tcgen05 kind::f16 needs one 16-bit format for both
+// operands), both K-major, fp32 accumulation in tensor memory.
 //
 // These are the dense contractions of the shared forward pass (Section 3.1 of the paper:
 // the forward "applies attention and feed-forward layers" to every row of the mixed
@@ -153,10 +154,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
   return d;
 }
 
-// Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128 * CG, N = BN.
+// Instruction descriptor: D fp32 (bit 4), A and B fp16 (format 0 in bits 7-9 and 10-12),
+// both K-major, M = 128 * CG, N = BN.
 template <int BN, int CG>
 __device__ __forceinline__ constexpr uint32_t make_idesc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+  return (1u << 4) | (0u << 7) | (0u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
          (static_cast<uint32_t>((BM * CG) >> 4) << 24);
 }
 
@@ -209,8 +211,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+// Two floats -> packed fp16 pair, saturating at the largest finite half.
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  lo = fminf(fmaxf(lo, -65504.0f), 65504.0f);
+  hi = fminf(fmaxf(hi, -65504.0f), 65504.0f);
+  __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
@@ -220,16 +225,16 @@ __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)
 template <int EPI>
 __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32]) {
   // col0 is a multiple of 32; N is a multiple of 8, so validity is decided per group of 8
-  if constexpr (EPI == HB_EPI_BF16) {
-    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + static_cast<size_t>(row) * g.ldc + col0;
+  if constexpr (EPI == HB_EPI_F16) {
+    __half* out = static_cast<__half*>(g.C) + static_cast<size_t>(row) * g.ldc + col0;
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
       if (col0 + v * 8 < g.N) {
         uint4 pk;
-        pk.x = pack_bf16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-        pk.y = pack_bf16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-        pk.z = pack_bf16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-        pk.w = pack_bf16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+        pk.x = pack_f16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+        pk.y = pack_f16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+        pk.z = pack_f16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+        pk.w = pack_f16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
         *reinterpret_cast<uint4*>(out + v * 8) = pk;
       }
     }
@@ -251,7 +256,7 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
       }
     }
   } else {  // HB_EPI_SWIGLU: columns (2j, 2j+1) = (gate_j, up_j) -> out column j
-    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + static_cast<size_t>(row) * g.ldc + col0 / 2;
+    __half* out = static_cast<__half*>(g.C) + static_cast<size_t>(row) * g.ldc + col0 / 2;
 #pragma unroll
     for (int v = 0; v < 2; ++v) {
       if (col0 + v * 16 < g.N) {
@@ -260,7 +265,7 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
         for (int j = 0; j < 4; ++j) {
           const float g0 = __uint_as_float(r[v * 16 + j * 4 + 0]), u0 = __uint_as_float(r[v * 16 + j * 4 + 1]);
           const float g1 = __uint_as_float(r[v * 16 + j * 4 + 2]), u1 = __uint_as_float(r[v * 16 + j * 4 + 3]);
-          pk[j] = pack_bf16(silu_f(g0) * u0, silu_f(g1) * u1);
+          pk[j] = pack_f16(silu_f(g0) * u0, silu_f(g1) * u1);
         }
         *reinterpret_cast<uint4*>(out + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
@@ -506,7 +511,7 @@ template <int BN, int CG>
 int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, int epi, const GemmArgs& a, int num_sms,
               cudaStream_t s) {
   switch (epi) {
-    case HB_EPI_BF16: return launch_one<BN, HB_EPI_BF16, CG>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_F16: return launch_one<BN, HB_EPI_F16, CG>(tmA, tmB, a, num_sms, s);
     case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, a, num_sms, s);
     case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, a, num_sms, s);
     case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, a, num_sms, s);

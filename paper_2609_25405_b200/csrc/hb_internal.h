@@ -3,6 +3,7 @@
 
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -53,13 +54,14 @@ struct DeviceDesc {
   const hb_seg* segs;       // [R]
   const int32_t* pages;     // [n_page_ids]
   const int32_t* logit_src; // [n_logit_rows] token row feeding logits row i
-  const AttnItem* attn_items;
+  const AttnItem* attn_items;  // decode splits and small chunk tiles (mma.sync kernel)
+  const AttnItem* tc_items;    // 128-row chunk tiles (tcgen05 kernel)
   const PoolItem* pool_items;
-  int32_t T, R, n_logit, n_attn_items, n_pool_items;
+  int32_t T, R, n_logit, n_attn_items, n_tc_items, n_pool_items;
 };
 
 struct KvGeom {
-  __nv_bfloat16* arena;
+  __half* arena;
   int64_t layer_stride;  // elements
   int64_t page_stride;   // elements: 2 * Hkv * P * Dh
   int32_t n_pages, Hkv, P, Dh;
@@ -110,9 +112,11 @@ int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaS
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
 int hb_launch_rope_append(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s);
 int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
+int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
                     int n_slots, float* out_emb, cudaStream_t s);
 int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s);
+int hb_launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s);
 
 struct hb_ctx {
   hb_model_cfg cfg;
@@ -124,12 +128,12 @@ struct hb_ctx {
   size_t ws_bytes;
   // workspace carve-up (device)
   float* x;                 // [max_tokens, d] residual stream, fp32
-  __nv_bfloat16* h;         // [max_tokens, d] normed activations
+  __half* h;                // [max_tokens, d] normed activations (fp16)
   float* qkv;               // [max_tokens, n_qkv] projection output, fp32
-  __nv_bfloat16* q;         // [max_tokens, Hq*Dh] rotated queries
-  __nv_bfloat16* attn_out;  // [max_tokens, Hq*Dh]
-  __nv_bfloat16* act;       // [max_tokens, F]
-  __nv_bfloat16* logit_in;  // [max_logit_rows, 2d] hi/lo split of final hidden rows
+  __half* q;                // [max_tokens, Hq*Dh] rotated queries (fp16)
+  __half* attn_out;         // [max_tokens, Hq*Dh] (fp16)
+  __half* act;              // [max_tokens, F] (fp16)
+  __half* logit_in;         // [max_logit_rows, 2d] hi/lo fp16 split of final hidden rows
   float* rope_cos;          // [max_pos, Dh/2]
   float* rope_sin;
   float* attn_part;         // split-KV partial results

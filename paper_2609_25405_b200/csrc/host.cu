@@ -12,7 +12,8 @@
 namespace {
 
 constexpr int POOL_ROWS = 32;   // rows per pooling work item
-constexpr int ATT_TILE_ROWS = 64;   // query rows (tokens x grouped heads) per chunk attention item
+constexpr int ATT_TILE_ROWS = 64;   // query rows (tokens x grouped heads) per small chunk attention item
+constexpr int ATT_TC_ROWS = 128;    // query rows per tcgen05 chunk attention item
 constexpr int ATT_SPLIT_KEYS = 512; // keys per decode attention item; depends on nothing but this constant
 constexpr int N_STAGING = 4;    // pinned descriptor staging ring
 
@@ -86,7 +87,7 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   dc += align_up(static_cast<size_t>(max_segs) * 4, 16);                // logit_src
   dc += align_up(static_cast<size_t>(L.max_attn_items) * sizeof(AttnItem), 16);
   dc += align_up(static_cast<size_t>(L.max_pool_items) * sizeof(PoolItem), 16);
-  L.desc_cap = dc + 64;
+  L.desc_cap = dc + 128;
   L.desc = cv.take(L.desc_cap);
   L.total = cv.off;
   return L;
@@ -236,12 +237,12 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   }
   c->ws_bytes = lay.total;
   c->x = reinterpret_cast<float*>(c->ws + lay.x);
-  c->h = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.h);
+  c->h = reinterpret_cast<__half*>(c->ws + lay.h);
   c->qkv = reinterpret_cast<float*>(c->ws + lay.qkv);
-  c->q = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.q);
-  c->attn_out = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.attn_out);
-  c->act = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.act);
-  c->logit_in = reinterpret_cast<__nv_bfloat16*>(c->ws + lay.logit_in);
+  c->q = reinterpret_cast<__half*>(c->ws + lay.q);
+  c->attn_out = reinterpret_cast<__half*>(c->ws + lay.attn_out);
+  c->act = reinterpret_cast<__half*>(c->ws + lay.act);
+  c->logit_in = reinterpret_cast<__half*>(c->ws + lay.logit_in);
   c->rope_cos = reinterpret_cast<float*>(c->ws + lay.rope_cos);
   c->rope_sin = reinterpret_cast<float*>(c->ws + lay.rope_sin);
   c->attn_part = reinterpret_cast<float*>(c->ws + lay.attn_part);
@@ -535,7 +536,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
   if (static_cast<int32_t>(pitems.size()) > ex->lay.max_pool_items) return HB_ERR_TOO_LARGE;
   // attention work list: chunk items (64 query rows x all visible keys) and decode items (one
   // split of ATT_SPLIT_KEYS keys); sorted by cost, largest first, so the tail of the launch is short
-  std::vector<AttnItem> aitems;
+  std::vector<AttnItem> aitems, titems;
   {
     const int G = cfg.n_heads / cfg.n_kv_heads;
     int32_t rec_at = 0;
@@ -558,14 +559,17 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
           }
           rec_at += ns;
         } else {
+          // chunk rows: full 128-row tiles (and a remainder above 64 rows) go to the tcgen05 kernel,
+          // a remainder of at most 64 rows to the mma.sync kernel
           const int32_t rows = sg.q_len * G;
-          for (int32_t row0 = 0; row0 < rows; row0 += ATT_TILE_ROWS) {
+          for (int32_t row0 = 0; row0 < rows; row0 += ATT_TC_ROWS) {
             AttnItem it{};
-            it.seg = r; it.kv_head = hk; it.row0 = row0; it.n_rows = std::min(ATT_TILE_ROWS, rows - row0);
+            it.seg = r; it.kv_head = hk; it.row0 = row0; it.n_rows = std::min(ATT_TC_ROWS, rows - row0);
             it.key0 = 0;
             it.key1 = sg.pos_start + (row0 + it.n_rows - 1) / G + 1;
             it.split = 0; it.n_splits = 1; it.part_base = 0; it.mode = 0;
-            aitems.push_back(it);
+            if (it.n_rows <= ATT_TILE_ROWS) aitems.push_back(it);
+            else titems.push_back(it);
           }
         }
       }
@@ -575,14 +579,18 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     };
     std::stable_sort(aitems.begin(), aitems.end(),
                      [&](const AttnItem& a, const AttnItem& b) { return cost(a) > cost(b); });
-    if (static_cast<int32_t>(aitems.size()) > ex->lay.max_attn_items) return HB_ERR_TOO_LARGE;
+    std::stable_sort(titems.begin(), titems.end(),
+                     [&](const AttnItem& a, const AttnItem& b) { return cost(a) > cost(b); });
+    if (static_cast<int32_t>(aitems.size() + titems.size()) > ex->lay.max_attn_items) return HB_ERR_TOO_LARGE;
     if (static_cast<size_t>(rec_at) * G * (cfg.head_dim + 2) > c->attn_part_floats) return HB_ERR_TOO_LARGE;
   }
   const size_t o_aitems = place(aitems.size() * sizeof(AttnItem));
+  const size_t o_titems = place(titems.size() * sizeof(AttnItem));
   const size_t o_pitems = place(pitems.size() * sizeof(PoolItem));
   if (off > c->desc_cap) return HB_ERR_TOO_LARGE;
   if (!pitems.empty()) memcpy(st.host + o_pitems, pitems.data(), pitems.size() * sizeof(PoolItem));
   if (!aitems.empty()) memcpy(st.host + o_aitems, aitems.data(), aitems.size() * sizeof(AttnItem));
+  if (!titems.empty()) memcpy(st.host + o_titems, titems.data(), titems.size() * sizeof(AttnItem));
   if (cudaMemcpyAsync(c->desc_dev, st.host, off, cudaMemcpyHostToDevice, s) != cudaSuccess) return HB_ERR_CUDA;
   if (cudaEventRecord(st.ev, s) != cudaSuccess) return HB_ERR_CUDA;
   st.pending = true;
@@ -595,15 +603,17 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
   dd.pages = reinterpret_cast<const int32_t*>(c->desc_dev + o_pages);
   dd.logit_src = reinterpret_cast<const int32_t*>(c->desc_dev + o_lsrc);
   dd.attn_items = reinterpret_cast<const AttnItem*>(c->desc_dev + o_aitems);
+  dd.tc_items = reinterpret_cast<const AttnItem*>(c->desc_dev + o_titems);
   dd.pool_items = reinterpret_cast<const PoolItem*>(c->desc_dev + o_pitems);
   dd.T = T;
   dd.R = R;
   dd.n_logit = d->n_logit_rows;
   dd.n_attn_items = static_cast<int32_t>(aitems.size());
+  dd.n_tc_items = static_cast<int32_t>(titems.size());
   dd.n_pool_items = static_cast<int32_t>(pitems.size());
 
   KvGeom kg;
-  kg.arena = static_cast<__nv_bfloat16*>(kv->arena);
+  kg.arena = static_cast<__half*>(kv->arena);
   kg.Hkv = cfg.n_kv_heads;
   kg.P = cfg.page_size;
   kg.Dh = cfg.head_dim;
@@ -665,7 +675,8 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     ga.C = c->qkv; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rope_append(c, kg, l, s));
-    HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
+    if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention_tc(c, kg, kv->map, l, s));
+    if (dd.n_attn_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s));
@@ -707,6 +718,17 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
 int hb_argmax(hb_ctx* c, const float* logits, int32_t n_rows, int32_t* out_tokens, void* stream) {
   if (!c || n_rows < 0 || (n_rows > 0 && (!logits || !out_tokens))) return HB_ERR_BAD_ARG;
   return hb_launch_argmax(logits, n_rows, c->cfg.vocab, out_tokens, static_cast<cudaStream_t>(stream));
+}
+
+int hb_weights_pack_f16(const void* src_bf16, void* dst_f16, size_t n_elems, void* stream) {
+  if (!src_bf16 || !dst_f16) return HB_ERR_BAD_ARG;
+  if ((reinterpret_cast<uintptr_t>(src_bf16) & 15u) || (reinterpret_cast<uintptr_t>(dst_f16) & 15u)) return HB_ERR_BAD_ARG;
+  if (src_bf16 != dst_f16) {   // partial overlap would corrupt the input
+    const char* a = static_cast<const char*>(src_bf16);
+    const char* b = static_cast<const char*>(dst_f16);
+    if (a < b + n_elems * 2 && b < a + n_elems * 2) return HB_ERR_BAD_ARG;
+  }
+  return hb_launch_bf16_to_f16(src_bf16, dst_f16, n_elems, static_cast<cudaStream_t>(stream));
 }
 
 int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
@@ -758,7 +780,7 @@ int hb_last_launch_count(const hb_ctx* c, int32_t* out_count) {
 int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int32_t epilogue,
             void* stream) {
   if (!c || !A || !B || !C || M < 1 || N < 8 || K < 8 || (N & 7) || (K & 7)) return HB_ERR_BAD_ARG;
-  if (epilogue < HB_EPI_BF16 || epilogue > HB_EPI_SWIGLU) return HB_ERR_BAD_ARG;
+  if (epilogue < HB_EPI_F16 || epilogue > HB_EPI_SWIGLU) return HB_ERR_BAD_ARG;
   if (epilogue == HB_EPI_SWIGLU && (N & 15)) return HB_ERR_BAD_ARG;
   if (reinterpret_cast<uintptr_t>(C) & 15u) return HB_ERR_BAD_ARG;
   const int bn = hb_gemm_pick_bn(M, N, c->num_sms);

@@ -67,23 +67,50 @@ class Weights:
     Interface used by the checker: .tok_emb, .final_norm, .lm_head and
     .layer(l) -> dict.  `cache=True` keeps generated tensors (small models)."""
 
-    def __init__(self, shape: ModelShape, seed: int = 0, std: float = 0.02, cache: bool = True):
+    def __init__(self, shape: ModelShape, seed: int = 0, std: float = 0.02, cache=True):
+        """cache: True keeps float32 tensors, "bits" keeps the uint16 bf16 patterns (half the
+        memory; converted on access), False regenerates on every access."""
         self.shape = shape
         self.seed = seed
         self.std = std
         self._cache = {} if cache else None
+        self._bits = (cache == "bits")
+
+    def _normal_bits(self, key, rows, cols):
+        rng = np.random.default_rng([self.seed, key[0], key[1]])
+        a = rng.standard_normal((rows, cols), dtype=np.float32)
+        a *= np.float32(self.std)
+        return f32_to_bf16_bits(a).reshape(rows, cols)
 
     def _normal_bf16(self, key, rows, cols):
-        rng = np.random.default_rng([self.seed, key[0], key[1]])
-        a = rng.standard_normal((rows, cols), dtype=np.float32) * np.float32(self.std)
-        return bf16_bits_to_f32(f32_to_bf16_bits(a)).reshape(rows, cols)
+        if self._bits:
+            return self._normal_bits(key, rows, cols)
+        return bf16_bits_to_f32(self._normal_bits(key, rows, cols)).reshape(rows, cols)
 
     def _get(self, key, maker):
         if self._cache is None:
-            return maker()
-        if key not in self._cache:
-            self._cache[key] = maker()
-        return self._cache[key]
+            v = maker()
+        else:
+            if key not in self._cache:
+                self._cache[key] = maker()
+            v = self._cache[key]
+        if v.dtype == np.uint16:
+            return bf16_bits_to_f32(v).reshape(v.shape)
+        return v
+
+    def prefetch(self, threads=8):
+        """Generate every tensor into the cache with a thread pool (numpy releases the GIL)."""
+        from concurrent.futures import ThreadPoolExecutor
+        jobs = [(l, n) for l in range(self.shape.L) for n in _TENSOR_IDS] + [(None, "tok_emb"), (None, "lm_head")]
+
+        def run(j):
+            if j[0] is None:
+                getattr(self, j[1])
+            else:
+                self.tensor(*j)
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(run, jobs))
+        return self
 
     def tensor(self, layer, name):
         s = self.shape

@@ -22,6 +22,11 @@ def _bf16_exact(rng, shape, std):
     return synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(a)).reshape(shape)
 
 
+def _f16_exact(rng, shape, std):
+    a = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
+    return a.astype(np.float16).astype(np.float32)
+
+
 # (M, N, K): several tiles, ragged M tail, N not a multiple of the tile, K not a multiple of 64,
 # a single row, more tiles than SMs (persistent loop + both TMEM accumulators), long K (ring wraps)
 SHAPES = [(128, 256, 64), (68, 768, 256), (300, 328, 200), (1, 1024, 256), (4, 1024, 512),
@@ -29,24 +34,24 @@ SHAPES = [(128, 256, 64), (68, 768, 256), (300, 328, 200), (1, 1024, 256), (4, 1
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
-@pytest.mark.parametrize("epi", ["f32", "bf16", "resid", "swiglu"])
+@pytest.mark.parametrize("epi", ["f32", "f16", "resid", "swiglu"])
 def test_gemm_matches_oracle(ctx, M, N, K, epi):
     from paper_2609_25405_b200 import binding as B
     if epi == "swiglu" and N % 16:
         pytest.skip("swiglu needs N % 16 == 0")
     rng = np.random.default_rng(M * 7 + N * 3 + K)
-    A = _bf16_exact(rng, (M, K), 1.0)
+    A = _f16_exact(rng, (M, K), 1.0)         # activations are fp16; bf16 weight values repacked to fp16
     Bm = _bf16_exact(rng, (N, K), 0.05)
-    dA, dB = B.bf16_from_f32(A), B.bf16_from_f32(Bm)
+    dA, dB = torch.from_numpy(A.astype(np.float16)).cuda(), B.pack_f16_(B.bf16_from_f32(Bm))
     scale = 0.05 * np.sqrt(K)
     if epi == "f32":
         out = torch.full((M + 1, N), 768.0, dtype=torch.float32, device="cuda")
         ctx.gemm(dA, dB, out, M, N, K, B.EPI_F32)
         ref = ops.projection(A, Bm, "plain")
         tol = 2e-5 * scale * np.sqrt(K) + 1e-6
-    elif epi == "bf16":
-        out = torch.full((M + 1, N), 768.0, dtype=torch.bfloat16, device="cuda")
-        ctx.gemm(dA, dB, out, M, N, K, B.EPI_BF16)
+    elif epi == "f16":
+        out = torch.full((M + 1, N), 768.0, dtype=torch.float16, device="cuda")
+        ctx.gemm(dA, dB, out, M, N, K, B.EPI_F16)
         ref = ops.projection(A, Bm, "plain")
         tol = None
     elif epi == "resid":
@@ -56,15 +61,15 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
         ref = ops.projection(A, Bm, "resid", C0[:M])
         tol = 2e-5 * scale * np.sqrt(K) + 1e-5
     else:
-        out = torch.full((M + 1, N // 2), 768.0, dtype=torch.bfloat16, device="cuda")
+        out = torch.full((M + 1, N // 2), 768.0, dtype=torch.float16, device="cuda")
         ctx.gemm(dA, dB, out, M, N, K, B.EPI_SWIGLU)
         ref = ops.projection(A, Bm, "swiglu")
         tol = None
     assert ctx.status_poll() == 0
     got = out.float().cpu().numpy().astype(np.float64)
-    if tol is None:   # bf16 output: one rounding of the fp32 result (2^-9 relative) + accumulation noise
+    if tol is None:   # fp16 output: one rounding of the fp32 result (2^-11 relative) + accumulation noise
         err = np.abs(got[:M] - ref)
-        assert np.all(err <= np.abs(ref) * 2.0 ** -8 + 2e-5 * scale * np.sqrt(K) + 1e-6), err.max()
+        assert np.all(err <= np.abs(ref) * 2.0 ** -10 + 2e-5 * scale * np.sqrt(K) + 1e-6), err.max()
     else:
         assert np.max(np.abs(got[:M] - ref)) <= tol
     # the row after the last one is never touched
@@ -72,3 +77,22 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
         assert np.array_equal(got[M], C0[M].astype(np.float64))
     else:
         assert np.all(got[M] == 768.0)
+
+
+def test_weights_pack_f16_matches_round_to_nearest(ctx):
+    """bf16 -> fp16 repack: exact in the fp16 normal range, round-to-nearest on the subnormal grid,
+    saturating above 65504; in place."""
+    from paper_2609_25405_b200 import binding as B
+    rng = np.random.default_rng(3)
+    vals = _bf16_exact(rng, (1, 4099), 0.02).ravel()
+    special = np.array([0.0, -0.0, 2.0 ** -14, 2.0 ** -15, 3e-8, -1e-9, 65280.0, 1e6, -1e6, 1.0], dtype=np.float32)
+    vals[:special.size] = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(special))
+    t = B.bf16_from_f32(vals)
+    h = B.pack_f16_(t)
+    torch.cuda.synchronize()
+    got = h.float().cpu().numpy()
+    ref = np.clip(vals, -65504.0, 65504.0).astype(np.float16).astype(np.float32)
+    assert np.array_equal(got, ref)
+    normal = np.abs(vals) >= 2.0 ** -14
+    assert np.array_equal(got[normal & (np.abs(vals) <= 65504)], vals[normal & (np.abs(vals) <= 65504)])
+    assert np.max(np.abs(got - vals)[~normal]) <= 2.0 ** -25

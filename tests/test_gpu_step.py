@@ -94,7 +94,7 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
         _check_emb(ge[j].astype(np.float64), re_[j])
     # ---- KV bookkeeping: exactly the expected slots were written, everything else is the sentinel
     W = weights[0]
-    kvv = eng.kv.view().cpu()                                   # [L, page, 2, Hkv, P, Dh] bf16
+    kvv = eng.kv.view().cpu()                                   # [L, page, 2, Hkv, P, Dh] fp16
     raw = eng.kv.arena.cpu().view(TINY.L, eng.kv.n_pages, 2, TINY.Hkv, 16, TINY.Dh)
     touched = torch.zeros((eng.kv.n_pages, 16), dtype=torch.bool)
     for req in gens + embs:
@@ -109,8 +109,8 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
             slots = torch.tensor([M.kv_slot(req.pages, p, 16)[1] for p in range(n)])
             k_gpu = kvv[l, :, 0][pages, :, slots, :].float().numpy()   # [n, Hkv, Dh]
             v_gpu = kvv[l, :, 1][pages, :, slots, :].float().numpy()
-            assert np.max(np.abs(k_gpu - kv_ref[l][0])) < 2e-2
-            assert np.max(np.abs(v_gpu - kv_ref[l][1])) < 2e-2
+            assert np.max(np.abs(k_gpu - kv_ref[l][0])) < 5e-3
+            assert np.max(np.abs(v_gpu - kv_ref[l][1])) < 5e-3
     untouched = ~touched[None, :, None, None, :, None].expand_as(raw)
     assert torch.all(raw[untouched] == KV_SENTINEL)
     # ---- pool bookkeeping: counters equal the oracle's integers; unused slots keep the sentinel
@@ -167,6 +167,33 @@ def test_random_chunkings_and_chunk_size_one(weights, mode):
         for j in (0, 1):
             _check_emb(ge[j].astype(np.float64), re_[j])
         eng.close()
+
+
+def test_long_chunks_take_the_tensor_core_attention_path(weights):
+    """Chunks of more than 64 query rows run on the tcgen05 attention kernel (128-row tiles, ragged
+    last tile, several key tiles, chunks that start inside a page); shorter remainders on the
+    mma.sync kernel.  Both must reproduce the single-pass oracle."""
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Request
+    W = weights[0]
+    rng = np.random.default_rng(11)
+    e1 = Request("embed", synth.token_ids(rng, 300, TINY.V), B.POOL_MEAN)
+    e2 = Request("embed", synth.token_ids(rng, 213, TINY.V), B.POOL_LAST)
+    g = Request("gen", synth.token_ids(rng, 200, TINY.V))
+    eng = _engine(weights, n_pages=96, max_tokens=768, max_pos=320)
+    _, _, _ = eng.step([(e1, 130), (g, 129), (e2, 213)])
+    _, lr, er = eng.step([(e1, 170), (g, 71)])
+    torch.cuda.synchronize()
+    assert eng.ctx.status_poll() == 0
+    _check_emb(eng.out_emb[er[e1]].cpu().numpy().astype(np.float64), T.embed(TINY, W, e1.tokens, "mean"))
+    _, ref = T.forward(TINY, W, g.tokens, logit_rows=[199])
+    assert np.max(np.abs(eng.out_logits[lr[g]].cpu().numpy() - ref[0])) <= LOGIT_ABS
+    eng2 = _engine(weights, n_pages=96, max_tokens=768, max_pos=320)
+    e2b = Request("embed", e2.tokens, B.POOL_LAST)
+    _, _, er = eng2.step([(e2b, 213)])
+    torch.cuda.synchronize()
+    _check_emb(eng2.out_emb[er[e2b]].cpu().numpy().astype(np.float64), T.embed(TINY, W, e2.tokens, "last"))
+    eng.close(); eng2.close()
 
 
 def test_batch_composition_independence(weights):
