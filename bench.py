@@ -191,6 +191,7 @@ def main():
     ap.add_argument("--packer-warm", type=int, default=50, help="host-only packer steps before the first GPU step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-alias", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -216,6 +217,8 @@ def main():
     if world > 1:   # independent replicas: each rank draws its own batch stream
         spec = workloads.MixSpec(**{**spec.__dict__, "seed": spec.seed + 7919 * rank})
     shape = synth.SHAPES[spec.shape]
+    if args.layers:
+        shape = shape.with_layers(args.layers)
     n_steps_total = args.warmup + args.steps
     max_pos = spec.ctx_hi + n_steps_total + 8 if spec.n_decode else spec.emb_hi + 8
     max_pos = max(max_pos, spec.emb_hi + 8)
@@ -236,7 +239,7 @@ def main():
         kvb[i:i + step_e].normal_(0.0, 1.0)
     pool = B.Pool(cfg, 256)
     ctx = B.Context(cfg, spec.budget, max_segs, max_page_ids)
-    wl = workloads.MixedWorkload(spec, kv, pool, max_pos, decode_alias=args.decode_alias)
+    wl = workloads.MixedWorkload(spec, kv, pool, max_pos, decode_alias=args.decode_alias, shape=shape)
     for _ in range(args.packer_warm):                # reach the packer's steady state (host only)
         _, commit = wl.next_step()
         commit(advance_decode=False)
@@ -354,7 +357,7 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "precision": "bf16 weights x fp16 activations / KV cache on the tensor cores, fp32 accumulation, "
                          "fp32 residual stream, norms, softmax and pooling",
-            "config": {"workload": spec.name, "shape": spec.shape, "tokens_per_step": w["T"],
+            "config": {"workload": spec.name, "shape": shape.name, "tokens_per_step": w["T"],
                        "decode_rows": spec.n_decode, "chunk": spec.chunk, "token_budget": spec.budget,
                        "l2": "inputs larger than L2 (weights and KV pages are re-streamed every step)",
                        "replicas": world, "decode_alias": args.decode_alias},

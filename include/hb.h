@@ -233,11 +233,12 @@ HB_API int hb_status_poll(hb_ctx* ctx, void* stream, uint32_t* out_code);
  * entries, and clears the record.  Classes: */
 enum {
   HB_CLASS_GEMM = 0,      /* QKV, O, gate/up, down projections                          */
-  HB_CLASS_ATTENTION = 1, /* varlen paged attention                                     */
+  HB_CLASS_ATTENTION = 1, /* paged attention: decode splits and short chunk tiles       */
   HB_CLASS_NORM_ROPE = 2, /* gather + RMSNorm, RMSNorm, RoPE + KV append                */
   HB_CLASS_POOL = 3,      /* final RMSNorm + pooler / logits-row preparation            */
   HB_CLASS_LM_HEAD = 4,   /* LM-head projection                                         */
-  HB_N_CLASSES = 5
+  HB_CLASS_ATTENTION_TC = 5, /* chunk-row attention on the tcgen05 tensor cores         */
+  HB_N_CLASSES = 6
 };
 HB_API int hb_profile_enable(hb_ctx* ctx, int on);
 HB_API int hb_profile_read(hb_ctx* ctx, float* ms_by_class, int32_t* launches_by_class);
@@ -262,6 +263,24 @@ enum {
  * aligned; K and N multiples of 8.  M may be any value >= 1. */
 HB_API int hb_gemm(hb_ctx* ctx, const void* A, const void* B, void* C, int32_t M, int32_t N,
             int32_t K, int32_t epilogue, void* stream);
+
+/* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
+ * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of
+ * the chunk's rows, then
+ *   mean: S <- S + sum_j rmsnorm(x_j) * gain, count <- count + n_rows
+ *         (first_chunk != 0 starts from S = 0, count = 0);
+ *   last: only the counters move until the final chunk;
+ * and on the final chunk out_emb = L2-normalised S / count (mean) or the
+ * normed last row (last).
+ *   x          device float [n_rows, d_model] residual-stream rows of the chunk
+ *   gain       device bf16 [d_model] final-norm gain
+ *   slot_sum   device float [d_model], slot_meta device uint32 [4] =
+ *              {count, chunks, mode, state}: the request's pool slot (in/out)
+ *   out_emb    device float [d_model] (written when is_final != 0)
+ * n_rows <= the context's max_tokens.  Uses the context's scratch. */
+HB_API int hb_pool_chunk(hb_ctx* ctx, const float* x, const void* gain, int32_t n_rows, int32_t mode,
+                         int32_t first_chunk, int32_t is_final, float* slot_sum, uint32_t* slot_meta,
+                         float* out_emb, void* stream);
 
 #ifdef __cplusplus
 }

@@ -84,6 +84,7 @@ _sig = {
     "hb_mixed_step": [_P, C.POINTER(BatchDesc), C.POINTER(Weights), _P, _P, _P, _P, _P],
     "hb_weights_pack_f16": [_P, _P, C.c_size_t, _P],
     "hb_argmax": [_P, _P, C.c_int32, _P, _P],
+    "hb_pool_chunk": [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P],
     "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
     "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
     "hb_profile_enable": [_P, C.c_int],
@@ -336,6 +337,13 @@ class Context:
     def gemm(self, A, B, Cout, M, N, K, epilogue, stream=None):
         check(lib.hb_gemm(self.handle, C.c_void_p(A.data_ptr()), C.c_void_p(B.data_ptr()),
                           C.c_void_p(Cout.data_ptr()), M, N, K, epilogue, _stream_ptr(stream)), "hb_gemm")
+
+    def pool_chunk(self, x, gain, n_rows, mode, first_chunk, is_final, slot_sum, slot_meta, out_emb, stream=None):
+        check(lib.hb_pool_chunk(self.handle, C.c_void_p(x.data_ptr()), C.c_void_p(gain.data_ptr()), n_rows, mode,
+                                1 if first_chunk else 0, 1 if is_final else 0, C.c_void_p(slot_sum.data_ptr()),
+                                C.c_void_p(slot_meta.data_ptr()),
+                                C.c_void_p(out_emb.data_ptr()) if out_emb is not None else None,
+                                _stream_ptr(stream)), "hb_pool_chunk")
 
     def status_poll(self, stream=None):
         """Synchronises the stream; returns the device status code (0 = clean)."""

@@ -166,11 +166,17 @@ struct TcCfg {
 
 template <int DH>
 __global__ void __launch_bounds__(TC_THREADS, 2)
-attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams p, int max_blk) {
+attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams p) {
   using C = TcCfg<DH>;
   extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
+  // The kernel has no static shared memory, so the dynamic window starts at the CTA's (1 KiB
+  // aligned) shared-memory base, which the swizzled tiles need; checked, not assumed.
+  const uint32_t base = smem_u32(smem_raw);
+  uint8_t* smem = smem_raw;
+  if (base & 1023u) {
+    if (threadIdx.x == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
+    return;
+  }
   const uint32_t q_s = base, ring_s = base + C::Q_BYTES, p_s = ring_s + C::RING, bar_s = base + C::BAR_OFF;
   auto kv_full = [&](int s) { return bar_s + 8u * s; };
   auto kv_empty = [&](int s) { return bar_s + 8u * (C::STAGES + s); };
@@ -179,7 +185,6 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   const uint32_t p_ready = bar_s + 8u * (2 * C::STAGES + 4), pv_done = bar_s + 8u * (2 * C::STAGES + 5);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  int32_t* pg_s = reinterpret_cast<int32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16);
 
   const AttnItem it = p.items[blockIdx.x];
   const hb_seg sg = p.segs[it.seg];
@@ -196,11 +201,11 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // page ids are checked once here; the producer reads them from global memory as it goes
   int bad = 0;
   for (int i = tid; i < n_blk; i += TC_THREADS) {
-    const int pg = (i < sg.pt_len && i < max_blk) ? p.pages[sg.pt_start + i] : -1;
+    const int pg = (i < sg.pt_len) ? p.pages[sg.pt_start + i] : -1;
     bad |= (pg < 0 || pg >= p.n_pages);
-    if (i < max_blk) pg_s[i] = pg;
   }
   // Q tile -> shared memory in the K-major 128-byte-swizzled layout ([SUB][128 rows][64]); rows past
   // n_rows are zero
@@ -240,7 +245,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         const uint32_t k_dst = ring_s + st * 2 * C::KV_HALF;
         mbar_arrive_expect_tx(kv_full(st), static_cast<uint32_t>(n_pg) * 2u * C::SUB * (16 * 128));
         for (int pi = 0; pi < n_pg; ++pi) {
-          const int64_t page = pg_s[kb / 16 + pi];
+          const int64_t page = __ldg(p.pages + sg.pt_start + kb / 16 + pi);
           const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.n_pages + page) * 2) * p.Hkv + hk) * 16);
           const int row_v = row_k + p.Hkv * 16;
 #pragma unroll
@@ -432,8 +437,8 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 template <int DH>
 int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_pos, cudaStream_t s) {
   using C = TcCfg<DH>;
-  const int max_blk = max_pos / 16 + 2;
-  const int smem = C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16 + max_blk * 4 + 1024;
+  (void)max_pos;
+  const int smem = C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16;   // two CTAs per SM at Dh = 128
   static int configured = 0;
   if (smem > 227 * 1024) return HB_ERR_UNSUPPORTED;
   if (configured < smem) {
@@ -441,7 +446,7 @@ int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_po
       return HB_ERR_CUDA;
     configured = smem;
   }
-  attn_chunk_tc_kernel<DH><<<n_items, TC_THREADS, smem, s>>>(kv_map, p, max_blk);
+  attn_chunk_tc_kernel<DH><<<n_items, TC_THREADS, smem, s>>>(kv_map, p);
   return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
 }
 

@@ -4,36 +4,9 @@
 // All global accesses are 16-byte vectors; row statistics use warp shuffles; sums run in a
 // fixed order (no floating-point atomics), so results do not depend on what else is batched.
 #include "hb_internal.h"
+#include "pool_block.cuh"
 
 namespace {
-
-constexpr int NORM_THREADS = 256;
-constexpr int MAX_VEC = 8;  // float4 per thread held in registers: d_model <= 256 * 4 * 8 = 8192
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// Sum over the block; every thread gets the result.  red must hold 32 floats.
-__device__ __forceinline__ float block_sum(float v, float* red) {
-  v = warp_sum(v);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  __syncthreads();
-  if (lane == 0) red[warp] = v;
-  __syncthreads();
-  float t = (lane < (blockDim.x >> 5)) ? red[lane] : 0.0f;
-  t = warp_sum(t);
-  return t;
-}
-
-__device__ __forceinline__ void bf16x4_to_float4(uint2 raw, float4& o) {
-  const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
-  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
-  const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
-  o = make_float4(fa.x, fa.y, fb.x, fb.y);
-}
 
 // Activations leave these kernels as fp16 (three more mantissa bits than bf16), saturating at
 // the largest finite half.
@@ -194,118 +167,37 @@ final_logit_rows_kernel(const float* __restrict__ x, const __nv_bfloat16* __rest
   }
 }
 
-// Final RMSNorm fused with the incremental pooler.  One block per work item = a block of rows
-// of one embedding segment.  Phase 1: one warp per row, shuffle-reduced sum of squares.
-// Phase 2: each thread owns column vectors and adds x * rstd over the item's rows in row
-// order.  The block's partial sum goes to scratch; the block that arrives last for a segment
-// adds the partials in block order, applies the gain, and updates the slot:
-//   S <- S + partial, count <- count + q_len            (Eq. 1-2 with w = 1)
-// (a request's first chunk overwrites instead, i.e. S(0) = 0, W(0) = 0).  On the final chunk
-// it emits S / count (mean) or the normed last row (last-token head), L2-normalised.
 __global__ void __launch_bounds__(NORM_THREADS)
 final_pool_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
                   const PoolItem* __restrict__ items, const hb_seg* __restrict__ segs, float* __restrict__ part,
                   uint32_t* __restrict__ counters, float* __restrict__ pool_sum, uint32_t* __restrict__ pool_meta,
                   float* __restrict__ out_emb, int d, float eps, int n_slots, uint32_t* status) {
-  __shared__ float red[32];
-  __shared__ float rstd_s[32];
-  __shared__ uint32_t is_last_s;
   const PoolItem it = items[blockIdx.x];
   const hb_seg sg = segs[it.seg];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nv = d >> 2;
-  if (sg.pool_slot < 0 || sg.pool_slot >= n_slots) {
-    if (threadIdx.x == 0) atomicOr(status, HB_DEV_POOL_BAD_INDEX);
-    return;
+  pool_block(it, sg, x, gain, part, counters, pool_sum, pool_meta, out_emb, d, eps, n_slots, status);
+}
+
+// The pooler on its own: one chunk of one request, rows x[0 .. n_rows), slot 0 of a one-slot pool.
+// Block b handles rows [32 b, 32 b + 32) (mean) or the last row (last-token head).
+__global__ void __launch_bounds__(NORM_THREADS)
+pool_chunk_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain, int n_rows, int mode,
+                  int first_chunk, int is_final, float* __restrict__ part, uint32_t* __restrict__ counters,
+                  float* __restrict__ slot_sum, uint32_t* __restrict__ slot_meta, float* __restrict__ out_emb, int d,
+                  float eps, uint32_t* status) {
+  hb_seg sg;
+  sg.kind = HB_KIND_EMBED_CHUNK; sg.q_start = 0; sg.q_len = n_rows; sg.pos_start = first_chunk ? 0 : 1;
+  sg.pt_start = 0; sg.pt_len = 0; sg.pool_slot = 0; sg.pool_mode = mode; sg.is_final = is_final;
+  sg.logits_row = -1; sg.emb_row = 0; sg.reserved = 0;
+  PoolItem it;
+  it.seg = 0; it.block = blockIdx.x; it.n_blocks = gridDim.x; it.part_base = 0; it.pad[0] = it.pad[1] = 0;
+  if (mode == HB_POOL_MEAN) {
+    it.row0 = blockIdx.x * 32;
+    it.n_rows = min(32, n_rows - it.row0);
+  } else {
+    it.row0 = n_rows - 1;
+    it.n_rows = is_final ? 1 : 0;
   }
-  // phase 1: row statistics (item rows <= 32)
-  for (int r = warp; r < it.n_rows; r += NORM_THREADS / 32) {
-    const float* xrow = x + static_cast<size_t>(it.row0 + r) * d;
-    float ss = 0.0f;
-    for (int v = lane; v < nv; v += 32) {
-      const float4 a = *reinterpret_cast<const float4*>(xrow + 4 * v);
-      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
-    }
-    ss = warp_sum(ss);
-    if (lane == 0) rstd_s[r] = rsqrtf(ss / static_cast<float>(d) + eps);
-  }
-  __syncthreads();
-  // phase 2: column sums over the item's rows, fixed row order
-  float* my_part = part + static_cast<size_t>(it.part_base + it.block) * d;
-#pragma unroll 1
-  for (int v = threadIdx.x; v < nv; v += NORM_THREADS) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int r = 0; r < it.n_rows; ++r) {
-      const float4 a = *reinterpret_cast<const float4*>(x + static_cast<size_t>(it.row0 + r) * d + 4 * v);
-      const float s = rstd_s[r];
-      acc.x += a.x * s; acc.y += a.y * s; acc.z += a.z * s; acc.w += a.w * s;
-    }
-    *reinterpret_cast<float4*>(my_part + 4 * v) = acc;
-  }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const uint32_t prev = atomicAdd(counters + it.seg, 1u);
-    is_last_s = (prev + 1u == static_cast<uint32_t>(it.n_blocks)) ? 1u : 0u;
-  }
-  __syncthreads();
-  if (!is_last_s) return;
-  __threadfence();
-  // segment tail: combine partials in block order, update the slot, maybe emit
-  const bool first_chunk = (sg.pos_start == 0);
-  float* S = pool_sum + static_cast<size_t>(sg.pool_slot) * d;
-  uint32_t* meta = pool_meta + static_cast<size_t>(sg.pool_slot) * 4;
-  const uint32_t old_count = first_chunk ? 0u : meta[0];
-  const uint32_t old_chunks = first_chunk ? 0u : meta[1];
-  const uint32_t new_count = old_count + static_cast<uint32_t>(sg.q_len);
-  const bool mean = (sg.pool_mode == HB_POOL_MEAN);
-  const bool emit = (sg.is_final != 0);
-  float4 e[MAX_VEC];
-  float nrm = 0.0f;
-#pragma unroll
-  for (int k = 0; k < MAX_VEC; ++k) {
-    const int v = threadIdx.x + k * NORM_THREADS;
-    e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (v < nv && (mean || emit)) {
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int b = 0; b < it.n_blocks; ++b) {
-        const float4 p = __ldcg(reinterpret_cast<const float4*>(part + static_cast<size_t>(it.part_base + b) * d + 4 * v));
-        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
-      }
-      float4 g;
-      bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
-      acc.x *= g.x; acc.y *= g.y; acc.z *= g.z; acc.w *= g.w;
-      if (mean) {
-        if (!first_chunk) {
-          const float4 o = *reinterpret_cast<const float4*>(S + 4 * v);
-          acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
-        }
-        *reinterpret_cast<float4*>(S + 4 * v) = acc;
-        const float inv = 1.0f / static_cast<float>(new_count);
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-      }
-      e[k] = acc;
-      nrm += acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
-    }
-  }
-  if (emit) {
-    const float tot = block_sum(nrm, red);
-    const float inv = 1.0f / fmaxf(sqrtf(tot), 1e-12f);
-    float* o = out_emb + static_cast<size_t>(sg.emb_row) * d;
-#pragma unroll
-    for (int k = 0; k < MAX_VEC; ++k) {
-      const int v = threadIdx.x + k * NORM_THREADS;
-      if (v < nv)
-        *reinterpret_cast<float4*>(o + 4 * v) = make_float4(e[k].x * inv, e[k].y * inv, e[k].z * inv, e[k].w * inv);
-    }
-  }
-  if (threadIdx.x == 0) {
-    meta[0] = new_count;
-    meta[1] = old_chunks + 1u;
-    meta[2] = static_cast<uint32_t>(sg.pool_mode);
-    meta[3] = emit ? 1u : 0u;
-    counters[it.seg] = 0u;  // ready for the next step
-  }
+  pool_block(it, sg, x, gain, part, counters, slot_sum, slot_meta, out_emb, d, eps, 1, status);
 }
 
 __global__ void __launch_bounds__(256)
@@ -402,6 +294,15 @@ int hb_launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s) 
   if (blocks < 1) blocks = 1;
   bf16_to_f16_kernel<<<static_cast<unsigned>(blocks), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(src),
                                                                    static_cast<__half*>(dst), n_vec, n);
+  return check_launch();
+}
+
+int hb_launch_pool_chunk(hb_ctx* c, const float* x, const void* gain, int n_rows, int mode, int first_chunk,
+                         int is_final, float* slot_sum, uint32_t* slot_meta, float* out_emb, cudaStream_t s) {
+  const int blocks = (mode == HB_POOL_MEAN) ? (n_rows + 31) / 32 : 1;
+  pool_chunk_kernel<<<blocks, NORM_THREADS, 0, s>>>(x, static_cast<const __nv_bfloat16*>(gain), n_rows, mode,
+                                                    first_chunk, is_final, c->pool_part, c->counters, slot_sum,
+                                                    slot_meta, out_emb, c->cfg.d_model, c->cfg.rms_eps, c->status);
   return check_launch();
 }
 

@@ -116,6 +116,8 @@ int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_ma
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
                     int n_slots, float* out_emb, cudaStream_t s);
 int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s);
+int hb_launch_pool_chunk(hb_ctx* c, const float* x, const void* gain, int n_rows, int mode, int first_chunk,
+                         int is_final, float* slot_sum, uint32_t* slot_meta, float* out_emb, cudaStream_t s);
 int hb_launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s);
 
 struct hb_ctx {

@@ -675,7 +675,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     ga.C = c->qkv; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rope_append(c, kg, l, s));
-    if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention_tc(c, kg, kv->map, l, s));
+    if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention_tc(c, kg, kv->map, l, s));
     if (dd.n_attn_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
@@ -729,6 +729,16 @@ int hb_weights_pack_f16(const void* src_bf16, void* dst_f16, size_t n_elems, voi
     if (a < b + n_elems * 2 && b < a + n_elems * 2) return HB_ERR_BAD_ARG;
   }
   return hb_launch_bf16_to_f16(src_bf16, dst_f16, n_elems, static_cast<cudaStream_t>(stream));
+}
+
+int hb_pool_chunk(hb_ctx* c, const float* x, const void* gain, int32_t n_rows, int32_t mode, int32_t first_chunk,
+                  int32_t is_final, float* slot_sum, uint32_t* slot_meta, float* out_emb, void* stream) {
+  if (!c || !x || !gain || !slot_sum || !slot_meta || n_rows < 1) return HB_ERR_BAD_ARG;
+  if (mode != HB_POOL_MEAN && mode != HB_POOL_LAST) return HB_ERR_BAD_ARG;
+  if (is_final && !out_emb) return HB_ERR_BAD_ARG;
+  if (n_rows > c->max_tokens) return HB_ERR_TOO_LARGE;
+  return hb_launch_pool_chunk(c, x, gain, n_rows, mode, first_chunk != 0, is_final != 0, slot_sum, slot_meta,
+                              out_emb, static_cast<cudaStream_t>(stream));
 }
 
 int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {

@@ -1,0 +1,150 @@
+// Device code of the incremental pooler (Section 3.3 of the paper, Eq. 1-2 and the last-token head)
+// and the small reduction helpers it shares with the other memory-bound kernels.  Included by the
+// translation units that launch it.
+#pragma once
+
+#include "hb_internal.h"
+
+namespace {
+
+constexpr int NORM_THREADS = 256;
+constexpr int MAX_VEC = 8;  // float4 per thread held in registers: d_model <= 256 * 4 * 8 = 8192
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over the block; every thread gets the result.  red must hold 32 floats.
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  v = warp_sum(v);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = (lane < (blockDim.x >> 5)) ? red[lane] : 0.0f;
+  t = warp_sum(t);
+  return t;
+}
+
+__device__ __forceinline__ void bf16x4_to_float4(uint2 raw, float4& o) {
+  const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+  const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+  o = make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+
+// Final RMSNorm fused with the incremental pooler.  One block per work item = a block of rows
+// of one embedding segment.  Phase 1: one warp per row, shuffle-reduced sum of squares.
+// Phase 2: each thread owns column vectors and adds x * rstd over the item's rows in row
+// order.  The block's partial sum goes to scratch; the block that arrives last for a segment
+// adds the partials in block order, applies the gain, and updates the slot:
+//   S <- S + partial, count <- count + q_len            (Eq. 1-2 with w = 1)
+// (a request's first chunk overwrites instead, i.e. S(0) = 0, W(0) = 0).  On the final chunk
+// it emits S / count (mean) or the normed last row (last-token head), L2-normalised.
+__device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg, const float* __restrict__ x,
+                                           const __nv_bfloat16* __restrict__ gain, float* __restrict__ part,
+                                           uint32_t* __restrict__ counters, float* __restrict__ pool_sum,
+                                           uint32_t* __restrict__ pool_meta, float* __restrict__ out_emb, int d,
+                                           float eps, int n_slots, uint32_t* status) {
+  __shared__ float red[32];
+  __shared__ float rstd_s[32];
+  __shared__ uint32_t is_last_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nv = d >> 2;
+  if (sg.pool_slot < 0 || sg.pool_slot >= n_slots) {
+    if (threadIdx.x == 0) atomicOr(status, HB_DEV_POOL_BAD_INDEX);
+    return;
+  }
+  // phase 1: row statistics (item rows <= 32)
+  for (int r = warp; r < it.n_rows; r += NORM_THREADS / 32) {
+    const float* xrow = x + static_cast<size_t>(it.row0 + r) * d;
+    float ss = 0.0f;
+    for (int v = lane; v < nv; v += 32) {
+      const float4 a = *reinterpret_cast<const float4*>(xrow + 4 * v);
+      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) rstd_s[r] = rsqrtf(ss / static_cast<float>(d) + eps);
+  }
+  __syncthreads();
+  // phase 2: column sums over the item's rows, fixed row order
+  float* my_part = part + static_cast<size_t>(it.part_base + it.block) * d;
+#pragma unroll 1
+  for (int v = threadIdx.x; v < nv; v += NORM_THREADS) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int r = 0; r < it.n_rows; ++r) {
+      const float4 a = *reinterpret_cast<const float4*>(x + static_cast<size_t>(it.row0 + r) * d + 4 * v);
+      const float s = rstd_s[r];
+      acc.x += a.x * s; acc.y += a.y * s; acc.z += a.z * s; acc.w += a.w * s;
+    }
+    *reinterpret_cast<float4*>(my_part + 4 * v) = acc;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t prev = atomicAdd(counters + it.seg, 1u);
+    is_last_s = (prev + 1u == static_cast<uint32_t>(it.n_blocks)) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!is_last_s) return;
+  __threadfence();
+  // segment tail: combine partials in block order, update the slot, maybe emit
+  const bool first_chunk = (sg.pos_start == 0);
+  float* S = pool_sum + static_cast<size_t>(sg.pool_slot) * d;
+  uint32_t* meta = pool_meta + static_cast<size_t>(sg.pool_slot) * 4;
+  const uint32_t old_count = first_chunk ? 0u : meta[0];
+  const uint32_t old_chunks = first_chunk ? 0u : meta[1];
+  const uint32_t new_count = old_count + static_cast<uint32_t>(sg.q_len);
+  const bool mean = (sg.pool_mode == HB_POOL_MEAN);
+  const bool emit = (sg.is_final != 0);
+  float4 e[MAX_VEC];
+  float nrm = 0.0f;
+#pragma unroll
+  for (int k = 0; k < MAX_VEC; ++k) {
+    const int v = threadIdx.x + k * NORM_THREADS;
+    e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (v < nv && (mean || emit)) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int b = 0; b < it.n_blocks; ++b) {
+        const float4 p = __ldcg(reinterpret_cast<const float4*>(part + static_cast<size_t>(it.part_base + b) * d + 4 * v));
+        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+      }
+      float4 g;
+      bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
+      acc.x *= g.x; acc.y *= g.y; acc.z *= g.z; acc.w *= g.w;
+      if (mean) {
+        if (!first_chunk) {
+          const float4 o = *reinterpret_cast<const float4*>(S + 4 * v);
+          acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+        }
+        *reinterpret_cast<float4*>(S + 4 * v) = acc;
+        const float inv = 1.0f / static_cast<float>(new_count);
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+      }
+      e[k] = acc;
+      nrm += acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
+    }
+  }
+  if (emit) {
+    const float tot = block_sum(nrm, red);
+    const float inv = 1.0f / fmaxf(sqrtf(tot), 1e-12f);
+    float* o = out_emb + static_cast<size_t>(sg.emb_row) * d;
+#pragma unroll
+    for (int k = 0; k < MAX_VEC; ++k) {
+      const int v = threadIdx.x + k * NORM_THREADS;
+      if (v < nv)
+        *reinterpret_cast<float4*>(o + 4 * v) = make_float4(e[k].x * inv, e[k].y * inv, e[k].z * inv, e[k].w * inv);
+    }
+  }
+  if (threadIdx.x == 0) {
+    meta[0] = new_count;
+    meta[1] = old_chunks + 1u;
+    meta[2] = static_cast<uint32_t>(sg.pool_mode);
+    meta[3] = emit ? 1u : 0u;
+    counters[it.seg] = 0u;  // ready for the next step
+  }
+}
+
+}  // namespace

@@ -38,6 +38,8 @@ SPECS = {
     # 7B-class shape: 64 decode rows, contexts U[512,4096]; embedding lengths lognormal(median 512,
     # sigma 1) clipped to [32,4096], chunk 512, last-token pooling, 4096-token budget
     "cfg3-7b": MixSpec("cfg3-7b", "7b", 64, 512, 4096, 4096, 512, "lognormal", 512, 32, 4096, B.POOL_LAST, 1003),
+    # small decode-heavy case for profiler captures (use with --layers and --decode-alias)
+    "dec-7b": MixSpec("dec-7b", "7b", 256, 2048, 2048, 512, 256, "uniform", 128, 128, 1024, B.POOL_MEAN, 1010),
 }
 
 
@@ -66,9 +68,9 @@ class MixedWorkload:
     (read-only sharing; every row still appends to a private tail page).
     """
 
-    def __init__(self, spec, kv, pool, max_pos, decode_alias=0):
+    def __init__(self, spec, kv, pool, max_pos, decode_alias=0, shape=None):
         self.spec = spec
-        self.shape = synth.SHAPES[spec.shape]
+        self.shape = shape if shape is not None else synth.SHAPES[spec.shape]
         self.kv, self.pool = kv, pool
         self.P = self.shape.page_size
         self.max_pos = max_pos
