@@ -282,6 +282,43 @@ HB_API int hb_pool_chunk(hb_ctx* ctx, const float* x, const void* gain, int32_t 
                          int32_t first_chunk, int32_t is_final, float* slot_sum, uint32_t* slot_meta,
                          float* out_emb, void* stream);
 
+/* ---- entry point that allocates nothing ------------------------------------ */
+
+/* Largest chunk and hidden size hb_pool_chunk_noalloc accepts. */
+#define HB_NOALLOC_MAX_ROWS 2048
+#define HB_NOALLOC_MAX_DMODEL 4096
+
+/* (The paper has no counterpart to this call; it exists for deployment.)
+ * hb_pool_chunk without a context and without any allocation: same arguments
+ * and results as hb_pool_chunk, with d_model and rms_eps passed directly.
+ *
+ * Who needs it: a caller that cannot allocate device memory -- for example a
+ * serving process whose own allocator claimed the whole device at start-up, or
+ * code running where a device allocation would fail or stall the GPU -- cannot
+ * create an hb_ctx (that allocates the workspace) and so cannot reach any other
+ * compute call.  Here the pooler's scratch (partial sums of 32-row blocks, an
+ * arrival counter, a status word) lives in a fixed array inside the library
+ * image instead: 1 MiB + 256 bytes on every GPU that loads the library, held
+ * until the process exits.  The call itself uses no cudaMalloc, cudaFree or
+ * any other allocating routine.
+ *
+ * Limits and rules
+ *  - n_rows <= HB_NOALLOC_MAX_ROWS and d_model <= HB_NOALLOC_MAX_DMODEL
+ *    (d_model a multiple of 4); anything larger returns HB_ERR_TOO_LARGE and
+ *    does nothing;
+ *  - the first call on a device looks up the array's device address (once per
+ *    device, with that device current); make that first call before starting
+ *    any stream capture;
+ *  - all calls on a device share the one array, which keeps the previous
+ *    call's contents (the call clears the words that must start at zero).
+ *    Two calls whose kernels can run at the same time on that device -- from
+ *    different streams or threads -- race on it: serialise them;
+ *  - the caller still owns and passes every input and output (x, gain,
+ *    slot_sum, slot_meta, out_emb: device pointers as in hb_pool_chunk). */
+HB_API int hb_pool_chunk_noalloc(const float* x, const void* gain, int32_t n_rows, int32_t d_model,
+                                 float rms_eps, int32_t mode, int32_t first_chunk, int32_t is_final,
+                                 float* slot_sum, uint32_t* slot_meta, float* out_emb, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -85,6 +85,8 @@ _sig = {
     "hb_weights_pack_f16": [_P, _P, C.c_size_t, _P],
     "hb_argmax": [_P, _P, C.c_int32, _P, _P],
     "hb_pool_chunk": [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P],
+    "hb_pool_chunk_noalloc": [_P, _P, C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P,
+                              _P],
     "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
     "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
     "hb_profile_enable": [_P, C.c_int],
@@ -378,6 +380,22 @@ class Context:
             self.close()
         except Exception:
             pass
+
+
+NOALLOC_MAX_ROWS, NOALLOC_MAX_DMODEL = 2048, 4096
+
+
+def pool_chunk_noalloc(x, gain, n_rows, d_model, rms_eps, mode, first_chunk, is_final, slot_sum, slot_meta,
+                       out_emb, stream=None):
+    """hb_pool_chunk_noalloc: the pooler for callers that may not allocate device memory (no
+    context; scratch is a fixed array inside the library).  Returns the status code; sizes beyond
+    NOALLOC_MAX_ROWS x NOALLOC_MAX_DMODEL give HB_ERR_TOO_LARGE (-5).  Calls that may overlap on
+    the GPU must be serialised by the caller."""
+    return lib.hb_pool_chunk_noalloc(C.c_void_p(x.data_ptr()), C.c_void_p(gain.data_ptr()), n_rows, d_model,
+                                     float(rms_eps), mode, 1 if first_chunk else 0, 1 if is_final else 0,
+                                     C.c_void_p(slot_sum.data_ptr()), C.c_void_p(slot_meta.data_ptr()),
+                                     C.c_void_p(out_emb.data_ptr()) if out_emb is not None else None,
+                                     _stream_ptr(stream))
 
 
 def validate_desc(cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, batch):
