@@ -80,7 +80,11 @@ typedef struct {
  * once with hb_weights_pack_f16 (the tensor cores take one 16-bit format for
  * both operands, and activations are fp16).  Gains and the token embedding
  * stay bf16.
- *   wqkv      fp16 [(n_heads + 2 n_kv_heads) * head_dim, d_model]: q rows, then k, then v
+ *   wqkv      fp16 [(n_heads + 2 n_kv_heads) * head_dim, d_model]: q rows, then k, then v;
+ *             inside every q and k head the rows are pair-interleaved for the rotary
+ *             step: row 2i = the head's row i, row 2i+1 = its row i + head_dim/2
+ *             (a fixed permutation of the head dimension, applied alike to q and k,
+ *             so q.k is unchanged; the KV cache holds k in this order)
  *   wo        fp16 [d_model, n_heads * head_dim]
  *   w_gate_up fp16 [2 * d_ffn, d_model]: row 2j = gate row j, row 2j+1 = up row j
  *   w_down    fp16 [d_model, d_ffn]

@@ -123,6 +123,24 @@ def bf16_from_f32(a, device="cuda"):
     return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
 
 
+def rope_pair_order(Dh):
+    """Stored position j of a q/k head holds rotary element rope_pair_order(Dh)[j]:
+    (0, Dh/2, 1, Dh/2 + 1, ...)."""
+    half = Dh // 2
+    order = np.empty(Dh, dtype=np.int64)
+    order[0::2] = np.arange(half)
+    order[1::2] = np.arange(half) + half
+    return order
+
+
+def rope_interleave_rows(w, Dh):
+    """Reorder the rows of a q or k projection [H*Dh, d] into the library's pair-interleaved
+    head layout (a layout change only: input marshalling)."""
+    H = w.shape[0] // Dh
+    idx = (np.arange(H)[:, None] * Dh + rope_pair_order(Dh)[None, :]).ravel()
+    return w[idx]
+
+
 def pack_f16_(t, stream=None):
     """Repack a bf16 tensor to fp16 in place (library kernel); returns the fp16 view."""
     assert t.dtype == torch.bfloat16 and t.is_contiguous()
@@ -160,7 +178,8 @@ class DeviceWeights:
             lw = self.layers[l]
             lw.attn_norm = up(w["attn_norm"])
             lw.ffn_norm = up(w["ffn_norm"])
-            lw.wqkv = upw(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0))
+            lw.wqkv = upw(np.concatenate([rope_interleave_rows(w["wq"], s.Dh), rope_interleave_rows(w["wk"], s.Dh),
+                                          w["wv"]], axis=0))
             lw.wo = upw(w["wo"])
             gu = np.empty((2 * s.F, s.d), dtype=np.float32)
             gu[0::2] = w["wg"]

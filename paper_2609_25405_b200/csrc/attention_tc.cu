@@ -237,21 +237,37 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
+      // page ids of tile j + 1 are requested while tile j is being issued (global-load latency off the path)
+      auto load_ids = [&](int j, int (&ids)[BN / 16]) {
+        const int kb = j * BN;
+#pragma unroll
+        for (int pi = 0; pi < BN / 16; ++pi)
+          ids[pi] = (kb + pi * 16 < it.key1) ? __ldg(p.pages + sg.pt_start + kb / 16 + pi) : 0;
+      };
+      int nxt[BN / 16];
+      load_ids(0, nxt);
       for (int j = 0; j < n_tiles; ++j) {
         const int st = j % C::STAGES;
+        int cur[BN / 16];
+#pragma unroll
+        for (int pi = 0; pi < BN / 16; ++pi) cur[pi] = nxt[pi];
+        if (j + 1 < n_tiles) load_ids(j + 1, nxt);
         if (!mbar_wait(kv_empty(st), static_cast<uint32_t>(((j / C::STAGES) & 1) ^ 1), abort_flag)) break;
         const int kb = j * BN;
         const int n_pg = min(BN / 16, (it.key1 - kb + 15) / 16);
         const uint32_t k_dst = ring_s + st * 2 * C::KV_HALF;
         mbar_arrive_expect_tx(kv_full(st), static_cast<uint32_t>(n_pg) * 2u * C::SUB * (16 * 128));
-        for (int pi = 0; pi < n_pg; ++pi) {
-          const int64_t page = __ldg(p.pages + sg.pt_start + kb / 16 + pi);
-          const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.n_pages + page) * 2) * p.Hkv + hk) * 16);
-          const int row_v = row_k + p.Hkv * 16;
 #pragma unroll
-          for (int h = 0; h < C::SUB; ++h) {
-            tma_load_2d(k_dst + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_k);
-            tma_load_2d(k_dst + C::KV_HALF + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_v);
+        for (int pi = 0; pi < BN / 16; ++pi) {
+          if (pi < n_pg) {
+            const int64_t page = cur[pi];
+            const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.n_pages + page) * 2) * p.Hkv + hk) * 16);
+            const int row_v = row_k + p.Hkv * 16;
+#pragma unroll
+            for (int h = 0; h < C::SUB; ++h) {
+              tma_load_2d(k_dst + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_k);
+              tma_load_2d(k_dst + C::KV_HALF + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_v);
+            }
           }
         }
       }

@@ -1,5 +1,4 @@
-// Memory-bound stages of the mixed step: token gather + RMSNorm, RMSNorm, rotary + KV-page
-// append, final RMSNorm fused with the incremental pooler (Section 3.3, Eq. 1-2 and the
+// Memory-bound stages of the mixed step: token gather + RMSNorm, RMSNorm, final RMSNorm fused with the incremental pooler (Section 3.3, Eq. 1-2 and the
 // last-token head) and with the hi/lo split that feeds the LM head, greedy argmax.
 // All global accesses are 16-byte vectors; row statistics use warp shuffles; sums run in a
 // fixed order (no floating-point atomics), so results do not depend on what else is batched.
@@ -65,60 +64,6 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
       float4 o = make_float4(buf[i].x * rstd * g.x, buf[i].y * rstd * g.y, buf[i].z * rstd * g.z,
                              buf[i].w * rstd * g.w);
       *reinterpret_cast<uint2*>(hrow + 4 * v) = float4_to_f16x4(o);
-    }
-  }
-}
-
-// Rotary embedding of q and k (rotate-half pairing: element i pairs with i + Dh/2, angle
-// pos * theta^(-2i/Dh) from a host-built table) and append of k, v to the request's KV page:
-// position pos lives in page pages[pt_start + pos / P], slot pos % P.
-__global__ void __launch_bounds__(256)
-rope_append_kernel(const float* __restrict__ qkv, __half* __restrict__ q_out, KvGeom kv, int layer,
-                   const int32_t* __restrict__ row_seg, const int32_t* __restrict__ row_pos,
-                   const hb_seg* __restrict__ segs, const int32_t* __restrict__ pages,
-                   const float* __restrict__ rope_cos, const float* __restrict__ rope_sin, int Hq, int max_pos,
-                   uint32_t* status) {
-  const int t = blockIdx.x;
-  const int Dh = kv.Dh, Hkv = kv.Hkv, half = Dh >> 1;
-  const int pos = row_pos[t];
-  const hb_seg sg = segs[row_seg[t]];
-  const int blk = pos / kv.P, slot = pos - blk * kv.P;
-  int page = (blk < sg.pt_len) ? pages[sg.pt_start + blk] : -1;
-  if (page < 0 || page >= kv.n_pages || pos >= max_pos) {
-    if (threadIdx.x == 0) atomicOr(status, HB_DEV_APPEND_BAD_INDEX);
-    return;  // skip the access
-  }
-  const int n_qkv = (Hq + 2 * Hkv) * Dh;
-  const float* row = qkv + static_cast<size_t>(t) * n_qkv;
-  __half* kbase = kv.arena + layer * kv.layer_stride + page * kv.page_stride + slot * Dh;
-  const int64_t head_stride = static_cast<int64_t>(kv.P) * Dh;
-  const float* cs = rope_cos + static_cast<size_t>(pos) * half;
-  const float* sn = rope_sin + static_cast<size_t>(pos) * half;
-  const int units_per_head = half >> 2;                 // 4 pairs per unit
-  const int rot_units = (Hq + Hkv) * units_per_head;
-  const int v_units = Hkv * (Dh >> 2);                  // 4 elements per unit
-  for (int u = threadIdx.x; u < rot_units + v_units; u += blockDim.x) {
-    if (u < rot_units) {
-      const int head = u / units_per_head, i = (u - head * units_per_head) << 2;
-      const float* src = row + head * Dh + i;
-      const float4 a = *reinterpret_cast<const float4*>(src);
-      const float4 b = *reinterpret_cast<const float4*>(src + half);
-      const float4 c = *reinterpret_cast<const float4*>(cs + i);
-      const float4 s = *reinterpret_cast<const float4*>(sn + i);
-      const float4 lo = make_float4(a.x * c.x - b.x * s.x, a.y * c.y - b.y * s.y, a.z * c.z - b.z * s.z,
-                                    a.w * c.w - b.w * s.w);
-      const float4 hi = make_float4(b.x * c.x + a.x * s.x, b.y * c.y + a.y * s.y, b.z * c.z + a.z * s.z,
-                                    b.w * c.w + a.w * s.w);
-      __half* dst = (head < Hq) ? q_out + static_cast<size_t>(t) * Hq * Dh + head * Dh + i
-                                       : kbase + (head - Hq) * head_stride + i;
-      *reinterpret_cast<uint2*>(dst) = float4_to_f16x4(lo);
-      *reinterpret_cast<uint2*>(dst + half) = float4_to_f16x4(hi);
-    } else {
-      const int w = u - rot_units;
-      const int head = w / (Dh >> 2), i = (w - head * (Dh >> 2)) << 2;
-      const float4 a = *reinterpret_cast<const float4*>(row + (Hq + Hkv + head) * Dh + i);
-      __half* dst = kbase + (Hkv + head) * head_stride + i;
-      *reinterpret_cast<uint2*>(dst) = float4_to_f16x4(a);
     }
   }
 }
@@ -259,13 +204,6 @@ int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaS
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s) {
   norm_kernel<false><<<c->dd.T, NORM_THREADS, 0, s>>>(nullptr, nullptr, static_cast<const __nv_bfloat16*>(gain), c->x,
                                                       c->h, c->cfg.d_model, c->cfg.rms_eps);
-  return check_launch();
-}
-
-int hb_launch_rope_append(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s) {
-  rope_append_kernel<<<c->dd.T, 256, 0, s>>>(c->qkv, c->q, kv, layer, c->dd.row_seg, c->dd.row_pos, c->dd.segs,
-                                             c->dd.pages, c->rope_cos, c->rope_sin, c->cfg.n_heads, c->cfg.max_pos,
-                                             c->status);
   return check_launch();
 }
 

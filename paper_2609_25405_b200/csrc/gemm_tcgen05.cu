@@ -38,7 +38,7 @@ struct Tile {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = B_ROWS * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TMEM_COLS = 2 * BN;  // two accumulators; 256 or 512 (powers of two)
+  static constexpr int TMEM_COLS = (2 * BN <= 256) ? 256 : 512;  // two accumulators, rounded to a power of two
   static constexpr int BAR_BYTES = 256;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
@@ -273,6 +273,46 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
   }
 }
 
+// QKV epilogue: one thread holds 32 consecutive output columns of one token row.  The q and k rows
+// of the weight are pair-interleaved inside each head (column 2i = rotary element i, column 2i+1 =
+// element i + Dh/2), so every rotation pair sits in adjacent columns.  q goes to the query buffer,
+// k and v to slot pos % P of the row's page; all as fp16.
+__device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32],
+                                                  int pos, int page) {
+  const int Dh = g.Dh;
+  const int head = col0 / Dh, off = col0 - head * Dh;
+  uint32_t pk[16];
+  __half* dst;
+  if (head < g.Hq + g.Hkv) {
+    const float4* cs = reinterpret_cast<const float4*>(g.rope_cos + static_cast<size_t>(pos) * (Dh >> 1) + (off >> 1));
+    const float4* sn = reinterpret_cast<const float4*>(g.rope_sin + static_cast<size_t>(pos) * (Dh >> 1) + (off >> 1));
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const float4 c = __ldg(cs + v), s = __ldg(sn + v);
+      const float cc[4] = {c.x, c.y, c.z, c.w}, ss[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float a = __uint_as_float(r[v * 8 + e * 2]), b = __uint_as_float(r[v * 8 + e * 2 + 1]);
+        pk[v * 4 + e] = pack_f16(a * cc[e] - b * ss[e], b * cc[e] + a * ss[e]);
+      }
+    }
+    if (head < g.Hq) {
+      dst = g.q_out + static_cast<size_t>(row) * g.Hq * Dh + col0;
+    } else {
+      dst = g.kv_layer + static_cast<int64_t>(page) * g.page_stride +
+            static_cast<int64_t>(head - g.Hq) * g.P * Dh + (pos % g.P) * Dh + off;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) pk[j] = pack_f16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+    dst = g.kv_layer + static_cast<int64_t>(page) * g.page_stride +
+          static_cast<int64_t>(head - g.Hq) * g.P * Dh + (pos % g.P) * Dh + off;   // V blocks follow the K blocks
+  }
+#pragma unroll
+  for (int v = 0; v < 4; ++v)
+    *reinterpret_cast<uint4*>(dst + v * 8) = make_uint4(pk[v * 4], pk[v * 4 + 1], pk[v * 4 + 2], pk[v * 4 + 3]);
+}
+
 template <int BN, int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -425,11 +465,26 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       tcgen05_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
+      int pos = 0, page = 0;
+      bool row_ok = row < g.M;
+      if constexpr (EPI == HB_EPI_QKV_ROPE) {
+        if (row_ok) {
+          pos = g.row_pos[row];
+          page = g.row_page[row];
+          if (page < 0 || page >= g.n_pages) {   // never write through a bad page id
+            atomicOr(g.status, HB_DEV_APPEND_BAD_INDEX);
+            row_ok = false;
+          }
+        }
+      }
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         uint32_t r[32];
         tmem_ld32(t_row + static_cast<uint32_t>(c), r);
-        if (row < g.M && n0 + c < g.N) epilogue_store<EPI>(g, row, n0 + c, r);
+        if (row_ok && n0 + c < g.N) {
+          if constexpr (EPI == HB_EPI_QKV_ROPE) epilogue_qkv_rope(g, row, n0 + c, r, pos, page);
+          else epilogue_store<EPI>(g, row, n0 + c, r);
+        }
       }
       tcgen05_fence_before();
       __syncwarp();
@@ -515,6 +570,7 @@ int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, int epi, const Gem
     case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, a, num_sms, s);
     case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, a, num_sms, s);
     case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_QKV_ROPE: return launch_one<BN, HB_EPI_QKV_ROPE, CG>(tmA, tmB, a, num_sms, s);
     default: return HB_ERR_BAD_ARG;
   }
 }
@@ -538,7 +594,10 @@ int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t 
 // Tile width: 256 columns halves the shared-memory traffic per flop; 128 gives more tiles
 // when the problem has too few to fill the SMs or the last wave would be mostly idle.
 int hb_gemm_pick_bn(int M, int N, int num_sms) {
-  // enough rows and columns for 256 x 256 pair tiles to fill the machine: use CTA pairs
+  // enough rows and columns for 256 x 256 pair tiles to fill the machine: use CTA pairs.  (A 256 x 192
+  // pair tile would shorten the last, partly filled wave of the N = 4096 and 6144 projections, but it
+  // measured 10-19 % slower on every 7B shape: the kernel is bound by bytes loaded per MMA cycle,
+  // which the narrower tile raises.)
   if (M > 128 && static_cast<long>((M + 255) / 256) * ((N + 255) / 256) >= num_sms / 2) return HB_GEMM_PAIR256;
   const int m_tiles = (M + BM - 1) / BM;
   const long t256 = static_cast<long>(m_tiles) * ((N + 255) / 256);

@@ -51,6 +51,7 @@ struct DeviceDesc {
   const int32_t* tok;       // [T]
   const int32_t* row_seg;   // [T]
   const int32_t* row_pos;   // [T]
+  const int32_t* row_page;  // [T] page holding the row's own position
   const hb_seg* segs;       // [R]
   const int32_t* pages;     // [n_page_ids]
   const int32_t* logit_src; // [n_logit_rows] token row feeding logits row i
@@ -88,12 +89,25 @@ struct hb_pool {
 };
 
 // ---- GEMM -------------------------------------------------------------------
+// Internal epilogue of the QKV projection: rotary embedding and KV-page append fused into the
+// accumulator read-out (not reachable through hb_gemm).
+constexpr int HB_EPI_QKV_ROPE = 4;
+
 struct GemmArgs {
   void* C;
   int32_t M, N, K;      // K = columns of A; B has K >> b_kshift columns
   int32_t ldc;          // elements
   int32_t b_kshift;     // B k-block index = A k-block index >> b_kshift
   uint32_t* status;
+  // HB_EPI_QKV_ROPE only
+  const int32_t* row_pos;   // [M] position of each row inside its request
+  const int32_t* row_page;  // [M] physical page that holds that position
+  const float* rope_cos;    // [max_pos, Dh/2]
+  const float* rope_sin;
+  __half* q_out;            // [M, Hq*Dh]
+  __half* kv_layer;         // this layer's slice of the KV arena
+  int64_t page_stride;      // elements per page: 2 * Hkv * P * Dh
+  int32_t Hq, Hkv, Dh, P, n_pages;
 };
 
 int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
@@ -110,7 +124,6 @@ int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int e
 struct hb_ctx;
 int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s);
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
-int hb_launch_rope_append(hb_ctx* c, const KvGeom& kv, int layer, cudaStream_t s);
 int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
 int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
@@ -131,7 +144,7 @@ struct hb_ctx {
   // workspace carve-up (device)
   float* x;                 // [max_tokens, d] residual stream, fp32
   __half* h;                // [max_tokens, d] normed activations (fp16)
-  float* qkv;               // [max_tokens, n_qkv] projection output, fp32
+  float* qkv;               // unused placeholder (the QKV epilogue writes q and the KV pages directly)
   __half* q;                // [max_tokens, Hq*Dh] rotated queries (fp16)
   __half* attn_out;         // [max_tokens, Hq*Dh] (fp16)
   __half* act;              // [max_tokens, F] (fp16)

@@ -61,7 +61,8 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.logit_rows_pad = static_cast<int32_t>(lrows);
   L.x = cv.take(rows * c.d_model * 4);
   L.h = cv.take(rows * c.d_model * 2);
-  L.qkv = cv.take(rows * n_qkv * 4);
+  L.qkv = cv.take(256);   // the QKV projection no longer has an intermediate: its epilogue writes q and the pages
+  (void)n_qkv;
   L.q = cv.take(rows * n_q * 2);
   L.attn_out = cv.take(rows * n_q * 2);
   L.act = cv.take(rows * c.d_ffn * 2);
@@ -81,7 +82,7 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.attn_counters = cv.take(static_cast<size_t>(max_segs) * c.n_kv_heads * 4);
   L.status = cv.take(256);
   size_t dc = 0;
-  dc += align_up(static_cast<size_t>(max_tokens) * 4, 16) * 3;          // tok, row_seg, row_pos
+  dc += align_up(static_cast<size_t>(max_tokens) * 4, 16) * 4;          // tok, row_seg, row_pos, row_page
   dc += align_up(static_cast<size_t>(max_segs) * sizeof(hb_seg), 16);
   dc += align_up(static_cast<size_t>(max_page_ids) * 4, 16);
   dc += align_up(static_cast<size_t>(max_segs) * 4, 16);                // logit_src
@@ -485,12 +486,14 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     return o;
   };
   const size_t o_tok = place(static_cast<size_t>(T) * 4), o_rseg = place(static_cast<size_t>(T) * 4),
-               o_rpos = place(static_cast<size_t>(T) * 4), o_segs = place(static_cast<size_t>(R) * sizeof(hb_seg)),
+               o_rpos = place(static_cast<size_t>(T) * 4), o_rpage = place(static_cast<size_t>(T) * 4),
+               o_segs = place(static_cast<size_t>(R) * sizeof(hb_seg)),
                o_pages = place(static_cast<size_t>(d->n_page_ids) * 4),
                o_lsrc = place(static_cast<size_t>(d->n_logit_rows) * 4);
   int32_t* tok = reinterpret_cast<int32_t*>(st.host + o_tok);
   int32_t* rseg = reinterpret_cast<int32_t*>(st.host + o_rseg);
   int32_t* rpos = reinterpret_cast<int32_t*>(st.host + o_rpos);
+  int32_t* rpage = reinterpret_cast<int32_t*>(st.host + o_rpage);
   hb_seg* segs = reinterpret_cast<hb_seg*>(st.host + o_segs);
   int32_t* pages = reinterpret_cast<int32_t*>(st.host + o_pages);
   int32_t* lsrc = reinterpret_cast<int32_t*>(st.host + o_lsrc);
@@ -504,6 +507,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     for (int32_t j = 0; j < sg.q_len; ++j) {
       rseg[sg.q_start + j] = r;
       rpos[sg.q_start + j] = sg.pos_start + j;
+      rpage[sg.q_start + j] = d->page_ids[sg.pt_start + (sg.pos_start + j) / cfg.page_size];
     }
     if (sg.logits_row >= 0) lsrc[sg.logits_row] = sg.q_start + sg.q_len - 1;
     if (sg.kind == HB_KIND_EMBED_CHUNK) {
@@ -599,6 +603,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
   dd.tok = reinterpret_cast<const int32_t*>(c->desc_dev + o_tok);
   dd.row_seg = reinterpret_cast<const int32_t*>(c->desc_dev + o_rseg);
   dd.row_pos = reinterpret_cast<const int32_t*>(c->desc_dev + o_rpos);
+  dd.row_page = reinterpret_cast<const int32_t*>(c->desc_dev + o_rpage);
   dd.segs = reinterpret_cast<const hb_seg*>(c->desc_dev + o_segs);
   dd.pages = reinterpret_cast<const int32_t*>(c->desc_dev + o_pages);
   dd.logit_src = reinterpret_cast<const int32_t*>(c->desc_dev + o_lsrc);
@@ -667,14 +672,17 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     }
     if (l == 0) HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
     else HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.attn_norm, s));
-    GemmArgs ga;
+    GemmArgs ga = {};
     ga.status = c->status;
     ga.b_kshift = 0;
     ga.M = T;
-    // QKV projection (fp32 out, rotated and appended next)
-    ga.C = c->qkv; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_F32, ga, c->num_sms, s));
-    HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rope_append(c, kg, l, s));
+    // QKV projection; its epilogue rotates q, k and appends k, v to the pages
+    ga.C = nullptr; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
+    ga.row_pos = dd.row_pos; ga.row_page = dd.row_page; ga.rope_cos = c->rope_cos; ga.rope_sin = c->rope_sin;
+    ga.q_out = c->q; ga.kv_layer = kg.arena + static_cast<int64_t>(l) * kg.layer_stride;
+    ga.page_stride = kg.page_stride; ga.Hq = cfg.n_heads; ga.Hkv = cfg.n_kv_heads; ga.Dh = cfg.head_dim;
+    ga.P = cfg.page_size; ga.n_pages = kg.n_pages;
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s));
     if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention_tc(c, kg, kv->map, l, s));
     if (dd.n_attn_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
     // O projection, added to the residual stream
@@ -704,7 +712,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
       if ((rc = hb_tmap_2d_bf16(&c->tm_lm, w->lm_head, cfg.vocab, cfg.d_model, 128)) != HB_OK) return rc;
       c->lm_key = w->lm_head;
     }
-    GemmArgs ga;
+    GemmArgs ga = {};
     ga.status = c->status;
     ga.b_kshift = 1;  // A holds (hi, lo) 64-column blocks: each weight k-block is used twice
     ga.M = dd.n_logit; ga.N = cfg.vocab; ga.K = 2 * cfg.d_model; ga.ldc = cfg.vocab; ga.C = out_logits;
@@ -799,7 +807,7 @@ int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t
   if (rc != HB_OK) return rc;
   rc = hb_tmap_2d_bf16(&tb, B, N, K, hb_gemm_box_rows(bn));
   if (rc != HB_OK) return rc;
-  GemmArgs ga;
+  GemmArgs ga = {};
   ga.C = C; ga.M = M; ga.N = N; ga.K = K; ga.b_kshift = 0; ga.status = c->status;
   ga.ldc = (epilogue == HB_EPI_SWIGLU) ? N / 2 : N;
   return hb_gemm_launch(ta, tb, bn, epilogue, ga, c->num_sms, static_cast<cudaStream_t>(stream));

@@ -30,7 +30,7 @@ def _f16_exact(rng, shape, std):
 # (M, N, K): several tiles, ragged M tail, N not a multiple of the tile, K not a multiple of 64,
 # a single row, more tiles than SMs (persistent loop + both TMEM accumulators), long K (ring wraps)
 SHAPES = [(128, 256, 64), (68, 768, 256), (300, 328, 200), (1, 1024, 256), (4, 1024, 512),
-          (515, 2048, 1024), (2500, 3072, 256), (256, 256, 4096), (4096, 1536, 512)]
+          (515, 2048, 1024), (2500, 3072, 256), (256, 256, 4096), (4096, 1536, 512), (1030, 4160, 128), (2100, 4608, 192)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)

@@ -93,6 +93,7 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
     for j in (0, 1):
         _check_emb(ge[j].astype(np.float64), re_[j])
     # ---- KV bookkeeping: exactly the expected slots were written, everything else is the sentinel
+    from paper_2609_25405_b200 import binding as B
     W = weights[0]
     kvv = eng.kv.view().cpu()                                   # [L, page, 2, Hkv, P, Dh] fp16
     raw = eng.kv.arena.cpu().view(TINY.L, eng.kv.n_pages, 2, TINY.Hkv, 16, TINY.Dh)
@@ -107,7 +108,9 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
         for l in range(TINY.L):
             pages = torch.tensor([M.kv_slot(req.pages, p, 16)[0] for p in range(n)])
             slots = torch.tensor([M.kv_slot(req.pages, p, 16)[1] for p in range(n)])
-            k_gpu = kvv[l, :, 0][pages, :, slots, :].float().numpy()   # [n, Hkv, Dh]
+            k_st = kvv[l, :, 0][pages, :, slots, :].float().numpy()    # [n, Hkv, Dh], pair-interleaved
+            k_gpu = np.empty_like(k_st)
+            k_gpu[..., B.rope_pair_order(TINY.Dh)] = k_st               # back to the rotary element order
             v_gpu = kvv[l, :, 1][pages, :, slots, :].float().numpy()
             assert np.max(np.abs(k_gpu - kv_ref[l][0])) < 5e-3
             assert np.max(np.abs(v_gpu - kv_ref[l][1])) < 5e-3
