@@ -201,7 +201,7 @@ def main():
 
     import torch
     from paper_2609_25405_b200 import binding as B
-    from paper_2609_25405_b200 import synth, workloads
+    from paper_2609_25405_b200 import replicas, synth, workloads
     from paper_2609_25405_b200.engine import build_batch
 
     rank = int(os.environ.get("RANK", "0"))
@@ -215,7 +215,7 @@ def main():
 
     spec = get_spec(args.workload)
     if world > 1:   # independent replicas: each rank draws its own batch stream
-        spec = workloads.MixSpec(**{**spec.__dict__, "seed": spec.seed + 7919 * rank})
+        spec = workloads.MixSpec(**{**spec.__dict__, "seed": replicas.rank_seed(spec.seed, rank)})
     shape = synth.SHAPES[spec.shape]
     if args.layers:
         shape = shape.with_layers(args.layers)
@@ -314,13 +314,7 @@ def main():
     status = ctx.status_poll()
 
     tokens = sum(work[i]["T"] for i in timed)
-    t_all = torch.tensor([ms, e2e_s * 1e3, float(tokens)], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        mx = t_all.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = t_all.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        ms, e2e_ms, tokens = float(mx[0]), float(mx[1]), float(sm[2])
-    else:
-        e2e_ms = e2e_s * 1e3
+    ms, e2e_ms, tokens = replicas.aggregate(dist, "cuda", ms, e2e_s * 1e3, tokens)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

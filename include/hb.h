@@ -158,8 +158,10 @@ HB_API int hb_destroy(hb_ctx* ctx);
 /* ---- paged KV cache ------------------------------------------------------- */
 
 /* Bytes of an arena of n_pages.  Arena layout (fp16; post-rotary K and V):
- * [layer][page][K|V][kv_head][slot 0..page_size)[head_dim], so the K (or V)
- * rows of one (layer, page, head) are contiguous.  Host only. */
+ * [layer][page][kv_head][K|V][head_dim/64][slot 0..page_size)[64], i.e. the
+ * head dimension is split into 64-element halves and the K+V block of one
+ * (layer, page, head) is contiguous (4-8 KiB): one TMA copy fetches it.
+ * Host only. */
 HB_API int hb_kv_arena_bytes(const hb_model_cfg* cfg, int32_t n_pages, size_t* out_bytes);
 
 /* Wrap a caller-owned device arena.  Only the free list lives in the library

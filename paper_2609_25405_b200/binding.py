@@ -236,10 +236,17 @@ class KvCache:
                                C.byref(self.handle)), "hb_kv_create")
 
     def view(self):
-        """fp16 view [L, page, 2, Hkv, P, Dh]."""
+        """fp16 view [L, page, Hkv, 2 (K|V), Dh/64, P, 64] (the arena's own layout)."""
         c = self.cfg
-        return self.arena.view(torch.float16).view(c.n_layers, self.n_pages, 2, c.n_kv_heads,
-                                                   c.page_size, c.head_dim)
+        return self.arena.view(torch.float16).view(c.n_layers, self.n_pages, c.n_kv_heads, 2, c.head_dim // 64,
+                                                   c.page_size, 64)
+
+    def rows(self, layer, pages, slots, is_v):
+        """K (is_v = 0) or V (1) rows of `layer` at (pages[i], slots[i]) as [n, Hkv, Dh] fp16, in the
+        stored head-dimension order."""
+        v = self.view()[layer][:, :, is_v]                      # [page, Hkv, H2, P, 64]
+        r = v[pages, :, :, slots, :]                            # [n, Hkv, H2, 64]
+        return r.reshape(r.shape[0], r.shape[1], -1)
 
     def alloc(self, n):
         ids = (C.c_int32 * max(n, 1))()

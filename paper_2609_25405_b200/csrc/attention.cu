@@ -12,9 +12,10 @@
 //                their partial (max, sum, output) are merged in shared memory, and the splits
 //                of a row through a scratch record per split, merged in split order by the CTA
 //                that arrives last (integer arrival counter; no floating-point atomics).
-// K/V tiles of 64 keys (4 pages) are gathered by TMA: one thread issues a 2-D tensor copy per
-// (page, 64-column half) into a 128-byte-swizzled shared-memory ring and the CTA waits on the
-// stage's mbarrier (bounded).  S = Q K^T and O += P V run on mma.sync m16n8k16 (fp16 in, fp32
+// K/V tiles of 64 keys (4 pages) are gathered by TMA: one thread issues one 2-D tensor copy per page
+// (the contiguous K+V block of this KV head, 4-8 KiB: the TMA unit's rate is per copy, so few large
+// copies) into a 128-byte-swizzled shared-memory ring and the CTA waits on the stage's mbarrier
+// (bounded).  S = Q K^T and O += P V run on mma.sync m16n8k16 (fp16 in, fp32
 // accumulate), softmax in fp32 with exp2.  Split decisions depend on the request's own length only, so a
 // request's result does not depend on its batch mates.
 #include "hb_internal.h"
@@ -120,11 +121,19 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
   return static_cast<uint32_t>((c >> 3) * (64 * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
+// Byte offset of 16-byte chunk `c` of key `r` of a 64-key K/V tile as TMA lands it: four page blocks,
+// each [K|V][DH/64 halves][16 keys][64] (the arena's own layout), 128-byte swizzle inside every row.
+template <int DH>
+__device__ __forceinline__ uint32_t kv_off(int r, int c, int is_v) {
+  return static_cast<uint32_t>((r >> 4) * (DH * 64) + is_v * (DH * 32) + (c >> 3) * 2048 + (r & 15) * 128 +
+                               (((c & 7) ^ (r & 7)) << 4));
+}
+
 // One warp: 16 query rows against NT*8 keys starting at tile-local key `kofs`.
 // qf: Q fragments; m, l: running max (scaled, log2 domain) and per-thread partial sums of the two
 // rows this thread touches (row lane/4 and row lane/4 + 8); oacc: unnormalised output.
 template <int DH, int NT>
-__device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], uint32_t k_tile, uint32_t v_tile,
+__device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], uint32_t kv_tile,
                                             int kofs, int key_base, int key_end, int pos_a, int pos_b,
                                             float scale_log2, float (&m)[2], float (&l)[2],
                                             float (&oacc)[DH / 8][4]) {
@@ -141,7 +150,7 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
       for (int np = 0; np < NT / 2; ++np) {
         const int key = kofs + np * 16 + (j >> 1) * 8 + rr;
         uint32_t b[4];
-        ldsm_x4(k_tile + tile_off<DH>(key, ks * 2 + (j & 1)), b);
+        ldsm_x4(kv_tile + kv_off<DH>(key, ks * 2 + (j & 1), 0), b);
         mma_f16(s[np * 2], qf[ks], b[0], b[1]);
         mma_f16(s[np * 2 + 1], qf[ks], b[2], b[3]);
       }
@@ -201,7 +210,7 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
 #pragma unroll
       for (int dp = 0; dp < DH / 16; ++dp) {
         uint32_t b[4];
-        ldsm_x4_trans(v_tile + tile_off<DH>(key, dp * 2 + (j >> 1)), b);
+        ldsm_x4_trans(kv_tile + kv_off<DH>(key, dp * 2 + (j >> 1), 1), b);
         mma_f16(oacc[dp * 2], a, b[0], b[1]);
         mma_f16(oacc[dp * 2 + 1], a, b[2], b[3]);
       }
@@ -214,7 +223,6 @@ __global__ void __launch_bounds__(ATT_THREADS)
 attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   constexpr int CH = DH / 8;                          // 16-byte chunks per row
   constexpr int TILE_BYTES = TILE_KEYS * DH * 2;
-  constexpr int PAGE_HALF_BYTES = 16 * 128;           // one page of one 64-column half
   constexpr int REC = DH + 2;                         // floats per row of a partial record
   extern __shared__ uint8_t smem_raw[];
   // carve-up (1024-byte aligned for the TMA swizzle): STAGES x (K tile, V tile) | barriers, flag | page ids.
@@ -264,23 +272,19 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   }
 
   const int n_tiles = (it.key1 - it.key0 + TILE_KEYS - 1) / TILE_KEYS;
-  // one thread: request the pages of tile kt from TMA (K and V, every 64-column half)
+  // one thread: request the pages of tile kt from TMA, one copy (K and V of this head) per page
+  constexpr int PAGE_BYTES = DH * 64;
   auto issue_tile = [&](int kt) {
     const int st = kt % STAGES;
     const uint32_t k_dst = kv_s + st * 2 * TILE_BYTES, bar = bar_s + 8u * st;
     const int kb = it.key0 + kt * TILE_KEYS;
     const int n_pg = min(TILE_KEYS / 16, (it.key1 - kb + 15) / 16);
     const int pi0 = kb / 16 - first_blk;
-    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n_pg) * 2u * (DH / 64) * PAGE_HALF_BYTES);
+    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n_pg) * PAGE_BYTES);
     for (int pi = 0; pi < n_pg; ++pi) {
       const int64_t page = pg_s[pi0 + pi];
-      const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.kv.n_pages + page) * 2) * p.kv.Hkv + hk) * 16);
-      const int row_v = row_k + p.kv.Hkv * 16;
-#pragma unroll
-      for (int h = 0; h < DH / 64; ++h) {
-        tma_load_2d(k_dst + h * (64 * 128) + pi * PAGE_HALF_BYTES, &kv_map, bar, h * 64, row_k);
-        tma_load_2d(k_dst + TILE_BYTES + h * (64 * 128) + pi * PAGE_HALF_BYTES, &kv_map, bar, h * 64, row_v);
-      }
+      const int row = static_cast<int>(((static_cast<int64_t>(p.layer) * p.kv.n_pages + page) * p.kv.Hkv + hk) * (DH / 2));
+      tma_load_2d(k_dst + pi * PAGE_BYTES, &kv_map, bar, 0, row);
     }
   };
   int issued = 0;
@@ -330,21 +334,19 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     if (valid_rows < TILE_KEYS) {
       // rows past the last key hold stale bytes (rest of the last page, pages not requested): zero the
       // V rows so that a zero probability times garbage cannot produce NaN (K rows are masked anyway)
-      uint8_t* v_gen = smem + (kt % STAGES) * 2 * TILE_BYTES + TILE_BYTES;
+      uint8_t* kv_gen = smem + (kt % STAGES) * 2 * TILE_BYTES;
       for (int u = tid; u < (TILE_KEYS - valid_rows) * CH; u += ATT_THREADS) {
         const int rr = valid_rows + u / CH, c = u % CH;
-        *reinterpret_cast<uint4*>(v_gen + tile_off<DH>(rr, c)) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(kv_gen + kv_off<DH>(rr, c, 1)) = make_uint4(0u, 0u, 0u, 0u);
       }
       __syncthreads();
     }
     if (decode) {
       if (key_base + warp * 16 < it.key1)
-        warp_attend<DH, 2>(qf, k_tile, k_tile + TILE_BYTES, warp * 16, key_base, it.key1, pos_a, pos_b,
-                           p.scale_log2, m, l, oacc);
+        warp_attend<DH, 2>(qf, k_tile, warp * 16, key_base, it.key1, pos_a, pos_b, p.scale_log2, m, l, oacc);
     } else {
       if (key_base <= warp_last)
-        warp_attend<DH, 8>(qf, k_tile, k_tile + TILE_BYTES, 0, key_base, it.key1, pos_a, pos_b, p.scale_log2, m,
-                           l, oacc);
+        warp_attend<DH, 8>(qf, k_tile, 0, key_base, it.key1, pos_a, pos_b, p.scale_log2, m, l, oacc);
     }
   }
   if (__syncthreads_or(failed)) {

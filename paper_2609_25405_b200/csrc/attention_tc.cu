@@ -4,9 +4,11 @@
 // One CTA handles 128 query rows = (128 / G) consecutive tokens x the G query heads of one KV head
 // (G = Hq / Hkv) of one chunk segment, against every key the rows may see, in tiles of 64 keys
 // (4 KV pages).  192 threads:
-//   warp 0    TMA: gathers the pages of each key tile (one 2-D copy per page and 64-column half)
-//             into a shared-memory ring in the 128-byte-swizzled layout the MMA descriptors expect
-//   warp 1    MMA: S_j = Q K_j^T (128 x 64, fp32 in TMEM, double buffered) and
+//   warp 0    TMA: gathers the pages of each key tile (one 2-D copy per page: the contiguous K+V
+//             block of this KV head) into a shared-memory ring in the 128-byte-swizzled layout the
+//             MMA descriptors expect
+//   warp 1    MMA: S_j = Q K_j^T (128 x 64, fp32 in TMEM, double buffered; 16 columns = one page
+//             per instruction, because a tile's keys live in four separate page blocks) and
 //             O += P_j V_j (128 x Dh, fp32 in TMEM), both tcgen05.mma kind::f16 from shared memory;
 //             S_{j+1} is issued before P_j V_j so the tensor pipe works while softmax runs
 //   warps 2-5 softmax: one thread per query row (TMEM lane): read its S row, mask, running max and
@@ -153,10 +155,11 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
 
 template <int DH>
 struct TcCfg {
-  static constexpr int SUB = DH / 64;                    // 64-column sub-tiles
   static constexpr int STAGES = (DH == 128) ? 2 : 4;
   static constexpr int Q_BYTES = BM * DH * 2;
-  static constexpr int KV_HALF = BN * DH * 2;            // K (or V) tile of one stage
+  static constexpr int KV_HALF = BN * DH * 2;            // K (or V) bytes of one stage
+  static constexpr int PAGE_BYTES = DH * 64;             // one page block: [K|V][SUB][16 keys][64]
+  static constexpr int KV_BLOCK = DH * 32;               // K (or V) part of a page block
   static constexpr int P_BYTES = BM * BN * 2;
   static constexpr int RING = STAGES * 2 * KV_HALF;
   static constexpr int BAR_OFF = Q_BYTES + RING + P_BYTES;
@@ -256,18 +259,13 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         const int kb = j * BN;
         const int n_pg = min(BN / 16, (it.key1 - kb + 15) / 16);
         const uint32_t k_dst = ring_s + st * 2 * C::KV_HALF;
-        mbar_arrive_expect_tx(kv_full(st), static_cast<uint32_t>(n_pg) * 2u * C::SUB * (16 * 128));
+        mbar_arrive_expect_tx(kv_full(st), static_cast<uint32_t>(n_pg) * C::PAGE_BYTES);
 #pragma unroll
         for (int pi = 0; pi < BN / 16; ++pi) {
           if (pi < n_pg) {
             const int64_t page = cur[pi];
-            const int row_k = static_cast<int>((((static_cast<int64_t>(p.layer) * p.n_pages + page) * 2) * p.Hkv + hk) * 16);
-            const int row_v = row_k + p.Hkv * 16;
-#pragma unroll
-            for (int h = 0; h < C::SUB; ++h) {
-              tma_load_2d(k_dst + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_k);
-              tma_load_2d(k_dst + C::KV_HALF + h * (BN * 128) + pi * 2048, &kv_map, kv_full(st), h * 64, row_v);
-            }
+            const int row = static_cast<int>(((static_cast<int64_t>(p.layer) * p.n_pages + page) * p.Hkv + hk) * (DH / 2));
+            tma_load_2d(k_dst + pi * C::PAGE_BYTES, &kv_map, kv_full(st), 0, row);   // K and V of this head, one copy
           }
         }
       }
@@ -276,7 +274,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(BN, false);
+      constexpr uint32_t idesc_s = make_idesc(16, false);   // one page of keys per MMA
       constexpr uint32_t idesc_o = make_idesc(DH, true);
       auto issue_s = [&](int j) -> bool {
         const int st = j % C::STAGES, b = j & 1;
@@ -284,11 +282,15 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         if (!mbar_wait(s_empty(b), static_cast<uint32_t>(((j >> 1) & 1) ^ 1), abort_flag)) return false;
         tc_fence_after();
         const uint32_t k_tile = ring_s + st * 2 * C::KV_HALF;
+        // the keys of a tile sit in four page blocks, so S is built 16 columns (one page) at a time
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-          const uint64_t ad = make_desc(q_s + (ks >> 2) * (BM * 128) + (ks & 3) * 32, 16, 1024);
-          const uint64_t bd = make_desc(k_tile + (ks >> 2) * (BN * 128) + (ks & 3) * 32, 16, 1024);
-          umma(tmem + static_cast<uint32_t>(b * BN), ad, bd, idesc_s, ks > 0 ? 1u : 0u);
+        for (int pi = 0; pi < BN / 16; ++pi) {
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks) {
+            const uint64_t ad = make_desc(q_s + (ks >> 2) * (BM * 128) + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = make_desc(k_tile + pi * C::PAGE_BYTES + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024);
+            umma(tmem + static_cast<uint32_t>(b * BN + pi * 16), ad, bd, idesc_s, ks > 0 ? 1u : 0u);
+          }
         }
         umma_commit(s_full(b));
         return true;
@@ -299,11 +301,11 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         if (!ok) break;
         if (!mbar_wait(p_ready, static_cast<uint32_t>(j & 1), abort_flag)) break;
         tc_fence_after();
-        const uint32_t v_tile = ring_s + (j % C::STAGES) * 2 * C::KV_HALF + C::KV_HALF;
+        const uint32_t kv_tile = ring_s + (j % C::STAGES) * 2 * C::KV_HALF;
 #pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks) {
+        for (int ks = 0; ks < BN / 16; ++ks) {   // one page (16 keys) per k-step
           const uint64_t ad = make_desc(p_s + ks * 32, 16, 1024);
-          const uint64_t bd = make_desc(v_tile + ks * 2048, BN * 128, 1024);
+          const uint64_t bd = make_desc(kv_tile + ks * C::PAGE_BYTES + C::KV_BLOCK, 2048, 1024);
           umma(tmem + static_cast<uint32_t>(C::O_COL), ad, bd, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(kv_empty(j % C::STAGES));
@@ -395,12 +397,12 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
       // keys past the end of the request hold stale bytes: zero those V rows (0 * garbage must stay 0)
       const int valid_keys = it.key1 - key_base;
       if (valid_keys < BN) {
-        uint8_t* v_gen = smem + C::Q_BYTES + (j % C::STAGES) * 2 * C::KV_HALF + C::KV_HALF;
+        uint8_t* kv_gen = smem + C::Q_BYTES + (j % C::STAGES) * 2 * C::KV_HALF;
         const int t4 = tid - 64;  // 0..127 over the four softmax warps
         for (int u = t4; u < (BN - valid_keys) * (DH / 8); u += 128) {
           const int kr = valid_keys + u / (DH / 8), c = u % (DH / 8);
-          *reinterpret_cast<uint4*>(v_gen + (c >> 3) * (BN * 128) + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) =
-              make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(kv_gen + (kr >> 4) * C::PAGE_BYTES + C::KV_BLOCK + (c >> 3) * 2048 + (kr & 15) * 128 +
+                                    (((c & 7) ^ (kr & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
         }
       }
       fence_async_smem();

@@ -277,6 +277,13 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
 // of the weight are pair-interleaved inside each head (column 2i = rotary element i, column 2i+1 =
 // element i + Dh/2), so every rotation pair sits in adjacent columns.  q goes to the query buffer,
 // k and v to slot pos % P of the row's page; all as fp16.
+// Address of 32 consecutive head-dimension elements starting at `off` of one cache row.  Arena layout:
+// [page][kv head][K|V][Dh/64 halves][P slots][64], so the K+V block of one (page, head) is contiguous.
+__device__ __forceinline__ __half* kv_slot_ptr(const GemmArgs& g, int page, int kv_head, int is_v, int slot, int off) {
+  return g.kv_layer + static_cast<int64_t>(page) * g.page_stride +
+         static_cast<int64_t>(kv_head * 2 + is_v) * g.Dh * g.P + (off >> 6) * (g.P * 64) + slot * 64 + (off & 63);
+}
+
 __device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32],
                                                   int pos, int page) {
   const int Dh = g.Dh;
@@ -299,14 +306,12 @@ __device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, in
     if (head < g.Hq) {
       dst = g.q_out + static_cast<size_t>(row) * g.Hq * Dh + col0;
     } else {
-      dst = g.kv_layer + static_cast<int64_t>(page) * g.page_stride +
-            static_cast<int64_t>(head - g.Hq) * g.P * Dh + (pos % g.P) * Dh + off;
+      dst = kv_slot_ptr(g, page, head - g.Hq, 0, pos % g.P, off);
     }
   } else {
 #pragma unroll
     for (int j = 0; j < 16; ++j) pk[j] = pack_f16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-    dst = g.kv_layer + static_cast<int64_t>(page) * g.page_stride +
-          static_cast<int64_t>(head - g.Hq) * g.P * Dh + (pos % g.P) * Dh + off;   // V blocks follow the K blocks
+    dst = kv_slot_ptr(g, page, head - g.Hq - g.Hkv, 1, pos % g.P, off);
   }
 #pragma unroll
   for (int v = 0; v < 4; ++v)

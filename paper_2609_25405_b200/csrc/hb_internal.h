@@ -64,13 +64,13 @@ struct DeviceDesc {
 struct KvGeom {
   __half* arena;
   int64_t layer_stride;  // elements
-  int64_t page_stride;   // elements: 2 * Hkv * P * Dh
+  int64_t page_stride;   // elements: Hkv * 2 * Dh * P; inside a page: [kv head][K|V][Dh/64][P][64]
   int32_t n_pages, Hkv, P, Dh;
 };
 
 struct hb_kv {
   hb_model_cfg cfg;
-  CUtensorMap map;      // arena as a 2-D bf16 tensor [rows of head_dim], box = one page x 64 columns
+  CUtensorMap map;      // arena as a 2-D tensor [rows of 64 fp16], box = the K+V block of one (page, kv head)
   bool has_map;
   void* arena;
   size_t arena_bytes;

@@ -339,8 +339,11 @@ int hb_kv_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32
   kv->cfg = *cfg;
   kv->has_map = false;
   if (arena) {
-    const uint64_t rows = static_cast<uint64_t>(cfg->n_layers) * n_pages * 2 * cfg->n_kv_heads * cfg->page_size;
-    if (rows > 0x7fffffffull || hb_tmap_2d_bf16(&kv->map, arena, rows, cfg->head_dim, 16) != HB_OK) {
+    // arena as rows of 64 elements; one copy box = the K+V block of one (page, kv head)
+    const uint64_t halves = cfg->head_dim / 64;
+    const uint64_t rows = static_cast<uint64_t>(cfg->n_layers) * n_pages * cfg->n_kv_heads * 2 * halves * cfg->page_size;
+    if (rows > 0x7fffffffull ||
+        hb_tmap_2d_bf16(&kv->map, arena, rows, 64, static_cast<uint32_t>(2 * halves * cfg->page_size)) != HB_OK) {
       delete kv;
       return rows > 0x7fffffffull ? HB_ERR_TOO_LARGE : HB_ERR_CUDA;
     }

@@ -69,7 +69,7 @@ def test_fullsize_sampled_requests_match_oracle(name):
         total = len(r.tokens) + n_steps + 1
         r.pages = eng.kv.alloc((total + P - 1) // P)
         sampled_pages[r] = list(r.pages)
-    view = eng.kv.arena.view(shape.L, n_pages, 2, shape.Hkv, P, shape.Dh)
+    view = eng.kv.arena.view(shape.L, n_pages, shape.Hkv, 2, shape.Dh // 64, P, 64)
     for r in gens + embs:
         view[:, torch.tensor(r.pages)] = KV_SENTINEL
     # ---- filler ----
@@ -166,16 +166,16 @@ def test_fullsize_sampled_requests_match_oracle(name):
         cos = float(got @ ref / (np.linalg.norm(got) * np.linalg.norm(ref)))
         assert cos >= EMB_COS and np.max(np.abs(got - ref)) <= EMB_ABS, (cos, np.max(np.abs(got - ref)))
     # ---- bookkeeping on the sampled requests' pages: written slots hold values, the rest the sentinel
-    raw = eng.kv.arena.view(shape.L, n_pages, 2, shape.Hkv, P, shape.Dh)
+    raw = eng.kv.arena.view(shape.L, n_pages, shape.Hkv, 2, shape.Dh // 64, P, 64)
     for r in gens + embs:
         n = r.n_done
         pages = sampled_pages[r]
         for blk, pg in enumerate(pages):
             written = max(0, min(P, n - blk * P))
             if written < P:
-                assert torch.all(raw[:, pg, :, :, written:, :] == KV_SENTINEL), (blk, pg)
+                assert torch.all(raw[:, pg, :, :, :, written:, :] == KV_SENTINEL), (blk, pg)
             if written > 0:
-                assert not torch.any(raw[0, pg, :, :, :written, :] == KV_SENTINEL)
+                assert not torch.any(raw[0, pg, :, :, :, :written, :] == KV_SENTINEL)
         cnt, chunks = M.pool_counters_after(synth.nominal_chunks(len(r.tokens), chunk)) if r.kind == "embed" else (0, 0)
         if r.kind == "embed":
             meta = eng.pool.meta()[r.slot].cpu().numpy()

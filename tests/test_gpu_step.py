@@ -95,8 +95,7 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
     # ---- KV bookkeeping: exactly the expected slots were written, everything else is the sentinel
     from paper_2609_25405_b200 import binding as B
     W = weights[0]
-    kvv = eng.kv.view().cpu()                                   # [L, page, 2, Hkv, P, Dh] fp16
-    raw = eng.kv.arena.cpu().view(TINY.L, eng.kv.n_pages, 2, TINY.Hkv, 16, TINY.Dh)
+    raw = eng.kv.arena.cpu().view(TINY.L, eng.kv.n_pages, TINY.Hkv, 2, TINY.Dh // 64, 16, 64)
     touched = torch.zeros((eng.kv.n_pages, 16), dtype=torch.bool)
     for req in gens + embs:
         n = req.n_done
@@ -106,15 +105,15 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
             page, slot = M.kv_slot(req.pages, pos, 16)
             touched[page, slot] = True
         for l in range(TINY.L):
-            pages = torch.tensor([M.kv_slot(req.pages, p, 16)[0] for p in range(n)])
-            slots = torch.tensor([M.kv_slot(req.pages, p, 16)[1] for p in range(n)])
-            k_st = kvv[l, :, 0][pages, :, slots, :].float().numpy()    # [n, Hkv, Dh], pair-interleaved
+            pages = torch.tensor([M.kv_slot(req.pages, p, 16)[0] for p in range(n)], device="cuda")
+            slots = torch.tensor([M.kv_slot(req.pages, p, 16)[1] for p in range(n)], device="cuda")
+            k_st = eng.kv.rows(l, pages, slots, 0).float().cpu().numpy()   # [n, Hkv, Dh], pair-interleaved
             k_gpu = np.empty_like(k_st)
-            k_gpu[..., B.rope_pair_order(TINY.Dh)] = k_st               # back to the rotary element order
-            v_gpu = kvv[l, :, 1][pages, :, slots, :].float().numpy()
+            k_gpu[..., B.rope_pair_order(TINY.Dh)] = k_st                   # back to the rotary element order
+            v_gpu = eng.kv.rows(l, pages, slots, 1).float().cpu().numpy()
             assert np.max(np.abs(k_gpu - kv_ref[l][0])) < 5e-3
             assert np.max(np.abs(v_gpu - kv_ref[l][1])) < 5e-3
-    untouched = ~touched[None, :, None, None, :, None].expand_as(raw)
+    untouched = ~touched[None, :, None, None, None, :, None].expand_as(raw)
     assert torch.all(raw[untouched] == KV_SENTINEL)
     # ---- pool bookkeeping: counters equal the oracle's integers; unused slots keep the sentinel
     meta = eng.pool.meta().cpu().numpy()
