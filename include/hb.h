@@ -158,9 +158,11 @@ HB_API int hb_destroy(hb_ctx* ctx);
 /* ---- paged KV cache ------------------------------------------------------- */
 
 /* Bytes of an arena of n_pages.  Arena layout (fp16; post-rotary K and V):
- * [layer][page][kv_head][K|V][head_dim/64][slot 0..page_size)[64], i.e. the
- * head dimension is split into 64-element halves and the K+V block of one
- * (layer, page, head) is contiguous (4-8 KiB): one TMA copy fetches it.
+ * [layer][page][kv_head][slot group][K|V][head_dim/64][8 slots][64]: slots 0-7
+ * and 8-15 of a page form two groups, the head dimension is split into
+ * 64-element halves, and the K+V block of one (layer, page, head) is contiguous
+ * (4-8 KiB), so one TMA copy fetches it and the blocks of consecutive pages
+ * line up in shared memory the way the tensor-core descriptors need.
  * Host only. */
 HB_API int hb_kv_arena_bytes(const hb_model_cfg* cfg, int32_t n_pages, size_t* out_bytes);
 

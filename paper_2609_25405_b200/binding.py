@@ -236,16 +236,16 @@ class KvCache:
                                C.byref(self.handle)), "hb_kv_create")
 
     def view(self):
-        """fp16 view [L, page, Hkv, 2 (K|V), Dh/64, P, 64] (the arena's own layout)."""
+        """fp16 view [L, page, Hkv, 2 (slot group), 2 (K|V), Dh/64, 8, 64] (the arena's own layout)."""
         c = self.cfg
-        return self.arena.view(torch.float16).view(c.n_layers, self.n_pages, c.n_kv_heads, 2, c.head_dim // 64,
-                                                   c.page_size, 64)
+        return self.arena.view(torch.float16).view(c.n_layers, self.n_pages, c.n_kv_heads, 2, 2, c.head_dim // 64,
+                                                   8, 64)
 
     def rows(self, layer, pages, slots, is_v):
         """K (is_v = 0) or V (1) rows of `layer` at (pages[i], slots[i]) as [n, Hkv, Dh] fp16, in the
         stored head-dimension order."""
-        v = self.view()[layer][:, :, is_v]                      # [page, Hkv, H2, P, 64]
-        r = v[pages, :, :, slots, :]                            # [n, Hkv, H2, 64]
+        v = self.view()[layer][:, :, :, is_v]                   # [page, Hkv, group, H2, 8, 64]
+        r = v[pages, :, slots // 8, :, slots % 8, :]            # [n, Hkv, H2, 64]
         return r.reshape(r.shape[0], r.shape[1], -1)
 
     def alloc(self, n):

@@ -121,12 +121,13 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
   return static_cast<uint32_t>((c >> 3) * (64 * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-// Byte offset of 16-byte chunk `c` of key `r` of a 64-key K/V tile as TMA lands it: four page blocks,
-// each [K|V][DH/64 halves][16 keys][64] (the arena's own layout), 128-byte swizzle inside every row.
+// Byte offset of 16-byte chunk `c` of key `r` of a 64-key K/V tile as TMA lands it: four page blocks
+// of DH*64 bytes, each [slot group][K|V][DH/64 halves][8 keys][64] (the arena's own layout), 128-byte
+// swizzle inside every row.
 template <int DH>
 __device__ __forceinline__ uint32_t kv_off(int r, int c, int is_v) {
-  return static_cast<uint32_t>((r >> 4) * (DH * 64) + is_v * (DH * 32) + (c >> 3) * 2048 + (r & 15) * 128 +
-                               (((c & 7) ^ (r & 7)) << 4));
+  return static_cast<uint32_t>((r >> 4) * (DH * 64) + ((r >> 3) & 1) * (DH * 32) + (is_v * (DH / 64) + (c >> 3)) * 1024 +
+                               (r & 7) * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
 // One warp: 16 query rows against NT*8 keys starting at tile-local key `kofs`.

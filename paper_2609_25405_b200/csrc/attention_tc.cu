@@ -7,8 +7,7 @@
 //   warp 0    TMA: gathers the pages of each key tile (one 2-D copy per page: the contiguous K+V
 //             block of this KV head) into a shared-memory ring in the 128-byte-swizzled layout the
 //             MMA descriptors expect
-//   warp 1    MMA: S_j = Q K_j^T (128 x 64, fp32 in TMEM, double buffered; 16 columns = one page
-//             per instruction, because a tile's keys live in four separate page blocks) and
+//   warp 1    MMA: S_j = Q K_j^T (128 x 64, fp32 in TMEM; Q is the A operand, held in TMEM) and
 //             O += P_j V_j (128 x Dh, fp32 in TMEM), both tcgen05.mma kind::f16 from shared memory;
 //             S_{j+1} is issued before P_j V_j so the tensor pipe works while softmax runs
 //   warps 2-5 softmax: one thread per query row (TMEM lane): read its S row, mask, running max and
@@ -85,10 +84,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
       : "memory");
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-  const int sz = valid ? 16 : 0;
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -116,6 +111,15 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// A operand from tensor memory (16-bit elements, two per 32-bit column), B from shared memory.
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -155,16 +159,18 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
 
 template <int DH>
 struct TcCfg {
-  static constexpr int STAGES = (DH == 128) ? 2 : 4;
-  static constexpr int Q_BYTES = BM * DH * 2;
+  static constexpr int STAGES = (DH == 128) ? 3 : 4;
   static constexpr int KV_HALF = BN * DH * 2;            // K (or V) bytes of one stage
-  static constexpr int PAGE_BYTES = DH * 64;             // one page block: [K|V][SUB][16 keys][64]
-  static constexpr int KV_BLOCK = DH * 32;               // K (or V) part of a page block
+  static constexpr int PAGE_BYTES = DH * 64;             // one page block: [slot group][K|V][DH/64][8 keys][64]
+  static constexpr int GROUP_BYTES = DH * 32;            // one slot group of a page block = stride of 8-key groups
+  static constexpr int V_OFF = (DH / 64) * 1024;         // V part inside a slot group
   static constexpr int P_BYTES = BM * BN * 2;
   static constexpr int RING = STAGES * 2 * KV_HALF;
-  static constexpr int BAR_OFF = Q_BYTES + RING + P_BYTES;
-  static constexpr int TMEM_COLS = 256;                  // S: 2 x 64 columns, O: DH columns
-  static constexpr int O_COL = 128;
+  static constexpr int BAR_OFF = RING + P_BYTES;
+  static constexpr int TMEM_COLS = 256;
+  static constexpr int S_COL = 0;                        // S: 64 columns (fp32)
+  static constexpr int Q_COL = 64;                       // Q: DH/2 columns (two fp16 per column)
+  static constexpr int O_COL = 128;                      // O: DH columns (fp32)
 };
 
 template <int DH>
@@ -180,12 +186,12 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     if (threadIdx.x == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
     return;
   }
-  const uint32_t q_s = base, ring_s = base + C::Q_BYTES, p_s = ring_s + C::RING, bar_s = base + C::BAR_OFF;
+  const uint32_t ring_s = base, p_s = ring_s + C::RING, bar_s = base + C::BAR_OFF;
   auto kv_full = [&](int s) { return bar_s + 8u * s; };
   auto kv_empty = [&](int s) { return bar_s + 8u * (C::STAGES + s); };
-  auto s_full = [&](int b) { return bar_s + 8u * (2 * C::STAGES + b); };
-  auto s_empty = [&](int b) { return bar_s + 8u * (2 * C::STAGES + 2 + b); };
-  const uint32_t p_ready = bar_s + 8u * (2 * C::STAGES + 4), pv_done = bar_s + 8u * (2 * C::STAGES + 5);
+  const uint32_t s_full = bar_s + 8u * (2 * C::STAGES), s_empty = bar_s + 8u * (2 * C::STAGES + 1);
+  const uint32_t q_ready = bar_s + 8u * (2 * C::STAGES + 2), p_ready = bar_s + 8u * (2 * C::STAGES + 4),
+                 pv_done = bar_s + 8u * (2 * C::STAGES + 5);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -198,7 +204,9 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 
   if (tid == 0) {
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(s_empty(b), 4); }
+    mbar_init(s_full, 1);
+    mbar_init(s_empty, 4);
+    mbar_init(q_ready, 4);
     mbar_init(p_ready, 4);
     mbar_init(pv_done, 1);
     *abort_flag = 0u;
@@ -210,19 +218,6 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     const int pg = (i < sg.pt_len) ? p.pages[sg.pt_start + i] : -1;
     bad |= (pg < 0 || pg >= p.n_pages);
   }
-  // Q tile -> shared memory in the K-major 128-byte-swizzled layout ([SUB][128 rows][64]); rows past
-  // n_rows are zero
-  for (int u = tid; u < BM * (DH / 8); u += TC_THREADS) {
-    const int rr = u / (DH / 8), c = u - rr * (DH / 8);
-    const int r = it.row0 + rr;
-    const bool valid = rr < it.n_rows;
-    const int tok = sg.q_start + (valid ? r / G : 0), head = hk * G + (valid ? r % G : 0);
-    const __half* src = p.q + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8;
-    const uint32_t off = static_cast<uint32_t>((c >> 3) * (BM * 128) + rr * 128 + (((c & 7) ^ (rr & 7)) << 4));
-    cp_async16(q_s + off, src, valid);
-  }
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-  fence_async_smem();   // Q was written through the generic proxy; the MMA reads it through the async proxy
   if (__syncthreads_or(bad)) {
     if (tid == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
     return;             // nothing requested from TMA, no TMEM held
@@ -274,38 +269,40 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(16, false);   // one page of keys per MMA
+      constexpr uint32_t idesc_s = make_idesc(BN, false);
       constexpr uint32_t idesc_o = make_idesc(DH, true);
+      // S_j = Q K_j^T: Q comes from TMEM (written once by the softmax warps), K from shared memory: the
+      // 8-key groups of the four page blocks of a tile are GROUP_BYTES apart, so one descriptor spans
+      // all 64 keys.
       auto issue_s = [&](int j) -> bool {
-        const int st = j % C::STAGES, b = j & 1;
+        const int st = j % C::STAGES;
         if (!mbar_wait(kv_full(st), static_cast<uint32_t>((j / C::STAGES) & 1), abort_flag)) return false;
-        if (!mbar_wait(s_empty(b), static_cast<uint32_t>(((j >> 1) & 1) ^ 1), abort_flag)) return false;
+        if (!mbar_wait(s_empty, static_cast<uint32_t>((j & 1) ^ 1), abort_flag)) return false;
         tc_fence_after();
         const uint32_t k_tile = ring_s + st * 2 * C::KV_HALF;
-        // the keys of a tile sit in four page blocks, so S is built 16 columns (one page) at a time
 #pragma unroll
-        for (int pi = 0; pi < BN / 16; ++pi) {
-#pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
-            const uint64_t ad = make_desc(q_s + (ks >> 2) * (BM * 128) + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = make_desc(k_tile + pi * C::PAGE_BYTES + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024);
-            umma(tmem + static_cast<uint32_t>(b * BN + pi * 16), ad, bd, idesc_s, ks > 0 ? 1u : 0u);
-          }
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint64_t bd = make_desc(k_tile + (ks >> 2) * 1024 + (ks & 3) * 32, 16, C::GROUP_BYTES);
+          umma_ts(tmem + static_cast<uint32_t>(C::S_COL), tmem + static_cast<uint32_t>(C::Q_COL + ks * 8), bd, idesc_s,
+                  ks > 0 ? 1u : 0u);
         }
-        umma_commit(s_full(b));
+        umma_commit(s_full);
         return true;
       };
-      bool ok = issue_s(0);
+      bool ok = mbar_wait(q_ready, 0u, abort_flag);
+      if (ok) ok = issue_s(0);
       for (int j = 0; ok && j < n_tiles; ++j) {
+        // S_{j+1} may start as soon as the softmax warps have read S_j out of TMEM
         if (j + 1 < n_tiles) ok = issue_s(j + 1);
         if (!ok) break;
         if (!mbar_wait(p_ready, static_cast<uint32_t>(j & 1), abort_flag)) break;
         tc_fence_after();
         const uint32_t kv_tile = ring_s + (j % C::STAGES) * 2 * C::KV_HALF;
 #pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks) {   // one page (16 keys) per k-step
+        for (int ks = 0; ks < BN / 16; ++ks) {   // one page (16 keys = two 8-key groups) per k-step
           const uint64_t ad = make_desc(p_s + ks * 32, 16, 1024);
-          const uint64_t bd = make_desc(kv_tile + ks * C::PAGE_BYTES + C::KV_BLOCK, 2048, 1024);
+          // V is the MN-major B operand: 64-column halves 1024 B apart, 8-key groups GROUP_BYTES apart
+          const uint64_t bd = make_desc(kv_tile + ks * C::PAGE_BYTES + C::V_OFF, 1024, C::GROUP_BYTES);
           umma(tmem + static_cast<uint32_t>(C::O_COL), ad, bd, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(kv_empty(j % C::STAGES));
@@ -327,17 +324,36 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     auto wait_w = [&](uint32_t bar, uint32_t parity) {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag)) != 0;
     };
+    // this thread's query row -> TMEM (two fp16 per column), the A operand of every S MMA
+    {
+      const int tok = sg.q_start + (row_valid ? r / G : 0), head = hk * G + (row_valid ? r % G : 0);
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(tok) * Hq + head) * DH);
+#pragma unroll
+      for (int c = 0; c < DH / 2; c += 32) {
+        uint32_t qr[32];
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+          const uint4 x = row_valid ? __ldg(src + c / 4 + v) : make_uint4(0u, 0u, 0u, 0u);
+          qr[v * 4 + 0] = x.x; qr[v * 4 + 1] = x.y; qr[v * 4 + 2] = x.z; qr[v * 4 + 3] = x.w;
+        }
+        tmem_st32(t_lane + static_cast<uint32_t>(C::Q_COL + c), qr);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(q_ready);
+    }
     for (int j = 0; j < n_tiles; ++j) {
-      const int b = j & 1, key_base = j * BN;
-      if (!wait_w(s_full(b), static_cast<uint32_t>((j >> 1) & 1))) { ok = false; break; }
+      const int key_base = j * BN;
+      if (!wait_w(s_full, static_cast<uint32_t>(j & 1))) { ok = false; break; }
       tc_fence_after();
       uint32_t sr[2][32];
-      tmem_ld32(t_lane + static_cast<uint32_t>(b * BN), sr[0]);
-      tmem_ld32(t_lane + static_cast<uint32_t>(b * BN + 32), sr[1]);
+      tmem_ld32(t_lane + static_cast<uint32_t>(C::S_COL), sr[0]);
+      tmem_ld32(t_lane + static_cast<uint32_t>(C::S_COL + 32), sr[1]);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(s_empty(b));
+      if (lane == 0) mbar_arrive(s_empty);
       // scale, mask (only tiles that touch the diagonal or the end of the keys), row maximum
       const bool need_mask = (key_base + BN - 1 > pos) || (key_base + BN > it.key1);
       float mx = -INFINITY;
@@ -378,7 +394,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
       }
       const float ms = (m_used == -INFINITY) ? 0.0f : m_used;
       // probabilities -> fp16 P row in shared memory (K-major, 128-byte swizzle)
-      uint8_t* prow = smem + C::Q_BYTES + C::RING + rr * 128;
+      uint8_t* prow = smem + C::RING + rr * 128;
       float sum = 0.0f;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -397,12 +413,13 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
       // keys past the end of the request hold stale bytes: zero those V rows (0 * garbage must stay 0)
       const int valid_keys = it.key1 - key_base;
       if (valid_keys < BN) {
-        uint8_t* kv_gen = smem + C::Q_BYTES + (j % C::STAGES) * 2 * C::KV_HALF;
+        uint8_t* kv_gen = smem + (j % C::STAGES) * 2 * C::KV_HALF;
         const int t4 = tid - 64;  // 0..127 over the four softmax warps
         for (int u = t4; u < (BN - valid_keys) * (DH / 8); u += 128) {
           const int kr = valid_keys + u / (DH / 8), c = u % (DH / 8);
-          *reinterpret_cast<uint4*>(kv_gen + (kr >> 4) * C::PAGE_BYTES + C::KV_BLOCK + (c >> 3) * 2048 + (kr & 15) * 128 +
-                                    (((c & 7) ^ (kr & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(kv_gen + (kr >> 4) * C::PAGE_BYTES + ((kr >> 3) & 1) * C::GROUP_BYTES + C::V_OFF +
+                                    (c >> 3) * 1024 + (kr & 7) * 128 + (((c & 7) ^ (kr & 7)) << 4)) =
+              make_uint4(0u, 0u, 0u, 0u);
         }
       }
       fence_async_smem();

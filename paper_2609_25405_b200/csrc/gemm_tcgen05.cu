@@ -278,10 +278,13 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
 // element i + Dh/2), so every rotation pair sits in adjacent columns.  q goes to the query buffer,
 // k and v to slot pos % P of the row's page; all as fp16.
 // Address of 32 consecutive head-dimension elements starting at `off` of one cache row.  Arena layout:
-// [page][kv head][K|V][Dh/64 halves][P slots][64], so the K+V block of one (page, head) is contiguous.
+// [page][kv head][slot group (slots 0-7 | 8-15)][K|V][Dh/64 halves][8 slots][64]: the K+V block of one
+// (page, head) is contiguous (one TMA copy), and the 8-row groups of K (or V) of consecutive pages
+// landed back to back in shared memory are a uniform stride apart, as the MMA descriptors need.
 __device__ __forceinline__ __half* kv_slot_ptr(const GemmArgs& g, int page, int kv_head, int is_v, int slot, int off) {
-  return g.kv_layer + static_cast<int64_t>(page) * g.page_stride +
-         static_cast<int64_t>(kv_head * 2 + is_v) * g.Dh * g.P + (off >> 6) * (g.P * 64) + slot * 64 + (off & 63);
+  const int halves = g.Dh >> 6;
+  return g.kv_layer + static_cast<int64_t>(page) * g.page_stride + static_cast<int64_t>(kv_head) * 2 * g.Dh * g.P +
+         (slot >> 3) * (g.Dh * g.P) + (is_v * halves + (off >> 6)) * 512 + (slot & 7) * 64 + (off & 63);
 }
 
 __device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, int col0, const uint32_t (&r)[32],

@@ -69,7 +69,7 @@ def test_fullsize_sampled_requests_match_oracle(name):
         total = len(r.tokens) + n_steps + 1
         r.pages = eng.kv.alloc((total + P - 1) // P)
         sampled_pages[r] = list(r.pages)
-    view = eng.kv.arena.view(shape.L, n_pages, shape.Hkv, 2, shape.Dh // 64, P, 64)
+    view = eng.kv.arena.view(shape.L, n_pages, shape.Hkv, 2, 2, shape.Dh // 64, 8, 64)
     for r in gens + embs:
         view[:, torch.tensor(r.pages)] = KV_SENTINEL
     # ---- filler ----
@@ -166,7 +166,8 @@ def test_fullsize_sampled_requests_match_oracle(name):
         cos = float(got @ ref / (np.linalg.norm(got) * np.linalg.norm(ref)))
         assert cos >= EMB_COS and np.max(np.abs(got - ref)) <= EMB_ABS, (cos, np.max(np.abs(got - ref)))
     # ---- bookkeeping on the sampled requests' pages: written slots hold values, the rest the sentinel
-    raw = eng.kv.arena.view(shape.L, n_pages, shape.Hkv, 2, shape.Dh // 64, P, 64)
+    raw = eng.kv.arena.view(shape.L, n_pages, shape.Hkv, 2, 2, shape.Dh // 64, 8, 64).permute(0, 1, 2, 4, 5, 3, 6, 7) \
+        .reshape(shape.L, n_pages, shape.Hkv, 2, shape.Dh // 64, P, 64)      # slots back in order 0..15
     for r in gens + embs:
         n = r.n_done
         pages = sampled_pages[r]

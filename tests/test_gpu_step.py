@@ -95,7 +95,7 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
     # ---- KV bookkeeping: exactly the expected slots were written, everything else is the sentinel
     from paper_2609_25405_b200 import binding as B
     W = weights[0]
-    raw = eng.kv.arena.cpu().view(TINY.L, eng.kv.n_pages, TINY.Hkv, 2, TINY.Dh // 64, 16, 64)
+    raw = eng.kv.arena.cpu().view(TINY.L, eng.kv.n_pages, TINY.Hkv, 2, 2, TINY.Dh // 64, 8, 64)   # slot = 8 g + s
     touched = torch.zeros((eng.kv.n_pages, 16), dtype=torch.bool)
     for req in gens + embs:
         n = req.n_done
@@ -113,7 +113,7 @@ def test_cfg1_mixed_workload_matches_oracle(weights):
             v_gpu = eng.kv.rows(l, pages, slots, 1).float().cpu().numpy()
             assert np.max(np.abs(k_gpu - kv_ref[l][0])) < 5e-3
             assert np.max(np.abs(v_gpu - kv_ref[l][1])) < 5e-3
-    untouched = ~touched[None, :, None, None, None, :, None].expand_as(raw)
+    untouched = ~touched.view(-1, 2, 8)[None, :, None, :, None, None, :, None].expand_as(raw)
     assert torch.all(raw[untouched] == KV_SENTINEL)
     # ---- pool bookkeeping: counters equal the oracle's integers; unused slots keep the sentinel
     meta = eng.pool.meta().cpu().numpy()
