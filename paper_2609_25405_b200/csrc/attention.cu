@@ -236,23 +236,60 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   int32_t* pg_s = reinterpret_cast<int32_t*>(smem + STAGES * 2 * TILE_BYTES + 64);
 
   const AttnItem it = p.items[blockIdx.x];
-  const hb_seg sg = p.segs[it.seg];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, Hq = p.Hq;
   const bool decode = (it.mode != 0);
   const int hk = it.kv_head;
 
+  const int n_tiles = (it.key1 - it.key0 + TILE_KEYS - 1) / TILE_KEYS;
+  const int first_blk = it.key0 / p.kv.P;
+  const int n_blk = (it.key1 + p.kv.P - 1) / p.kv.P - first_blk;
+  constexpr int PAGE_BYTES = DH * 64;
+  // one thread: request the pages of tile kt from TMA, one copy (K and V of this head) per page
+  auto issue_pages = [&](int kt, const int (&ids)[TILE_KEYS / 16]) {
+    const int st = kt % STAGES;
+    const uint32_t k_dst = kv_s + st * 2 * TILE_BYTES, bar = bar_s + 8u * st;
+    const int kb = it.key0 + kt * TILE_KEYS;
+    const int n_pg = min(TILE_KEYS / 16, (it.key1 - kb + 15) / 16);
+    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n_pg) * PAGE_BYTES);
+#pragma unroll
+    for (int pi = 0; pi < TILE_KEYS / 16; ++pi) {
+      if (pi < n_pg) {
+        const int row = static_cast<int>(((static_cast<int64_t>(p.layer) * p.kv.n_pages + ids[pi]) * p.kv.Hkv + hk) * (DH / 2));
+        tma_load_2d(k_dst + pi * PAGE_BYTES, &kv_map, bar, 0, row);
+      }
+    }
+  };
+  auto issue_tile = [&](int kt) {
+    int ids[TILE_KEYS / 16];
+    const int pi0 = (it.key0 + kt * TILE_KEYS) / 16 - first_blk;
+#pragma unroll
+    for (int pi = 0; pi < TILE_KEYS / 16; ++pi) ids[pi] = (pi0 + pi < n_blk) ? pg_s[pi0 + pi] : 0;
+    issue_pages(kt, ids);
+  };
+  int issued = 0, bad = 0;
   if (tid == 0) {
     for (int st = 0; st < STAGES; ++st) mbar_init(bar_s + 8u * st, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // the first tiles are requested right away, with page ids read straight from global memory, so
+    // that their latency overlaps the rest of the set-up
+    for (; issued < STAGES - 1 && issued < n_tiles && !bad; ++issued) {
+      int ids[TILE_KEYS / 16];
+      const int pi0 = issued * (TILE_KEYS / 16);
+#pragma unroll
+      for (int pi = 0; pi < TILE_KEYS / 16; ++pi) {
+        const int blk = first_blk + pi0 + pi;
+        ids[pi] = (pi0 + pi < n_blk) ? ((blk < it.pt_len) ? __ldg(p.pages + it.pt_start + blk) : -1) : 0;
+        bad |= (ids[pi] < 0 || ids[pi] >= p.kv.n_pages);
+      }
+      if (bad) break;
+      issue_pages(issued, ids);
+    }
   }
   // page ids of the keys this item reads -> shared memory (checked once)
-  const int first_blk = it.key0 / p.kv.P;
-  const int n_blk = (it.key1 + p.kv.P - 1) / p.kv.P - first_blk;
-  int bad = 0;
   for (int i = tid; i < n_blk; i += ATT_THREADS) {
     const int blk = first_blk + i;
-    const int pg = (blk < sg.pt_len) ? p.pages[sg.pt_start + blk] : -1;
+    const int pg = (blk < it.pt_len) ? p.pages[it.pt_start + blk] : -1;
     bad |= (pg < 0 || pg >= p.kv.n_pages);
     pg_s[i] = pg;
   }
@@ -261,49 +298,32 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     const int rr = u / CH, c = u - rr * CH;
     const int r = it.row0 + rr;
     const bool valid = rr < it.n_rows;
-    const int tok = sg.q_start + (valid ? r / G : 0), head = hk * G + (valid ? r % G : 0);
+    const int tok = it.q_start + (valid ? r / G : 0), head = hk * G + (valid ? r % G : 0);
     const __half* src = p.q + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8;
     cp_async16(q_s + tile_off<DH>(rr, c), src, valid);
   }
   cp_async_commit();
   if (__syncthreads_or(bad)) {  // also publishes the barrier initialisation and the page ids
-    if (tid == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
-    cp_async_wait<0>();
-    return;                     // nothing was requested from TMA yet
-  }
-
-  const int n_tiles = (it.key1 - it.key0 + TILE_KEYS - 1) / TILE_KEYS;
-  // one thread: request the pages of tile kt from TMA, one copy (K and V of this head) per page
-  constexpr int PAGE_BYTES = DH * 64;
-  auto issue_tile = [&](int kt) {
-    const int st = kt % STAGES;
-    const uint32_t k_dst = kv_s + st * 2 * TILE_BYTES, bar = bar_s + 8u * st;
-    const int kb = it.key0 + kt * TILE_KEYS;
-    const int n_pg = min(TILE_KEYS / 16, (it.key1 - kb + 15) / 16);
-    const int pi0 = kb / 16 - first_blk;
-    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n_pg) * PAGE_BYTES);
-    for (int pi = 0; pi < n_pg; ++pi) {
-      const int64_t page = pg_s[pi0 + pi];
-      const int row = static_cast<int>(((static_cast<int64_t>(p.layer) * p.kv.n_pages + page) * p.kv.Hkv + hk) * (DH / 2));
-      tma_load_2d(k_dst + pi * PAGE_BYTES, &kv_map, bar, 0, row);
+    if (tid == 0) {
+      atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
+      for (int st = 0; st < issued; ++st) mbar_wait(bar_s + 8u * st, 0u);   // copies already requested must land
     }
-  };
-  int issued = 0;
-  if (tid == 0) {
-    for (; issued < STAGES - 1 && issued < n_tiles; ++issued) issue_tile(issued);
+    cp_async_wait<0>();
+    __syncthreads();
+    return;
   }
 
   // rows of this thread: chunk items: warp-private rows; decode items: rows 0..15 for every warp
   const int row_base = decode ? 0 : warp * 16;
   const int ra = row_base + (lane >> 2), rb = ra + 8;
   // position of the rows (rows past n_rows get -1: nothing visible)
-  const int pos_a = (ra < it.n_rows) ? sg.pos_start + (it.row0 + ra) / G : -1;
-  const int pos_b = (rb < it.n_rows) ? sg.pos_start + (it.row0 + rb) / G : -1;
+  const int pos_a = (ra < it.n_rows) ? it.pos_start + (it.row0 + ra) / G : -1;
+  const int pos_b = (rb < it.n_rows) ? it.pos_start + (it.row0 + rb) / G : -1;
   // last position any row of this warp can see (skip tiles past it)
   int warp_last = -1;
   {
     const int last_row = min(row_base + 15, it.n_rows - 1);
-    if (last_row >= row_base) warp_last = sg.pos_start + (it.row0 + last_row) / G;
+    if (last_row >= row_base) warp_last = it.pos_start + (it.row0 + last_row) / G;
   }
 
   uint32_t qf[DH / 16][4];
@@ -381,7 +401,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
       const int rr = row_base + u / CH, c = u % CH;
       if (rr < it.n_rows) {
         const int r = it.row0 + rr;
-        const int tok = sg.q_start + r / G, head = hk * G + r % G;
+        const int tok = it.q_start + r / G, head = hk * G + r % G;
         const uint4 v = *reinterpret_cast<const uint4*>(stage + tile_off<DH>(rr, c));
         *reinterpret_cast<uint4*>(p.out + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8) = v;
       }
@@ -410,7 +430,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     }
   }
   __syncthreads();
-  const int tok = sg.q_start;  // a decode segment has one row
+  const int tok = it.q_start;  // a decode segment has one row
   float* rec = p.part + static_cast<size_t>(it.part_base + it.split) * G * REC;
   for (int idx = tid; idx < G * DH; idx += ATT_THREADS) {
     const int g = idx / DH, d = idx - g * DH;

@@ -196,7 +196,6 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const AttnItem it = p.items[blockIdx.x];
-  const hb_seg sg = p.segs[it.seg];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, Hq = p.Hq, hk = it.kv_head;
   const int n_tiles = (it.key1 + BN - 1) / BN;           // key0 is 0 for chunk items
@@ -215,7 +214,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   // page ids are checked once here; the producer reads them from global memory as it goes
   int bad = 0;
   for (int i = tid; i < n_blk; i += TC_THREADS) {
-    const int pg = (i < sg.pt_len) ? p.pages[sg.pt_start + i] : -1;
+    const int pg = (i < it.pt_len) ? p.pages[it.pt_start + i] : -1;
     bad |= (pg < 0 || pg >= p.n_pages);
   }
   if (__syncthreads_or(bad)) {
@@ -240,7 +239,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         const int kb = j * BN;
 #pragma unroll
         for (int pi = 0; pi < BN / 16; ++pi)
-          ids[pi] = (kb + pi * 16 < it.key1) ? __ldg(p.pages + sg.pt_start + kb / 16 + pi) : 0;
+          ids[pi] = (kb + pi * 16 < it.key1) ? __ldg(p.pages + it.pt_start + kb / 16 + pi) : 0;
       };
       int nxt[BN / 16];
       load_ids(0, nxt);
@@ -316,7 +315,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     const int rr = quarter * 32 + lane;                     // row of the tile = TMEM lane
     const bool row_valid = rr < it.n_rows;
     const int r = it.row0 + rr;
-    const int pos = row_valid ? sg.pos_start + r / G : -1;
+    const int pos = row_valid ? it.pos_start + r / G : -1;
     const uint32_t t_lane = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
     float m_used = -INFINITY, l = 0.0f;
     bool ok = true;
@@ -326,7 +325,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     };
     // this thread's query row -> TMEM (two fp16 per column), the A operand of every S MMA
     {
-      const int tok = sg.q_start + (row_valid ? r / G : 0), head = hk * G + (row_valid ? r % G : 0);
+      const int tok = it.q_start + (row_valid ? r / G : 0), head = hk * G + (row_valid ? r % G : 0);
       const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(tok) * Hq + head) * DH);
 #pragma unroll
       for (int c = 0; c < DH / 2; c += 32) {
@@ -431,7 +430,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     if (ok && n_tiles > 0 && wait_w(pv_done, static_cast<uint32_t>((n_tiles - 1) & 1))) {
       tc_fence_after();
       const float inv = (l > 0.0f) ? 1.0f / l : 0.0f;
-      const int tok = sg.q_start + (row_valid ? r / G : 0), head = hk * G + (row_valid ? r % G : 0);
+      const int tok = it.q_start + (row_valid ? r / G : 0), head = hk * G + (row_valid ? r % G : 0);
       __half* orow = p.out + (static_cast<size_t>(tok) * Hq + head) * DH;
 #pragma unroll 1
       for (int c = 0; c < DH; c += 32) {

@@ -31,7 +31,12 @@ struct AttnItem {
   int32_t split;      // split index, n_splits
   int32_t n_splits;
   int32_t part_base;  // first partial-result record of this (seg, kv_head)
-  int32_t mode;       // 0 = chunk item (64 query rows, all keys), 1 = decode item (one split)
+  int32_t mode;       // 0 = chunk item (query-row tile, all keys), 1 = decode item (one split)
+  // copied from the segment so that a CTA needs one load to know its work
+  int32_t q_start;    // first token row of the segment
+  int32_t pos_start;  // tokens already cached when the segment starts
+  int32_t pt_start;   // offset of the request's page list inside the page-id array
+  int32_t pt_len;
   int32_t pad[2];
 };
 

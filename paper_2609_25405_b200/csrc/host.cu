@@ -14,7 +14,7 @@ namespace {
 constexpr int POOL_ROWS = 32;   // rows per pooling work item
 constexpr int ATT_TILE_ROWS = 64;   // query rows (tokens x grouped heads) per small chunk attention item
 constexpr int ATT_TC_ROWS = 128;    // query rows per tcgen05 chunk attention item
-constexpr int ATT_SPLIT_KEYS = 512; // keys per decode attention item; depends on nothing but this constant
+constexpr int ATT_SPLIT_KEYS = 1024; // keys per decode attention item; depends on nothing but this constant
 constexpr int N_STAGING = 4;    // pinned descriptor staging ring
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -562,6 +562,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
             it.key0 = sp * per;
             it.key1 = std::min(n_keys, it.key0 + per);
             it.split = sp; it.n_splits = ns; it.part_base = rec_at; it.mode = 1;
+            it.q_start = sg.q_start; it.pos_start = sg.pos_start; it.pt_start = sg.pt_start; it.pt_len = sg.pt_len;
             aitems.push_back(it);
           }
           rec_at += ns;
@@ -575,6 +576,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
             it.key0 = 0;
             it.key1 = sg.pos_start + (row0 + it.n_rows - 1) / G + 1;
             it.split = 0; it.n_splits = 1; it.part_base = 0; it.mode = 0;
+            it.q_start = sg.q_start; it.pos_start = sg.pos_start; it.pt_start = sg.pt_start; it.pt_len = sg.pt_len;
             if (it.n_rows <= ATT_TILE_ROWS) aitems.push_back(it);
             else titems.push_back(it);
           }
