@@ -53,9 +53,12 @@ enum {
  * request type"). */
 enum { HB_KIND_DECODE = 0, HB_KIND_PREFILL_CHUNK = 1, HB_KIND_EMBED_CHUNK = 2 };
 
-/* Pooling heads (Section 3.3): additive mean (Eq. 1-2 with w = 1) and the
- * positional last-token head. */
-enum { HB_POOL_NONE = 0, HB_POOL_MEAN = 1, HB_POOL_LAST = 2 };
+/* Pooling heads (Section 3.3).  Additive (Eq. 1-2): mean (w = 1) and weighted
+ * mean with w = 1-based position of the token in its request (the paper
+ * leaves the weights open; this is the common position weighting).
+ * Positional: last token (H of the last row of the final chunk) and CLS (H of
+ * the first row of the first chunk, retained in the slot). */
+enum { HB_POOL_NONE = 0, HB_POOL_MEAN = 1, HB_POOL_LAST = 2, HB_POOL_CLS = 3, HB_POOL_WMEAN = 4 };
 
 typedef struct hb_ctx hb_ctx;
 typedef struct hb_kv hb_kv;
@@ -275,11 +278,13 @@ HB_API int hb_gemm(hb_ctx* ctx, const void* A, const void* B, void* C, int32_t M
 /* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
  * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of
  * the chunk's rows, then
- *   mean: S <- S + sum_j rmsnorm(x_j) * gain, count <- count + n_rows
- *         (first_chunk != 0 starts from S = 0, count = 0);
- *   last: only the counters move until the final chunk;
- * and on the final chunk out_emb = L2-normalised S / count (mean) or the
- * normed last row (last).
+ *   mean / weighted mean: S <- S + sum_j w_j rmsnorm(x_j) * gain, count <-
+ *         count + n_rows (first_chunk != 0 starts from S = 0, count = 0; the
+ *         position weights continue from the slot's count);
+ *   last: only the counters move until the final chunk; cls: the first
+ *         chunk's first normed row is kept in S;
+ * and on the final chunk out_emb = L2-normalised S / W (W = count, or
+ * count (count + 1) / 2 for position weights) or the retained row.
  *   x          device float [n_rows, d_model] residual-stream rows of the chunk
  *   gain       device bf16 [d_model] final-norm gain
  *   slot_sum   device float [d_model], slot_meta device uint32 [4] =

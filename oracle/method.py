@@ -117,7 +117,9 @@ def embed_chunked(cfg, W, tokens, sizes, mode, dtype=np.float64):
     out = None
     for k, c in enumerate(sizes):
         H = chunk_forward(cfg, W, st, tokens[at:at + c], dtype)
-        out = pool_update(st, H, mode, is_final=(k == len(sizes) - 1))
+        # position weights w_{k,j} = 1-based position of row j of chunk k in the whole text
+        w = np.arange(at + 1, at + c + 1) if mode == "wmean" else None
+        out = pool_update(st, H, mode, is_final=(k == len(sizes) - 1), weights=w)
         at += c
     return out, st
 

@@ -130,12 +130,17 @@ def embed(cfg, W, tokens, mode, dtype=np.float64):
     """Single-pass embedding of the whole text.
 
     mode "mean": (1/n) sum_t Hhat_t  (Eq. 1-2 with w = 1 and one chunk);
-    mode "last": Hhat_{n-1}; mode "cls": Hhat_0 (positional heads, Section 3.3).
-    The pooled vector is L2-normalised.
+    mode "wmean": sum_t w_t Hhat_t / sum_t w_t with w_t = t + 1, the 1-based
+    position (Eq. 1-2; the paper leaves the weights open, this is the reading
+    taken); mode "last": Hhat_{n-1}; mode "cls": Hhat_0 (positional heads,
+    Section 3.3).  The pooled vector is L2-normalised.
     """
     hhat, _ = forward(cfg, W, tokens, logit_rows=[], dtype=dtype)
     if mode == "mean":
         e = np.sum(hhat, axis=0) / hhat.shape[0]
+    elif mode == "wmean":
+        w = np.arange(1, hhat.shape[0] + 1, dtype=hhat.dtype)
+        e = np.sum(w[:, None] * hhat, axis=0) / np.sum(w)
     elif mode == "last":
         e = hhat[-1]
     elif mode == "cls":

@@ -18,7 +18,7 @@ ERRORS = {0: "HB_OK", -1: "HB_ERR_BAD_ARG", -2: "HB_ERR_CUDA", -3: "HB_ERR_OOM_P
           -4: "HB_ERR_OOM_SLOTS", -5: "HB_ERR_TOO_LARGE", -6: "HB_ERR_BAD_DESC",
           -7: "HB_ERR_DEVICE_STATUS", -8: "HB_ERR_UNSUPPORTED"}
 from .consts import (KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK, POOL_NONE, POOL_MEAN,  # noqa: F401,E402
-                     POOL_LAST, EPI_F16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
+                     POOL_LAST, POOL_CLS, POOL_WMEAN, EPI_F16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
 
 
 class HbError(RuntimeError):

@@ -152,6 +152,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// 2^x on the special-function unit (-inf -> 0).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -353,22 +359,25 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(s_empty);
-      // scale, mask (only tiles that touch the diagonal or the end of the keys), row maximum
+      // row maximum of the raw scores; masking only on tiles that touch the diagonal or the end of the keys
       const bool need_mask = (key_base + BN - 1 > pos) || (key_base + BN > it.key1);
       float mx = -INFINITY;
+      if (!need_mask) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float v = __uint_as_float(sr[h][i]) * p.scale_log2;
-          if (need_mask) {
-            const int key = key_base + h * 32 + i;
-            if (key > pos || key >= it.key1) v = -INFINITY;
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[h][i]));
+      } else {
+        const int last = min(pos, it.key1 - 1) - key_base;   // last visible column of this row in the tile
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (h * 32 + i > last) sr[h][i] = 0xff800000u;   // -inf
+            mx = fmaxf(mx, __uint_as_float(sr[h][i]));
           }
-          sr[h][i] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
-        }
       }
+      mx *= p.scale_log2;   // scores enter the exponent as s * log2(e) / sqrt(Dh)
       const float m_new = fmaxf(m_used, mx);
       const bool grow = (m_new > m_used + 8.0f) || (m_used == -INFINITY && m_new > -INFINITY);
       // P_{j-1} V_{j-1} must have completed before O is rescaled or P is overwritten
@@ -391,8 +400,8 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         l *= f;
         if (grow) m_used = m_new;
       }
-      const float ms = (m_used == -INFINITY) ? 0.0f : m_used;
-      // probabilities -> fp16 P row in shared memory (K-major, 128-byte swizzle)
+      const float neg_ms = (m_used == -INFINITY) ? 0.0f : -m_used;
+      // probabilities p = 2^(s * scale - m) -> fp16 P row in shared memory (K-major, 128-byte swizzle)
       uint8_t* prow = smem + C::RING + rr * 128;
       float sum = 0.0f;
 #pragma unroll
@@ -401,8 +410,8 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int i = c * 8 + e * 2;
-          const float p0 = exp2f(__uint_as_float(sr[i >> 5][i & 31]) - ms);
-          const float p1 = exp2f(__uint_as_float(sr[(i + 1) >> 5][(i + 1) & 31]) - ms);
+          const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i >> 5][i & 31]), p.scale_log2, neg_ms));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(sr[(i + 1) >> 5][(i + 1) & 31]), p.scale_log2, neg_ms));
           sum += p0 + p1;
           pk[e] = pack_h2(p0, p1);
         }

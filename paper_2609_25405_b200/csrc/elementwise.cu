@@ -133,15 +133,7 @@ pool_chunk_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__
   sg.kind = HB_KIND_EMBED_CHUNK; sg.q_start = 0; sg.q_len = n_rows; sg.pos_start = first_chunk ? 0 : 1;
   sg.pt_start = 0; sg.pt_len = 0; sg.pool_slot = 0; sg.pool_mode = mode; sg.is_final = is_final;
   sg.logits_row = -1; sg.emb_row = 0; sg.reserved = 0;
-  PoolItem it;
-  it.seg = 0; it.block = blockIdx.x; it.n_blocks = gridDim.x; it.part_base = 0; it.pad[0] = it.pad[1] = 0;
-  if (mode == HB_POOL_MEAN) {
-    it.row0 = blockIdx.x * 32;
-    it.n_rows = min(32, n_rows - it.row0);
-  } else {
-    it.row0 = n_rows - 1;
-    it.n_rows = is_final ? 1 : 0;
-  }
+  const PoolItem it = pool_chunk_item(mode, 0, n_rows, first_chunk != 0, is_final != 0, blockIdx.x, gridDim.x);
   pool_block(it, sg, x, gain, part, counters, slot_sum, slot_meta, out_emb, d, eps, 1, status);
 }
 
@@ -237,7 +229,7 @@ int hb_launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s) 
 
 int hb_launch_pool_chunk(hb_ctx* c, const float* x, const void* gain, int n_rows, int mode, int first_chunk,
                          int is_final, float* slot_sum, uint32_t* slot_meta, float* out_emb, cudaStream_t s) {
-  const int blocks = (mode == HB_POOL_MEAN) ? (n_rows + 31) / 32 : 1;
+  const int blocks = (mode == HB_POOL_MEAN || mode == HB_POOL_WMEAN) ? (n_rows + 31) / 32 : 1;
   pool_chunk_kernel<<<blocks, NORM_THREADS, 0, s>>>(x, static_cast<const __nv_bfloat16*>(gain), n_rows, mode,
                                                     first_chunk, is_final, c->pool_part, c->counters, slot_sum,
                                                     slot_meta, out_emb, c->cfg.d_model, c->cfg.rms_eps, c->status);

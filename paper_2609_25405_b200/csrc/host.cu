@@ -131,7 +131,7 @@ int validate(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_
     }
     const bool embed = (s.kind == HB_KIND_EMBED_CHUNK);
     if (embed) {
-      if (s.pool_mode != HB_POOL_MEAN && s.pool_mode != HB_POOL_LAST) return HB_ERR_BAD_DESC;
+      if (s.pool_mode < HB_POOL_MEAN || s.pool_mode > HB_POOL_WMEAN) return HB_ERR_BAD_DESC;
       if (s.pool_slot < 0 || s.pool_slot >= n_slots || slot_used[s.pool_slot]) return HB_ERR_BAD_DESC;
       slot_used[s.pool_slot] = 1;
       if (s.logits_row != -1) return HB_ERR_BAD_DESC;
@@ -514,7 +514,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     }
     if (sg.logits_row >= 0) lsrc[sg.logits_row] = sg.q_start + sg.q_len - 1;
     if (sg.kind == HB_KIND_EMBED_CHUNK) {
-      if (sg.pool_mode == HB_POOL_MEAN) {
+      if (sg.pool_mode == HB_POOL_MEAN || sg.pool_mode == HB_POOL_WMEAN) {
         const int32_t nb = (sg.q_len + POOL_ROWS - 1) / POOL_ROWS;
         for (int32_t b = 0; b < nb; ++b) {
           PoolItem it{};
@@ -527,11 +527,12 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
           pitems.push_back(it);
         }
         part_at += nb;
-      } else {  // last-token head: only the final chunk's last row is read
+      } else {  // positional heads: CLS reads the first row of the first chunk, last-token the last row of the final one
         PoolItem it{};
         it.seg = r;
-        it.row0 = sg.q_start + sg.q_len - 1;
-        it.n_rows = sg.is_final ? 1 : 0;
+        const bool cls = (sg.pool_mode == HB_POOL_CLS);
+        it.row0 = cls ? sg.q_start : sg.q_start + sg.q_len - 1;
+        it.n_rows = cls ? (sg.pos_start == 0 ? 1 : 0) : (sg.is_final ? 1 : 0);
         it.block = 0;
         it.n_blocks = 1;
         it.part_base = part_at;
@@ -747,7 +748,7 @@ int hb_weights_pack_f16(const void* src_bf16, void* dst_f16, size_t n_elems, voi
 int hb_pool_chunk(hb_ctx* c, const float* x, const void* gain, int32_t n_rows, int32_t mode, int32_t first_chunk,
                   int32_t is_final, float* slot_sum, uint32_t* slot_meta, float* out_emb, void* stream) {
   if (!c || !x || !gain || !slot_sum || !slot_meta || n_rows < 1) return HB_ERR_BAD_ARG;
-  if (mode != HB_POOL_MEAN && mode != HB_POOL_LAST) return HB_ERR_BAD_ARG;
+  if (mode < HB_POOL_MEAN || mode > HB_POOL_WMEAN) return HB_ERR_BAD_ARG;
   if (is_final && !out_emb) return HB_ERR_BAD_ARG;
   if (n_rows > c->max_tokens) return HB_ERR_TOO_LARGE;
   return hb_launch_pool_chunk(c, x, gain, n_rows, mode, first_chunk != 0, is_final != 0, slot_sum, slot_meta,

@@ -35,14 +35,37 @@ __device__ __forceinline__ void bf16x4_to_float4(uint2 raw, float4& o) {
   o = make_float4(fa.x, fa.y, fb.x, fb.y);
 }
 
-// Final RMSNorm fused with the incremental pooler.  One block per work item = a block of rows
-// of one embedding segment.  Phase 1: one warp per row, shuffle-reduced sum of squares.
-// Phase 2: each thread owns column vectors and adds x * rstd over the item's rows in row
-// order.  The block's partial sum goes to scratch; the block that arrives last for a segment
-// adds the partials in block order, applies the gain, and updates the slot:
-//   S <- S + partial, count <- count + q_len            (Eq. 1-2 with w = 1)
-// (a request's first chunk overwrites instead, i.e. S(0) = 0, W(0) = 0).  On the final chunk
-// it emits S / count (mean) or the normed last row (last-token head), L2-normalised.
+// Work item of the pooler for block `block` of `n_blocks` of one chunk.  Additive heads (mean,
+// weighted mean) take 32 rows per block; positional heads read one row (CLS: the first row of the
+// first chunk, last-token: the last row of the final chunk) or none.
+__device__ __forceinline__ PoolItem pool_chunk_item(int mode, int q_start, int n_rows, bool first_chunk, bool is_final,
+                                                    int block, int n_blocks) {
+  PoolItem it;
+  it.seg = 0; it.block = block; it.n_blocks = n_blocks; it.part_base = 0; it.pad[0] = it.pad[1] = 0;
+  if (mode == HB_POOL_MEAN || mode == HB_POOL_WMEAN) {
+    it.row0 = q_start + block * 32;
+    it.n_rows = min(32, n_rows - block * 32);
+  } else if (mode == HB_POOL_CLS) {
+    it.row0 = q_start;
+    it.n_rows = first_chunk ? 1 : 0;
+  } else {
+    it.row0 = q_start + n_rows - 1;
+    it.n_rows = is_final ? 1 : 0;
+  }
+  return it;
+}
+
+// Final RMSNorm fused with the incremental pooler (Section 3.3).  One block per work item = a block
+// of rows of one embedding segment.  Phase 1: one warp per row, shuffle-reduced sum of squares.
+// Phase 2: each thread owns column vectors and adds w_j * x_j * rstd_j over the item's rows in row
+// order.  The block's partial sum goes to scratch; the block that arrives last for a segment adds
+// the partials in block order, applies the gain, and updates the slot:
+//   S <- S + sum_j w_j H_j,  W <- W + sum_j w_j                       (Eq. 1-2)
+// with w = 1 (mean) or w = position + 1 (weighted mean; W is then count (count + 1) / 2, so the
+// integer token count is the only counter kept).  A request's first chunk overwrites the slot
+// (S(0) = 0, W(0) = 0).  Positional heads keep one row: CLS stores the first row of the first chunk
+// in S, last-token reads the last row of the final chunk.  On the final chunk the block emits
+// S / W (or the retained row), L2-normalised.
 __device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg, const float* __restrict__ x,
                                            const __nv_bfloat16* __restrict__ gain, float* __restrict__ part,
                                            uint32_t* __restrict__ counters, float* __restrict__ pool_sum,
@@ -57,7 +80,14 @@ __device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg,
     if (threadIdx.x == 0) atomicOr(status, HB_DEV_POOL_BAD_INDEX);
     return;
   }
-  // phase 1: row statistics (item rows <= 32)
+  const bool first_chunk = (sg.pos_start == 0);
+  const bool additive = (sg.pool_mode == HB_POOL_MEAN || sg.pool_mode == HB_POOL_WMEAN);
+  const bool cls = (sg.pool_mode == HB_POOL_CLS);
+  float* S = pool_sum + static_cast<size_t>(sg.pool_slot) * d;
+  uint32_t* meta = pool_meta + static_cast<size_t>(sg.pool_slot) * 4;
+  // tokens pooled before this chunk = position of the chunk's first row (only the last block writes meta)
+  const uint32_t old_count = first_chunk ? 0u : meta[0];
+  // phase 1: row statistics (item rows <= 32), with the row's weight folded in
   for (int r = warp; r < it.n_rows; r += NORM_THREADS / 32) {
     const float* xrow = x + static_cast<size_t>(it.row0 + r) * d;
     float ss = 0.0f;
@@ -66,7 +96,12 @@ __device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg,
       ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
     }
     ss = warp_sum(ss);
-    if (lane == 0) rstd_s[r] = rsqrtf(ss / static_cast<float>(d) + eps);
+    if (lane == 0) {
+      const float w = (sg.pool_mode == HB_POOL_WMEAN)
+                          ? static_cast<float>(old_count + static_cast<uint32_t>(it.row0 + r - sg.q_start) + 1u)
+                          : 1.0f;
+      rstd_s[r] = rsqrtf(ss / static_cast<float>(d) + eps) * w;
+    }
   }
   __syncthreads();
   // phase 2: column sums over the item's rows, fixed row order
@@ -91,37 +126,41 @@ __device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg,
   if (!is_last_s) return;
   __threadfence();
   // segment tail: combine partials in block order, update the slot, maybe emit
-  const bool first_chunk = (sg.pos_start == 0);
-  float* S = pool_sum + static_cast<size_t>(sg.pool_slot) * d;
-  uint32_t* meta = pool_meta + static_cast<size_t>(sg.pool_slot) * 4;
-  const uint32_t old_count = first_chunk ? 0u : meta[0];
   const uint32_t old_chunks = first_chunk ? 0u : meta[1];
   const uint32_t new_count = old_count + static_cast<uint32_t>(sg.q_len);
-  const bool mean = (sg.pool_mode == HB_POOL_MEAN);
   const bool emit = (sg.is_final != 0);
+  const bool from_rows = additive || (cls && first_chunk) || (sg.pool_mode == HB_POOL_LAST && emit);
+  // total weight W: count for the mean, count (count + 1) / 2 for position weights
+  const double W = (sg.pool_mode == HB_POOL_WMEAN) ? 0.5 * static_cast<double>(new_count) * (new_count + 1.0)
+                                                   : static_cast<double>(new_count);
+  const float inv_W = static_cast<float>(1.0 / W);
   float4 e[MAX_VEC];
   float nrm = 0.0f;
 #pragma unroll
   for (int k = 0; k < MAX_VEC; ++k) {
     const int v = threadIdx.x + k * NORM_THREADS;
     e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (v < nv && (mean || emit)) {
+    if (v < nv && (from_rows || emit)) {
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int b = 0; b < it.n_blocks; ++b) {
-        const float4 p = __ldcg(reinterpret_cast<const float4*>(part + static_cast<size_t>(it.part_base + b) * d + 4 * v));
-        acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+      if (from_rows) {
+        for (int b = 0; b < it.n_blocks; ++b) {
+          const float4 p = __ldcg(reinterpret_cast<const float4*>(part + static_cast<size_t>(it.part_base + b) * d + 4 * v));
+          acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+        }
+        float4 g;
+        bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
+        acc.x *= g.x; acc.y *= g.y; acc.z *= g.z; acc.w *= g.w;
       }
-      float4 g;
-      bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
-      acc.x *= g.x; acc.y *= g.y; acc.z *= g.z; acc.w *= g.w;
-      if (mean) {
+      if (additive) {
         if (!first_chunk) {
           const float4 o = *reinterpret_cast<const float4*>(S + 4 * v);
           acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
         }
         *reinterpret_cast<float4*>(S + 4 * v) = acc;
-        const float inv = 1.0f / static_cast<float>(new_count);
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        acc.x *= inv_W; acc.y *= inv_W; acc.z *= inv_W; acc.w *= inv_W;
+      } else if (cls) {
+        if (first_chunk) *reinterpret_cast<float4*>(S + 4 * v) = acc;      // retain H_1 of the first chunk
+        else acc = *reinterpret_cast<const float4*>(S + 4 * v);
       }
       e[k] = acc;
       nrm += acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;

@@ -35,15 +35,7 @@ pool_chunk_static_kernel(float* __restrict__ scratch, const float* __restrict__ 
   sg.kind = HB_KIND_EMBED_CHUNK; sg.q_start = 0; sg.q_len = n_rows; sg.pos_start = first_chunk ? 0 : 1;
   sg.pt_start = 0; sg.pt_len = 0; sg.pool_slot = 0; sg.pool_mode = mode; sg.is_final = is_final;
   sg.logits_row = -1; sg.emb_row = 0; sg.reserved = 0;
-  PoolItem it;
-  it.seg = 0; it.block = blockIdx.x; it.n_blocks = gridDim.x; it.part_base = 0; it.pad[0] = it.pad[1] = 0;
-  if (mode == HB_POOL_MEAN) {
-    it.row0 = blockIdx.x * 32;
-    it.n_rows = min(32, n_rows - it.row0);
-  } else {
-    it.row0 = n_rows - 1;
-    it.n_rows = is_final ? 1 : 0;
-  }
+  const PoolItem it = pool_chunk_item(mode, 0, n_rows, first_chunk != 0, is_final != 0, blockIdx.x, gridDim.x);
   pool_block(it, sg, x, gain, scratch, tail, slot_sum, slot_meta, out_emb, d, eps, 1, tail + 1);
 }
 
@@ -71,7 +63,7 @@ extern "C" int hb_pool_chunk_noalloc(const float* x, const void* gain, int32_t n
                                      int32_t mode, int32_t first_chunk, int32_t is_final, float* slot_sum,
                                      uint32_t* slot_meta, float* out_emb, void* stream) {
   if (!x || !gain || !slot_sum || !slot_meta || n_rows < 1 || d_model < 4 || (d_model & 3)) return HB_ERR_BAD_ARG;
-  if (mode != HB_POOL_MEAN && mode != HB_POOL_LAST) return HB_ERR_BAD_ARG;
+  if (mode < HB_POOL_MEAN || mode > HB_POOL_WMEAN) return HB_ERR_BAD_ARG;
   if (is_final && !out_emb) return HB_ERR_BAD_ARG;
   if (!(rms_eps >= 0.0f)) return HB_ERR_BAD_ARG;
   // beyond the fixed scratch: refuse, never truncate
@@ -82,7 +74,7 @@ extern "C" int hb_pool_chunk_noalloc(const float* x, const void* gain, int32_t n
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // the array keeps whatever the previous call left: the arrival counter and the status word must start at zero
   if (cudaMemsetAsync(scratch + PART_FLOATS, 0, TAIL_WORDS * sizeof(float), s) != cudaSuccess) return HB_ERR_CUDA;
-  const int blocks = (mode == HB_POOL_MEAN) ? (n_rows + 31) / 32 : 1;
+  const int blocks = (mode == HB_POOL_MEAN || mode == HB_POOL_WMEAN) ? (n_rows + 31) / 32 : 1;
   pool_chunk_static_kernel<<<blocks, NORM_THREADS, 0, s>>>(scratch, x, static_cast<const __nv_bfloat16*>(gain), n_rows,
                                                            mode, first_chunk != 0, is_final != 0, slot_sum, slot_meta,
                                                            out_emb, d_model, rms_eps);

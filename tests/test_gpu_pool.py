@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("d", [256, 2048, 4096])
-@pytest.mark.parametrize("mode", ["mean", "last"])
+@pytest.mark.parametrize("mode", ["mean", "last", "cls", "wmean"])
 def test_pool_chunks_match_oracle(d, mode):
     from paper_2609_25405_b200 import binding as B
     shape = synth.ModelShape("pool", 1, d, d // 64, d // 64, 64, 64, 64)
@@ -25,19 +25,24 @@ def test_pool_chunks_match_oracle(d, mode):
     slot_meta = torch.full((4,), 12345, dtype=torch.int32, device="cuda")
     out = torch.zeros(d, device="cuda")
     st = M.RequestState(shape)
-    code = B.POOL_MEAN if mode == "mean" else B.POOL_LAST
+    code = {"mean": B.POOL_MEAN, "last": B.POOL_LAST, "cls": B.POOL_CLS, "wmean": B.POOL_WMEAN}[mode]
+    at = 0
     for k, n in enumerate(sizes):
         x = (3.0 * rng.standard_normal((n, d), dtype=np.float32)).astype(np.float32)
         H = T.rmsnorm(x.astype(np.float64), gain_f.astype(np.float64), shape.rms_eps)
         final = (k == len(sizes) - 1)
-        ref = M.pool_update(st, H, mode, final)
+        ref = M.pool_update(st, H, mode, final, weights=np.arange(at + 1, at + n + 1) if mode == "wmean" else None)
+        at += n
         ctx.pool_chunk(torch.from_numpy(x).cuda(), gain, n, code, k == 0, final, slot_sum, slot_meta, out)
         torch.cuda.synchronize()
         meta = slot_meta.cpu().numpy()
         assert list(meta) == [st.count, st.chunks, code, 1 if final else 0]
-        if mode == "mean":
+        if mode in ("mean", "wmean"):
             S = slot_sum.cpu().numpy().astype(np.float64)
-            assert np.max(np.abs(S - st.S)) <= 1e-5 * np.sqrt(st.count) * 4 + 1e-6 * np.max(np.abs(st.S))
+            assert np.max(np.abs(S - st.S)) <= 1e-5 * np.sqrt(st.count) * 4 + 2e-6 * np.max(np.abs(st.S))
+        if mode == "cls":
+            S = slot_sum.cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(S - st.retained)) <= 1e-5
     got = out.cpu().numpy().astype(np.float64)
     assert float(got @ ref) >= 1 - 1e-6 and np.max(np.abs(got - ref)) <= 1e-5
     assert ctx.status_poll() == 0

@@ -47,7 +47,7 @@ def run_cfg1(weights, wl, pool_mode="mean", chunkings=None):
     from paper_2609_25405_b200.engine import Request
     W = weights[0]
     eng = _engine(weights)
-    mode = B.POOL_MEAN if pool_mode == "mean" else B.POOL_LAST
+    mode = {"mean": B.POOL_MEAN, "last": B.POOL_LAST, "cls": B.POOL_CLS, "wmean": B.POOL_WMEAN}[pool_mode]
     gens = [Request("gen", p) for p in wl.prompts]
     embs = [Request("embed", t, mode) for t in wl.embed_tokens]
     if chunkings is None:
@@ -155,7 +155,7 @@ def test_cfg1_mean_state_after_each_chunk(weights):
     eng.close()
 
 
-@pytest.mark.parametrize("mode", ["mean", "last"])
+@pytest.mark.parametrize("mode", ["mean", "last", "cls", "wmean"])
 def test_random_chunkings_and_chunk_size_one(weights, mode):
     """Any partition of the text gives the single-pass embedding (chunks straddle pages)."""
     wl = synth.cfg1_workload(seed=77, embed_lens=(53, 19))

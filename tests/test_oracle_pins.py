@@ -249,7 +249,7 @@ def _compositions(n):
         yield sizes
 
 
-@pytest.mark.parametrize("mode", ["mean", "last", "cls"])
+@pytest.mark.parametrize("mode", ["mean", "last", "cls", "wmean"])
 def test_invariant1_every_partition_equals_single_pass(mode):
     """Chunked execution with the incremental pooler equals the single-pass
     embedding for EVERY ordered partition of a 7-token text."""
@@ -291,6 +291,19 @@ def test_pool_state_closed_form_after_each_chunk():
         at += c
         assert st.count == at and st.W == float(at) and st.chunks == k + 1
         assert np.max(np.abs(st.S - hh[:at].sum(0))) < 1e-6
+
+
+def test_position_weighted_mean_closed_form():
+    """With w_t = t + 1 the total weight of n tokens is n (n + 1) / 2, and for hidden states that
+    grow linearly with the position, H_t = (t + 1) u, the pooled vector is (2n + 1) / 3 * u."""
+    n, u = 11, np.array([0.5, -2.0, 1.25])
+    H = np.arange(1, n + 1)[:, None] * u[None, :]
+    st = types.SimpleNamespace(S=np.zeros(3), W=0.0, count=0, chunks=0, retained=None)
+    M.pool_update(st, H[:4], "wmean", False, np.arange(1, 5))
+    e = M.pool_update(st, H[4:], "wmean", True, np.arange(5, n + 1))
+    assert st.W == n * (n + 1) / 2
+    pooled = (2 * n + 1) / 3.0 * u
+    assert np.allclose(e, pooled / np.linalg.norm(pooled), atol=1e-12)
 
 
 def test_weighted_mean_matches_direct_formula():
