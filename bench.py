@@ -27,6 +27,10 @@ if ROOT not in sys.path:
 METRIC = "mixed-batch tokens/s (decode+embed) on 1 B200 and % of roofline"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (read + write) per launch of the projection GEMM at the 7B shape, T = 4096, mean of the four
+# projections of a layer, from the ncu capture summarised in profiles/gemm_tcgen05_cfg3-7b_layers2.md
+# (QKV 128.4 MB, O 169.5 MB, gate/up 403.1 MB, down 736.2 MB; algorithmic 134 / 201 / 386 / 369 MB)
+NCU_GEMM_TRAFFIC_BYTES = {"7b": 359.3e6}
 
 
 def load_peaks():
@@ -178,6 +182,43 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------
+# config 5: synthetic iterative-retrieval trace, virtual-clock replay (1B shape)
+# ------------------------------------------------------------------------------------------
+
+def run_trace(args):
+    import torch
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200 import synth, trace
+    from paper_2609_25405_b200.engine import Engine
+    shape = synth.SHAPES["1b"]
+    n_sessions = args.sessions
+    sessions = trace.make_trace(shape.V, seed=1005, n_sessions=n_sessions)
+    budget, chunk = 4096, 256
+    max_pos = 2048 + 128 + 8
+    P = shape.page_size
+    n_pages = n_sessions * ((max_pos + P - 1) // P) + 64
+    weights = B.DeviceWeights.random_on_device(shape, seed=0)
+    eng = Engine(shape, weights, n_pages=n_pages, n_slots=n_sessions + 8, max_tokens=budget,
+                 max_segs=n_sessions + budget // 16 + 8, max_pos=max_pos)
+    t0 = time.perf_counter()
+    out = trace.replay(sessions, eng, budget, chunk)
+    wall = time.perf_counter() - t0
+    status = eng.ctx.status_poll()
+    line = {"metric": METRIC, "value": out["rows"] / out["busy_s"], "unit": UNIT, "n_gpus": 1, "steps": out["steps"],
+            "warmup": 0, "ms_per_step": 1e3 * out["busy_s"] / max(out["steps"], 1), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "cfg5-trace-1b", "shape": shape.name, "sessions": n_sessions,
+                       "arrival_rate_per_s": 20.0, "token_budget": budget, "chunk": chunk, "scheduler": "IBS",
+                       "clock": "virtual: advances by measured GPU time per step, jumps over idle gaps"},
+            "rows": out["rows"], "expected_rows": trace.trace_tokens(sessions),
+            "busy_s": out["busy_s"], "virtual_clock_s": out["clock_s"],
+            "tokens_per_s_over_clock": out["rows"] / out["clock_s"], "host_wall_s": wall,
+            "sessions_done": out["sessions_done"], "device_status": status}
+    print(json.dumps(line))
+    eng.close()
+
+
+# ------------------------------------------------------------------------------------------
 # the CUDA path
 # ------------------------------------------------------------------------------------------
 
@@ -192,6 +233,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-alias", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
+    ap.add_argument("--sessions", type=int, default=256, help="sessions of the cfg5-trace-1b workload")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -203,6 +245,10 @@ def main():
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200 import replicas, synth, workloads
     from paper_2609_25405_b200.engine import build_batch
+
+    if args.workload.startswith("cfg5-trace"):
+        run_trace(args)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -329,7 +375,8 @@ def main():
     peak_tf = peaks["bf16_tflops_sustained"]
     roofline = {"bound": "tensor", "kernel": "hb_gemm_tcgen05_kernel (QKV, O, gate/up, down projections)",
                 "achieved": ach_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": (ach_tf / peak_tf) if ach_tf else None, "traffic": None,
+                "frac": (ach_tf / peak_tf) if ach_tf else None,
+                "traffic": NCU_GEMM_TRAFFIC_BYTES.get(spec.shape) if (not args.layers and w["T"] == 4096) else None,
                 "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step)",
                 "frac_of_burst": (ach_tf / peaks["bf16_tflops"]) if ach_tf else None,
                 "launches": gemm_n, "flops_per_launch": gemm_flops_launch}

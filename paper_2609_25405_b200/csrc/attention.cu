@@ -33,7 +33,6 @@ struct AttnParams {
   KvGeom kv;
   int layer;
   const AttnItem* items;
-  const hb_seg* segs;
   const int32_t* pages;
   float* part;                // split records: [record][G][Dh + 2]
   uint32_t* counters;         // [seg * Hkv + kv_head]
@@ -510,7 +509,6 @@ int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, 
   p.kv = kv;
   p.layer = layer;
   p.items = c->dd.attn_items;
-  p.segs = c->dd.segs;
   p.pages = c->dd.pages;
   p.part = c->attn_part;
   p.counters = c->attn_counters;

@@ -30,7 +30,6 @@ struct TcParams {
   __half* out;                // [T, Hq*Dh]
   int n_pages, Hkv, Hq, G, layer;
   const AttnItem* items;
-  const hb_seg* segs;
   const int32_t* pages;
   uint32_t* status;
   float scale_log2;
@@ -506,7 +505,6 @@ int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_ma
   p.G = c->cfg.n_heads / c->cfg.n_kv_heads;
   p.layer = layer;
   p.items = c->dd.tc_items;
-  p.segs = c->dd.segs;
   p.pages = c->dd.pages;
   p.status = c->status;
   p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));

@@ -149,7 +149,6 @@ struct hb_ctx {
   // workspace carve-up (device)
   float* x;                 // [max_tokens, d] residual stream, fp32
   __half* h;                // [max_tokens, d] normed activations (fp16)
-  float* qkv;               // unused placeholder (the QKV epilogue writes q and the KV pages directly)
   __half* q;                // [max_tokens, Hq*Dh] rotated queries (fp16)
   __half* attn_out;         // [max_tokens, Hq*Dh] (fp16)
   __half* act;              // [max_tokens, F] (fp16)

@@ -44,7 +44,7 @@ struct Carve {
 };
 
 struct Layout {
-  size_t x, h, qkv, q, attn_out, act, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
+  size_t x, h, q, attn_out, act, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
       status, desc;
   size_t total, desc_cap, attn_part_floats, pool_part_floats;
   int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items;
@@ -55,14 +55,11 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   Carve cv;
   const size_t rows = align_up(static_cast<size_t>(max_tokens), 128);
   const size_t lrows = align_up(static_cast<size_t>(max_segs), 128);
-  const size_t n_qkv = static_cast<size_t>(c.n_heads + 2 * c.n_kv_heads) * c.head_dim;
   const size_t n_q = static_cast<size_t>(c.n_heads) * c.head_dim;
   L.rows_pad = static_cast<int32_t>(rows);
   L.logit_rows_pad = static_cast<int32_t>(lrows);
   L.x = cv.take(rows * c.d_model * 4);
   L.h = cv.take(rows * c.d_model * 2);
-  L.qkv = cv.take(256);   // the QKV projection no longer has an intermediate: its epilogue writes q and the pages
-  (void)n_qkv;
   L.q = cv.take(rows * n_q * 2);
   L.attn_out = cv.take(rows * n_q * 2);
   L.act = cv.take(rows * c.d_ffn * 2);
@@ -239,7 +236,6 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->ws_bytes = lay.total;
   c->x = reinterpret_cast<float*>(c->ws + lay.x);
   c->h = reinterpret_cast<__half*>(c->ws + lay.h);
-  c->qkv = reinterpret_cast<float*>(c->ws + lay.qkv);
   c->q = reinterpret_cast<__half*>(c->ws + lay.q);
   c->attn_out = reinterpret_cast<__half*>(c->ws + lay.attn_out);
   c->act = reinterpret_cast<__half*>(c->ws + lay.act);
