@@ -12,7 +12,13 @@ brute-forced on small shapes:
       S^(k) = S^(k-1) + sum_j w_{k,j} H_j^(k),   S^(0) = 0        (Eq. 1)
       W^(k) = W^(k-1) + sum_j w_{k,j},           W^(0) = 0        (Eq. 2)
   emitting S^(K)/W^(K) after the final chunk; mean pooling is w = 1; the
-  positional heads keep one row: CLS H_1^(1), last token H_{c_K}^(K);
+  positional heads keep one row: CLS H_1^(1), last token H_{c_K}^(K); a
+  head that needs all rows buffers A^(k) = [A^(k-1); H^(k)] and runs after
+  the final chunk (element-wise max is the example used);
+* with a shared backbone, rows of embedding requests carry a low-rank
+  adapter on every projection and rows of generation requests do not
+  (Section 2.1 "Parameter sharing", Section 5.1): taken here as the
+  unmerged two-branch product per request;
 * a decode token is a chunk of one row whose logits are wanted
   (Section 3.2: "decode tokens process exactly one token per request").
 
@@ -39,12 +45,27 @@ class RequestState:
         self.count = 0                             # integer token count (mean: equals W)
         self.chunks = 0
         self.retained = None
+        self.A = np.zeros((0, cfg.d), dtype=dtype)  # buffered heads: A^(0) is empty
 
 
-def chunk_forward(cfg, W, st, tokens, dtype=np.float64):
+def _proj(h, w, name, lora, l, dtype):
+    """One projection of this request's rows.  Base: h W^T.  With an adapter
+    (requests of the adapted type only) the low-rank branch is taken as two
+    thin products and added, never merged into W:
+        y = h W^T + (alpha / r) (h A^T) B^T."""
+    y = h @ w[name].astype(dtype).T
+    if lora is not None:
+        A, B = lora.factors(l, name)
+        y = y + lora.scale * ((h @ A.astype(dtype).T) @ B.astype(dtype).T)
+    return y
+
+
+def chunk_forward(cfg, W, st, tokens, dtype=np.float64, lora=None):
     """One iteration's rows of one request: c = len(tokens) new rows at
     positions st.n_cached .. st.n_cached+c-1.  Appends their K/V to the
-    request's lists and returns the final-normed hidden states H^(k) [c, d]."""
+    request's lists and returns the final-normed hidden states H^(k) [c, d].
+    `lora`: adapter factors applied to this request's rows (embedding
+    requests in the shared-backbone deployment), None for base-model rows."""
     tokens = np.asarray(tokens, dtype=np.int64)
     c = tokens.shape[0]
     p0 = st.n_cached
@@ -55,9 +76,9 @@ def chunk_forward(cfg, W, st, tokens, dtype=np.float64):
     for l in range(cfg.L):
         w = W.layer(l)
         h = rmsnorm(x, w["attn_norm"].astype(dtype), cfg.rms_eps)
-        q = apply_rope((h @ w["wq"].astype(dtype).T).reshape(c, cfg.Hq, cfg.Dh), cos, sin)
-        k = apply_rope((h @ w["wk"].astype(dtype).T).reshape(c, cfg.Hkv, cfg.Dh), cos, sin)
-        v = (h @ w["wv"].astype(dtype).T).reshape(c, cfg.Hkv, cfg.Dh)
+        q = apply_rope(_proj(h, w, "wq", lora, l, dtype).reshape(c, cfg.Hq, cfg.Dh), cos, sin)
+        k = apply_rope(_proj(h, w, "wk", lora, l, dtype).reshape(c, cfg.Hkv, cfg.Dh), cos, sin)
+        v = _proj(h, w, "wv", lora, l, dtype).reshape(c, cfg.Hkv, cfg.Dh)
         st.k[l] = np.concatenate([st.k[l], k], axis=0)
         st.v[l] = np.concatenate([st.v[l], v], axis=0)
         o = np.empty((c, cfg.Hq, cfg.Dh), dtype=dtype)
@@ -70,10 +91,10 @@ def chunk_forward(cfg, W, st, tokens, dtype=np.float64):
                 p = np.exp(s)
                 p = p / np.sum(p)
                 o[j, a, :] = p @ st.v[l][:n_vis, b, :]
-        x = x + o.reshape(c, cfg.Hq * cfg.Dh) @ w["wo"].astype(dtype).T
+        x = x + _proj(o.reshape(c, cfg.Hq * cfg.Dh), w, "wo", lora, l, dtype)
         h = rmsnorm(x, w["ffn_norm"].astype(dtype), cfg.rms_eps)
-        act = silu(h @ w["wg"].astype(dtype).T) * (h @ w["wu"].astype(dtype).T)
-        x = x + act @ w["wd"].astype(dtype).T
+        act = silu(_proj(h, w, "wg", lora, l, dtype)) * _proj(h, w, "wu", lora, l, dtype)
+        x = x + _proj(act, w, "wd", lora, l, dtype)
     st.n_cached = p0 + c
     return rmsnorm(x, np.asarray(W.final_norm).astype(dtype), cfg.rms_eps)
 
@@ -104,19 +125,24 @@ def pool_update(st, H, mode, is_final, weights=None):
             st.retained = H[0].copy()                          # H_1^(1)
         if is_final:
             return l2_normalise(st.retained)
+    elif mode == "max":
+        # buffered head: A^(k) = [A^(k-1); H^(k)], the head runs once over all n rows
+        st.A = np.concatenate([st.A, H], axis=0)
+        if is_final:
+            return l2_normalise(np.max(st.A, axis=0))
     else:
         raise ValueError(mode)
     return None
 
 
-def embed_chunked(cfg, W, tokens, sizes, mode, dtype=np.float64):
+def embed_chunked(cfg, W, tokens, sizes, mode, dtype=np.float64, lora=None):
     """Chunked embedding with incremental pooling: one chunk per iteration."""
     assert sum(sizes) == len(tokens) and all(c > 0 for c in sizes)
     st = RequestState(cfg, dtype)
     at = 0
     out = None
     for k, c in enumerate(sizes):
-        H = chunk_forward(cfg, W, st, tokens[at:at + c], dtype)
+        H = chunk_forward(cfg, W, st, tokens[at:at + c], dtype, lora)
         # position weights w_{k,j} = 1-based position of row j of chunk k in the whole text
         w = np.arange(at + 1, at + c + 1) if mode == "wmean" else None
         out = pool_update(st, H, mode, is_final=(k == len(sizes) - 1), weights=w)

@@ -121,6 +121,46 @@ def forward(cfg, W, tokens, logit_rows=None, dtype=np.float64, pos_offset=0,
     return hhat, logits
 
 
+class MergedLora:
+    """Weights of the adapted model in the plain definition: every adapted
+    projection W [out, in] becomes W + (alpha / r) B A with A [r, in] and
+    B [out, r] (a low-rank update of the shared backbone, Section 2.1
+    "Parameter sharing").  The embedding, the norm gains and the LM head are
+    shared unchanged.  `adapters.factors(l, name) -> (A, B)`, `adapters.scale`
+    = alpha / r.  Requests of the adapted type (embedding) run `forward` /
+    `embed` on this object; requests of the other type run them on the base
+    weights: that per-request choice is the whole of the row-type dependence.
+    """
+
+    TARGETS = ("wq", "wk", "wv", "wo", "wg", "wu", "wd")
+
+    def __init__(self, W, adapters, dtype=np.float64):
+        self.W, self.adapters, self.dtype = W, adapters, dtype
+        self._layers = {}
+
+    @property
+    def tok_emb(self):
+        return self.W.tok_emb
+
+    @property
+    def final_norm(self):
+        return self.W.final_norm
+
+    @property
+    def lm_head(self):
+        return self.W.lm_head
+
+    def layer(self, l):
+        if l not in self._layers:
+            w = dict(self.W.layer(l))
+            for name in self.TARGETS:
+                A, B = self.adapters.factors(l, name)
+                w[name] = (np.asarray(w[name]).astype(self.dtype)
+                           + self.adapters.scale * (B.astype(self.dtype) @ A.astype(self.dtype)))
+            self._layers[l] = w
+        return self._layers[l]
+
+
 def l2_normalise(e, eps=1e-12):
     """e / max(||e||_2, eps); the zero vector maps to zeros."""
     return e / max(float(np.sqrt(np.sum(e * e))), eps)
@@ -133,7 +173,10 @@ def embed(cfg, W, tokens, mode, dtype=np.float64):
     mode "wmean": sum_t w_t Hhat_t / sum_t w_t with w_t = t + 1, the 1-based
     position (Eq. 1-2; the paper leaves the weights open, this is the reading
     taken); mode "last": Hhat_{n-1}; mode "cls": Hhat_0 (positional heads,
-    Section 3.3).  The pooled vector is L2-normalised.
+    Section 3.3); mode "max": the element-wise maximum over all rows of Hhat, the
+    example taken here of an "arbitrary deterministic head" that needs every
+    row at once (Section 3.3, buffered heads).  The pooled vector is
+    L2-normalised.
     """
     hhat, _ = forward(cfg, W, tokens, logit_rows=[], dtype=dtype)
     if mode == "mean":
@@ -145,6 +188,8 @@ def embed(cfg, W, tokens, mode, dtype=np.float64):
         e = hhat[-1]
     elif mode == "cls":
         e = hhat[0]
+    elif mode == "max":
+        e = np.max(hhat, axis=0)
     else:
         raise ValueError(mode)
     return l2_normalise(e)

@@ -140,6 +140,45 @@ class Weights:
         return np.ones(self.shape.d, dtype=np.float32)
 
 
+
+LORA_TARGETS = ("wq", "wk", "wv", "wo", "wg", "wu", "wd")
+
+
+class LoraAdapters:
+    """Seeded random low-rank adapter factors for every projection of every layer (inputs only; how
+    they enter the forward pass is for each side to state).  For projection `name` of layer l with
+    weight [out, in]: A [rank, in] and B [out, rank], both N(0, std^2) rounded to bf16 and returned
+    as float32; `alpha` is the usual scaling numerator (the update is scaled by alpha / rank)."""
+
+    def __init__(self, shape: ModelShape, rank: int, seed: int = 7, std: float = 0.02, alpha=None):
+        assert 1 <= rank <= 64
+        self.shape, self.rank, self.seed, self.std = shape, int(rank), seed, std
+        self.alpha = float(2 * rank if alpha is None else alpha)
+        self._cache = {}
+
+    @property
+    def scale(self):
+        return self.alpha / self.rank
+
+    def _dims(self, name):
+        s = self.shape
+        return {"wq": (s.Hq * s.Dh, s.d), "wk": (s.Hkv * s.Dh, s.d), "wv": (s.Hkv * s.Dh, s.d),
+                "wo": (s.d, s.Hq * s.Dh), "wg": (s.F, s.d), "wu": (s.F, s.d), "wd": (s.d, s.F)}[name]
+
+    def factors(self, layer, name):
+        """(A [rank, in], B [out, rank]) of one projection."""
+        key = (layer, name)
+        if key not in self._cache:
+            out, inn = self._dims(name)
+            t = LORA_TARGETS.index(name)
+            rng = np.random.default_rng([self.seed, 1000 + layer, t])
+            a = rng.standard_normal((self.rank, inn), dtype=np.float32) * np.float32(self.std)
+            b = rng.standard_normal((out, self.rank), dtype=np.float32) * np.float32(self.std)
+            self._cache[key] = (bf16_bits_to_f32(f32_to_bf16_bits(a)).reshape(a.shape),
+                                bf16_bits_to_f32(f32_to_bf16_bits(b)).reshape(b.shape))
+        return self._cache[key]
+
+
 def token_ids(rng, n, V):
     """n token ids uniform in [0, V)."""
     return rng.integers(0, V, size=n, dtype=np.int64)

@@ -249,7 +249,7 @@ def _compositions(n):
         yield sizes
 
 
-@pytest.mark.parametrize("mode", ["mean", "last", "cls", "wmean"])
+@pytest.mark.parametrize("mode", ["mean", "last", "cls", "wmean", "max"])
 def test_invariant1_every_partition_equals_single_pass(mode):
     """Chunked execution with the incremental pooler equals the single-pass
     embedding for EVERY ordered partition of a 7-token text."""
@@ -314,6 +314,138 @@ def test_weighted_mean_matches_direct_formula():
     e = M.pool_update(st, H[4:], "wmean", True, w[4:])
     direct = (w[:, None] * H).sum(0) / w.sum()
     assert np.allclose(e, direct / np.linalg.norm(direct), atol=1e-12)
+
+
+def test_buffered_max_head_closed_form():
+    """Buffered head (Section 3.3): the buffer after chunk k holds the first c_1+..+c_k rows in order,
+    and the element-wise maximum of hand-written rows is known."""
+    H = np.array([[1.0, -5.0, 0.0], [-2.0, -1.0, 0.5], [0.5, -3.0, 4.0], [0.0, -9.0, -1.0]])
+    st = types.SimpleNamespace(S=np.zeros(3), W=0.0, count=0, chunks=0, retained=None, A=np.zeros((0, 3)))
+    assert M.pool_update(st, H[:1], "max", False) is None
+    assert M.pool_update(st, H[1:3], "max", False) is None
+    assert np.array_equal(st.A, H[:3])
+    e = M.pool_update(st, H[3:], "max", True)
+    assert np.array_equal(st.A, H) and (st.count, st.chunks) == (4, 3)
+    pooled = np.array([1.0, -1.0, 4.0])
+    assert np.allclose(e, pooled / np.sqrt(18.0), atol=1e-15)
+    # the single-pass form on a real forward: max over rows of the final hidden states
+    W = _w(MICRO, 4, std=0.2)
+    toks = synth.token_ids(np.random.default_rng(3), 9, MICRO.V)
+    hh, _ = T.forward(MICRO, W, toks, logit_rows=[])
+    m = hh.max(0)
+    assert np.allclose(T.embed(MICRO, W, toks, "max"), m / np.linalg.norm(m), atol=1e-14)
+
+
+# --------------------------------------------------------------------------
+# low-rank adapters on the shared backbone
+# --------------------------------------------------------------------------
+
+class _HandAdapters:
+    """Rank-1 factors written by hand for one projection; zero elsewhere."""
+    scale = 2.0
+
+    def __init__(self, shape, name, a, b):
+        self.shape, self.name, self.a, self.b = shape, name, np.asarray(a, float), np.asarray(b, float)
+        self._ref = synth.LoraAdapters(shape, 1)
+
+    def factors(self, l, name):
+        out, inn = self._ref._dims(name)
+        if name == self.name and l == 0:
+            return self.a.reshape(1, inn), self.b.reshape(out, 1)
+        return np.zeros((1, inn)), np.zeros((out, 1))
+
+
+def test_merged_adapter_rank1_by_hand():
+    """W + (alpha / r) B A for r = 1 is W + s b a^T: entry (i, j) grows by s b_i a_j.  On the
+    non-square key projection a transposed factor cannot even be formed."""
+    cfg = MICRO1                                   # d = 8, Hkv * Dh = 8, F = 8: use the gate [F, d]
+    W = _w(cfg, 1)
+    a = np.arange(1, cfg.d + 1) * 0.5              # [in]
+    b = np.array([1.0, -1.0, 2.0, 0.0, 0.0, 3.0, 0.0, -2.0])   # [out = F]
+    mw = T.MergedLora(W, _HandAdapters(cfg, "wg", a, b)).layer(0)
+    base = W.layer(0)
+    assert np.array_equal(mw["wq"], np.asarray(base["wq"], dtype=np.float64))     # zero factors change nothing
+    delta = mw["wg"] - base["wg"]
+    assert np.allclose(delta[2], 2.0 * 2.0 * a, atol=1e-12)      # row i = s b_i a
+    assert np.allclose(delta[:, 3], 2.0 * b * 2.0, atol=1e-12)   # column j = s a_j b, a_3 = 2.0
+    assert np.allclose(delta[3], 0.0) and np.allclose(delta[7, 0], 2.0 * -2.0 * 0.5)
+    shapes = {n: synth.LoraAdapters(MICRO, 3).factors(1, n) for n in synth.LORA_TARGETS}
+    assert shapes["wk"][0].shape == (3, MICRO.d) and shapes["wk"][1].shape == (MICRO.Hkv * MICRO.Dh, 3)
+    assert shapes["wd"][0].shape == (3, MICRO.F) and shapes["wd"][1].shape == (MICRO.d, 3)
+
+
+def test_zero_adapter_is_the_base_model():
+    cfg, W = MICRO, _w(MICRO, 4, std=0.2)
+    toks = synth.token_ids(np.random.default_rng(5), 9, cfg.V)
+    ad = synth.LoraAdapters(cfg, 4, std=0.0)
+    assert np.array_equal(T.embed(cfg, T.MergedLora(W, ad), toks, "mean"), T.embed(cfg, W, toks, "mean"))
+    e, _ = M.embed_chunked(cfg, W, toks, [4, 5], "mean", lora=ad)
+    e0, _ = M.embed_chunked(cfg, W, toks, [4, 5], "mean")
+    assert np.array_equal(e, e0)
+
+
+@pytest.mark.parametrize("rank", [1, 3, 8])
+def test_two_branch_adapter_equals_merged_weights(rank):
+    """The method's unmerged form, h W^T + s (h A^T) B^T on embedding rows, chunked, against the
+    plain definition: one pass with the merged matrices.  The adapter must change the result
+    (so the comparison is not vacuous) and a generation request must not see it."""
+    cfg, W = MICRO, _w(MICRO, 4, std=0.2)
+    ad = synth.LoraAdapters(cfg, rank, std=0.2)
+    toks = synth.token_ids(np.random.default_rng(6), 10, cfg.V)
+    for mode in ("mean", "last"):
+        ref = T.embed(cfg, T.MergedLora(W, ad), toks, mode)
+        base = T.embed(cfg, W, toks, mode)
+        assert np.max(np.abs(ref - base)) > 1e-2
+        for sizes in ([10], [3, 7], [1, 4, 5], [2] * 5):
+            e, _ = M.embed_chunked(cfg, W, toks, sizes, mode, lora=ad)
+            assert float(e @ ref) > 1 - 1e-9 and np.max(np.abs(e - ref)) < 1e-6, (mode, sizes)
+    _, lg = M.prefill_then_decode(cfg, W, toks, [4, 6], 3)
+    _, lg_ref = T.generate(cfg, W, toks, 3)
+    assert np.max(np.abs(lg - lg_ref)) < 1e-6
+
+
+def test_merged_adapter_forward_matches_torch_linear_pair():
+    """The adapted model assembled from torch library routines with the two-branch linear
+    (F.linear twice per projection), against the oracle's merged single pass."""
+    cfg, W = MICRO, _w(MICRO, 2, std=0.2)
+    ad = synth.LoraAdapters(cfg, 2, std=0.2)
+    toks = synth.token_ids(np.random.default_rng(9), 8, cfg.V)
+
+    class Two:
+        tok_emb, final_norm, lm_head = W.tok_emb, W.final_norm, W.lm_head
+
+        @staticmethod
+        def layer(l):
+            return W.layer(l)
+
+    F = torch.nn.functional
+    real_linear = F.linear
+    tt = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    state = {"l": 0, "i": 0}
+    order = ["wq", "wk", "wv", "wo", "wg", "wu", "wd"]
+
+    def lora_linear(x, w, *rest):
+        # the projections of a layer are called in a fixed order by _torch_forward; the LM head comes last
+        if state["l"] >= cfg.L:
+            return real_linear(x, w)
+        name = order[state["i"]]
+        A, B = ad.factors(state["l"], name)
+        y = real_linear(x, w) + ad.scale * real_linear(real_linear(x, tt(A)), tt(B))
+        state["i"] += 1
+        if state["i"] == len(order):
+            state["i"], state["l"] = 0, state["l"] + 1
+        return y
+
+    F.linear = lora_linear
+    try:
+        hh_t, _ = _torch_forward(cfg, Two, toks)
+    finally:
+        F.linear = real_linear
+    hh, _ = T.forward(cfg, T.MergedLora(W, ad), toks, logit_rows=[])
+    # the oracle holds cos/sin in fp32 precision, the torch assembly in fp64: same bound as the base pin
+    assert np.max(np.abs(hh - hh_t)) < 1e-6
+    hh_base, _ = T.forward(cfg, W, toks, logit_rows=[])
+    assert np.max(np.abs(hh - hh_base)) > 1e-2
 
 
 def test_invariant3_decode_after_prefill_equals_full_forward():
