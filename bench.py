@@ -206,7 +206,7 @@ def run_trace(args):
     status = eng.ctx.status_poll()
     line = {"metric": METRIC, "value": out["rows"] / out["busy_s"], "unit": UNIT, "n_gpus": 1, "steps": out["steps"],
             "warmup": 0, "ms_per_step": 1e3 * out["busy_s"] / max(out["steps"], 1), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
             "config": {"workload": "cfg5-trace-1b", "shape": shape.name, "sessions": n_sessions,
                        "arrival_rate_per_s": 20.0, "token_budget": budget, "chunk": chunk, "scheduler": "IBS",
                        "clock": "virtual: advances by measured GPU time per step, jumps over idle gaps"},
@@ -377,7 +377,8 @@ def main():
                 "achieved": ach_tf, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": (ach_tf / peak_tf) if ach_tf else None,
                 "traffic": NCU_GEMM_TRAFFIC_BYTES.get(spec.shape) if (not args.layers and w["T"] == 4096) else None,
-                "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step)",
+                "peak_kind": f"{peak_kind} cuBLAS bf16, sustained (kernel timed inside a long step); the kernel's "
+                             "fp16 operands have the same nominal tensor rate as bf16 (ratio 1)",
                 "frac_of_burst": (ach_tf / peaks["bf16_tflops"]) if ach_tf else None,
                 "launches": gemm_n, "flops_per_launch": gemm_flops_launch}
     step_ms = ms / K
@@ -395,9 +396,10 @@ def main():
     breakdown = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in prof.items()}
     line = {"metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "precision": "bf16 weights x fp16 activations / KV cache on the tensor cores, fp32 accumulation, "
-                         "fp32 residual stream, norms, softmax and pooling",
+            "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "precision": "bf16 random-init weights, repacked once to fp16; fp16 x fp16 operands (weights, "
+                         "activations, KV cache) on the tensor cores with fp32 accumulation; fp32 residual "
+                         "stream, norms, softmax and pooling",
             "config": {"workload": spec.name, "shape": shape.name, "tokens_per_step": w["T"],
                        "decode_rows": spec.n_decode, "chunk": spec.chunk, "token_budget": spec.budget,
                        "l2": "inputs larger than L2 (weights and KV pages are re-streamed every step)",

@@ -58,7 +58,7 @@ enum { HB_KIND_DECODE = 0, HB_KIND_PREFILL_CHUNK = 1, HB_KIND_EMBED_CHUNK = 2 };
  * leaves the weights open; this is the common position weighting).
  * Positional: last token (H of the last row of the final chunk) and CLS (H of
  * the first row of the first chunk, retained in the slot). */
-enum { HB_POOL_NONE = 0, HB_POOL_MEAN = 1, HB_POOL_LAST = 2, HB_POOL_CLS = 3, HB_POOL_WMEAN = 4 };
+enum { HB_POOL_NONE = 0, HB_POOL_MEAN = 1, HB_POOL_LAST = 2, HB_POOL_CLS = 3, HB_POOL_WMEAN = 4, HB_POOL_MAX = 5 };
 
 typedef struct hb_ctx hb_ctx;
 typedef struct hb_kv hb_kv;
@@ -194,6 +194,21 @@ HB_API int hb_pool_destroy(hb_pool* pool);
 HB_API int hb_pool_alloc_slot(hb_pool* pool, int32_t* out_slot);
 HB_API int hb_pool_free_slot(hb_pool* pool, int32_t slot);
 
+/* Row buffer for buffered heads (Section 3.3: a head that is neither additive
+ * nor positional keeps A(k) = [A(k-1); H(k)], every final hidden state of the
+ * request, at O(n d) memory, and runs after the final chunk).  Layout:
+ * float rows[n_slots][max_rows][d_model]; row p of a slot holds the final
+ * RMSNorm output of the request's token at position p.  The caller owns the
+ * memory (device, 256-byte aligned); attach it once, before the first step
+ * that uses HB_POOL_MAX.  HB_POOL_MAX is the buffered head built in: every
+ * chunk appends its rows, the final chunk emits the element-wise maximum over
+ * all n rows, L2-normalised.  After the final chunk the buffer holds all n
+ * rows, so a caller can run any other head over them itself.  A segment with
+ * pos_start + q_len > max_rows, or HB_POOL_MAX without an attached buffer, is
+ * HB_ERR_BAD_DESC.  max_rows in 1..cfg.max_pos.  Host only. */
+HB_API int hb_pool_row_buffer_bytes(const hb_model_cfg* cfg, int32_t n_slots, int32_t max_rows, size_t* out_bytes);
+HB_API int hb_pool_attach_row_buffer(hb_pool* pool, void* buf, size_t bytes, int32_t max_rows);
+
 /* ---- the step ------------------------------------------------------------- */
 
 /* Host-only validation of a descriptor against the limits (what hb_mixed_step
@@ -253,6 +268,15 @@ enum {
 };
 HB_API int hb_profile_enable(hb_ctx* ctx, int on);
 HB_API int hb_profile_read(hb_ctx* ctx, float* ms_by_class, int32_t* launches_by_class);
+
+/* Failure-path self-test.  Every wait inside the kernels (on an mbarrier fed by TMA, by the tensor
+ * cores or by another warp role) is bounded in time; when a bound expires the kernel raises a bit
+ * in the status word and returns normally.  This call launches a one-thread kernel that runs the
+ * same bounded wait on a barrier nothing arrives on, with a limit of limit_ms (1..1000)
+ * milliseconds, so that the path "wait expires -> status bit -> hb_status_poll returns
+ * HB_ERR_DEVICE_STATUS -> context still usable" can be exercised without faulting or hanging the
+ * GPU.  The status code it raises is 32. */
+HB_API int hb_selftest_wait_expiry(hb_ctx* ctx, uint32_t limit_ms, void* stream);
 
 /* Kernels launched by the last hb_mixed_step on this context. */
 HB_API int hb_last_launch_count(const hb_ctx* ctx, int32_t* out_count);

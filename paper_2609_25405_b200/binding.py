@@ -18,7 +18,7 @@ ERRORS = {0: "HB_OK", -1: "HB_ERR_BAD_ARG", -2: "HB_ERR_CUDA", -3: "HB_ERR_OOM_P
           -4: "HB_ERR_OOM_SLOTS", -5: "HB_ERR_TOO_LARGE", -6: "HB_ERR_BAD_DESC",
           -7: "HB_ERR_DEVICE_STATUS", -8: "HB_ERR_UNSUPPORTED"}
 from .consts import (KIND_DECODE, KIND_PREFILL_CHUNK, KIND_EMBED_CHUNK, POOL_NONE, POOL_MEAN,  # noqa: F401,E402
-                     POOL_LAST, POOL_CLS, POOL_WMEAN, EPI_F16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
+                     POOL_LAST, POOL_CLS, POOL_WMEAN, POOL_MAX, EPI_F16, EPI_F32, EPI_RESID_F32, EPI_SWIGLU, CLASSES)
 
 
 class HbError(RuntimeError):
@@ -79,6 +79,8 @@ _sig = {
     "hb_pool_destroy": [_P],
     "hb_pool_alloc_slot": [_P, C.POINTER(C.c_int32)],
     "hb_pool_free_slot": [_P, C.c_int32],
+    "hb_pool_row_buffer_bytes": [_P, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)],
+    "hb_pool_attach_row_buffer": [_P, _P, C.c_size_t, C.c_int32],
     "hb_validate_desc": [C.POINTER(ModelCfg), C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                          C.POINTER(BatchDesc)],
     "hb_mixed_step": [_P, C.POINTER(BatchDesc), C.POINTER(Weights), _P, _P, _P, _P, _P],
@@ -89,6 +91,7 @@ _sig = {
                               _P],
     "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
     "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
+    "hb_selftest_wait_expiry": [_P, C.c_uint32, _P],
     "hb_profile_enable": [_P, C.c_int],
     "hb_profile_read": [_P, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
     "hb_gemm": [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
@@ -293,6 +296,19 @@ class Pool:
         check(lib.hb_pool_create(C.byref(cfg), C.c_void_p(self.arena.data_ptr()), nbytes.value, n_slots,
                                  C.byref(self.handle)), "hb_pool_create")
 
+    def attach_row_buffer(self, max_rows, fill=None):
+        """Row buffer for buffered heads (POOL_MAX): [n_slots, max_rows, d] fp32, caller-owned."""
+        nbytes = C.c_size_t()
+        check(lib.hb_pool_row_buffer_bytes(C.byref(self.cfg), self.n_slots, max_rows, C.byref(nbytes)),
+              "hb_pool_row_buffer_bytes")
+        self.rows = torch.empty((self.n_slots, max_rows, self.cfg.d_model), dtype=torch.float32,
+                                device=self.arena.device)
+        if fill is not None:
+            self.rows.fill_(fill)
+        check(lib.hb_pool_attach_row_buffer(self.handle, C.c_void_p(self.rows.data_ptr()), nbytes.value, max_rows),
+              "hb_pool_attach_row_buffer")
+        return self.rows
+
     def sums(self):
         d = self.cfg.d_model
         return self.arena[: self.n_slots * d].view(torch.float32).view(self.n_slots, d)
@@ -390,6 +406,9 @@ class Context:
         n = (C.c_int32 * len(CLASSES))()
         check(lib.hb_profile_read(self.handle, ms, n), "hb_profile_read")
         return {CLASSES[i]: (float(ms[i]), int(n[i])) for i in range(len(CLASSES))}
+
+    def selftest_wait_expiry(self, limit_ms=20, stream=None):
+        check(lib.hb_selftest_wait_expiry(self.handle, limit_ms, _stream_ptr(stream)), "hb_selftest_wait_expiry")
 
     def last_launch_count(self):
         n = C.c_int32()

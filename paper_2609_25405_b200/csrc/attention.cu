@@ -19,6 +19,7 @@
 // accumulate), softmax in fp32 with exp2.  Split decisions depend on the request's own length only, so a
 // request's result does not depend on its batch mates.
 #include "hb_internal.h"
+#include "ptx.cuh"
 
 namespace {
 
@@ -26,6 +27,7 @@ constexpr int ATT_THREADS = 128;
 constexpr int TILE_KEYS = 64;
 constexpr int TILE_ROWS = 64;
 constexpr int STAGES = 3;
+constexpr uint64_t ATT_WAIT_NS = 1000000000ull;  // 1 s
 
 struct AttnParams {
   const __half* q;            // [T, Hq*Dh] fp16
@@ -40,78 +42,6 @@ struct AttnParams {
   int Hq, G;
   float scale_log2;           // log2(e) / sqrt(Dh)
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-  const int sz = valid ? 16 : 0;  // 0 source bytes: the 16 destination bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");  // may sleep ~2 us per try, no spinning
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait (1 s).  Returns false if it expired.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0u && global_ns() - t0 > 1000000000ull) return false;
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c_inner,
-                                            int c_outer) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
-      : "memory");
-}
-
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-
-__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __half2 v = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 // Byte offset of 16-byte chunk `c` of row `r` in a 64-row tile stored as [DH/64 halves][64 rows][64]
 // bf16 with the 128-byte swizzle TMA applies (chunk index XOR row mod 8 inside each 128-byte row).
@@ -202,10 +132,10 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
 #pragma unroll
     for (int kp = 0; kp < NT / 2; ++kp) {
       uint32_t a[4];
-      a[0] = pack2(s[kp * 2][0], s[kp * 2][1]);
-      a[1] = pack2(s[kp * 2][2], s[kp * 2][3]);
-      a[2] = pack2(s[kp * 2 + 1][0], s[kp * 2 + 1][1]);
-      a[3] = pack2(s[kp * 2 + 1][2], s[kp * 2 + 1][3]);
+      a[0] = pack_half2(s[kp * 2][0], s[kp * 2][1]);
+      a[1] = pack_half2(s[kp * 2][2], s[kp * 2][3]);
+      a[2] = pack_half2(s[kp * 2 + 1][0], s[kp * 2 + 1][1]);
+      a[3] = pack_half2(s[kp * 2 + 1][2], s[kp * 2 + 1][3]);
       const int key = kofs + kp * 16 + (j & 1) * 8 + rr;
 #pragma unroll
       for (int dp = 0; dp < DH / 16; ++dp) {
@@ -269,7 +199,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   int issued = 0, bad = 0;
   if (tid == 0) {
     for (int st = 0; st < STAGES; ++st) mbar_init(bar_s + 8u * st, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
     // the first tiles are requested right away, with page ids read straight from global memory, so
     // that their latency overlaps the rest of the set-up
     for (; issued < STAGES - 1 && issued < n_tiles && !bad; ++issued) {
@@ -305,7 +235,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   if (__syncthreads_or(bad)) {  // also publishes the barrier initialisation and the page ids
     if (tid == 0) {
       atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
-      for (int st = 0; st < issued; ++st) mbar_wait(bar_s + 8u * st, 0u);   // copies already requested must land
+      for (int st = 0; st < issued; ++st) mbar_wait(bar_s + 8u * st, 0u, nullptr, ATT_WAIT_NS);   // copies already requested must land
     }
     cp_async_wait<0>();
     __syncthreads();
@@ -338,7 +268,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   for (int kt = 0; kt < n_tiles; ++kt) {
     if (__syncthreads_or(failed)) { failed = 1; break; }   // everyone is done with tile kt - 1 (and Q landed)
     if (tid == 0 && kt > 0) {   // at kt = 0 the last stage still holds Q
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // stages were read / patched by generic accesses
+      fence_async_smem();  // stages were read / patched by generic accesses
       for (; issued < n_tiles && issued < kt + STAGES; ++issued) issue_tile(issued);
     }
     if (kt == 0) {
@@ -349,7 +279,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     }
     const uint32_t k_tile = kv_s + (kt % STAGES) * 2 * TILE_BYTES;
     const int key_base = it.key0 + kt * TILE_KEYS;
-    if (!mbar_wait(bar_s + 8u * (kt % STAGES), static_cast<uint32_t>((kt / STAGES) & 1))) failed = 1;
+    if (!mbar_wait(bar_s + 8u * (kt % STAGES), static_cast<uint32_t>((kt / STAGES) & 1), nullptr, ATT_WAIT_NS)) failed = 1;
     const int valid_rows = it.key1 - key_base;
     if (valid_rows < TILE_KEYS) {
       // rows past the last key hold stale bytes (rest of the last page, pages not requested): zero the
@@ -390,8 +320,8 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     uint8_t* stage = smem;  // the ring is idle now; this warp touches its own 16 rows of the first tile only
 #pragma unroll
     for (int dn = 0; dn < DH / 8; ++dn) {
-      const uint32_t va = pack2(oacc[dn][0] * inv_a, oacc[dn][1] * inv_a);
-      const uint32_t vb = pack2(oacc[dn][2] * inv_b, oacc[dn][3] * inv_b);
+      const uint32_t va = pack_half2(oacc[dn][0] * inv_a, oacc[dn][1] * inv_a);
+      const uint32_t vb = pack_half2(oacc[dn][2] * inv_b, oacc[dn][3] * inv_b);
       *reinterpret_cast<uint32_t*>(stage + tile_off<DH>(ra, dn) + (lane & 3) * 4) = va;
       *reinterpret_cast<uint32_t*>(stage + tile_off<DH>(rb, dn) + (lane & 3) * 4) = vb;
     }

@@ -17,6 +17,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises a status bit and leaves without
 // storing.  The work split depends on the segment's own lengths only.
 #include "hb_internal.h"
+#include "ptx.cuh"
 
 namespace {
 
@@ -34,133 +35,6 @@ struct TcParams {
   uint32_t* status;
   float scale_log2;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");  // may sleep ~2 us per try, no spinning
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait; false if it expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > WAIT_NS) {
-        *abort_flag = 1u;
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c_inner,
-                                            int c_outer) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
-      : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, 128-byte swizzle.  K-major operand: rows 128 B apart, 8-row groups
-// `sbo` bytes apart (lbo unused).  MN-major operand: `lbo` = distance between 64-element column
-// groups, `sbo` = distance between groups of 8 K-rows.
-__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
-  d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-// D fp32, A and B fp16; b_mn: B operand is MN-major (V: head dimension contiguous).
-__device__ __forceinline__ constexpr uint32_t make_idesc(int n, bool b_mn) {
-  return (1u << 4) | (0u << 7) | (0u << 10) | ((b_mn ? 1u : 0u) << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
-         (static_cast<uint32_t>(BM >> 4) << 24);
-}
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-// A operand from tensor memory (16-bit elements, two per 32-bit column), B from shared memory.
-__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// 2^x on the special-function unit (-inf -> 0).
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
-  __half2 v = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
 
 template <int DH>
 struct TcCfg {
@@ -214,7 +88,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     mbar_init(p_ready, 4);
     mbar_init(pv_done, 1);
     *abort_flag = 0u;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
   // page ids are checked once here; the producer reads them from global memory as it goes
   int bad = 0;
@@ -254,7 +128,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 #pragma unroll
         for (int pi = 0; pi < BN / 16; ++pi) cur[pi] = nxt[pi];
         if (j + 1 < n_tiles) load_ids(j + 1, nxt);
-        if (!mbar_wait(kv_empty(st), static_cast<uint32_t>(((j / C::STAGES) & 1) ^ 1), abort_flag)) break;
+        if (!mbar_wait(kv_empty(st), static_cast<uint32_t>(((j / C::STAGES) & 1) ^ 1), abort_flag, WAIT_NS)) break;
         const int kb = j * BN;
         const int n_pg = min(BN / 16, (it.key1 - kb + 15) / 16);
         const uint32_t k_dst = ring_s + st * 2 * C::KV_HALF;
@@ -273,15 +147,15 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc(BN, false);
-      constexpr uint32_t idesc_o = make_idesc(DH, true);
+      constexpr uint32_t idesc_s = make_idesc_f16(BM, BN, false);
+      constexpr uint32_t idesc_o = make_idesc_f16(BM, DH, true);
       // S_j = Q K_j^T: Q comes from TMEM (written once by the softmax warps), K from shared memory: the
       // 8-key groups of the four page blocks of a tile are GROUP_BYTES apart, so one descriptor spans
       // all 64 keys.
       auto issue_s = [&](int j) -> bool {
         const int st = j % C::STAGES;
-        if (!mbar_wait(kv_full(st), static_cast<uint32_t>((j / C::STAGES) & 1), abort_flag)) return false;
-        if (!mbar_wait(s_empty, static_cast<uint32_t>((j & 1) ^ 1), abort_flag)) return false;
+        if (!mbar_wait(kv_full(st), static_cast<uint32_t>((j / C::STAGES) & 1), abort_flag, WAIT_NS)) return false;
+        if (!mbar_wait(s_empty, static_cast<uint32_t>((j & 1) ^ 1), abort_flag, WAIT_NS)) return false;
         tc_fence_after();
         const uint32_t k_tile = ring_s + st * 2 * C::KV_HALF;
 #pragma unroll
@@ -293,13 +167,13 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         umma_commit(s_full);
         return true;
       };
-      bool ok = mbar_wait(q_ready, 0u, abort_flag);
+      bool ok = mbar_wait(q_ready, 0u, abort_flag, WAIT_NS);
       if (ok) ok = issue_s(0);
       for (int j = 0; ok && j < n_tiles; ++j) {
         // S_{j+1} may start as soon as the softmax warps have read S_j out of TMEM
         if (j + 1 < n_tiles) ok = issue_s(j + 1);
         if (!ok) break;
-        if (!mbar_wait(p_ready, static_cast<uint32_t>(j & 1), abort_flag)) break;
+        if (!mbar_wait(p_ready, static_cast<uint32_t>(j & 1), abort_flag, WAIT_NS)) break;
         tc_fence_after();
         const uint32_t kv_tile = ring_s + (j % C::STAGES) * 2 * C::KV_HALF;
 #pragma unroll
@@ -307,7 +181,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
           const uint64_t ad = make_desc(p_s + ks * 32, 16, 1024);
           // V is the MN-major B operand: 64-column halves 1024 B apart, 8-key groups GROUP_BYTES apart
           const uint64_t bd = make_desc(kv_tile + ks * C::PAGE_BYTES + C::V_OFF, 1024, C::GROUP_BYTES);
-          umma(tmem + static_cast<uint32_t>(C::O_COL), ad, bd, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+          umma_ss(tmem + static_cast<uint32_t>(C::O_COL), ad, bd, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(kv_empty(j % C::STAGES));
         umma_commit(pv_done);
@@ -326,7 +200,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     bool ok = true;
     // the lanes of a warp leave the loop together (warp-wide votes and tcgen05.ld/st follow)
     auto wait_w = [&](uint32_t bar, uint32_t parity) {
-      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag)) != 0;
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, WAIT_NS)) != 0;
     };
     // this thread's query row -> TMEM (two fp16 per column), the A operand of every S MMA
     {
@@ -412,7 +286,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
           const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i >> 5][i & 31]), p.scale_log2, neg_ms));
           const float p1 = ex2_approx(fmaf(__uint_as_float(sr[(i + 1) >> 5][(i + 1) & 31]), p.scale_log2, neg_ms));
           sum += p0 + p1;
-          pk[e] = pack_h2(p0, p1);
+          pk[e] = pack_half2(p0, p1);
         }
         *reinterpret_cast<uint4*>(prow + ((c ^ (rr & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
@@ -449,10 +323,10 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             uint4 pk;
-            pk.x = pack_h2(__uint_as_float(o[v * 8 + 0]) * inv, __uint_as_float(o[v * 8 + 1]) * inv);
-            pk.y = pack_h2(__uint_as_float(o[v * 8 + 2]) * inv, __uint_as_float(o[v * 8 + 3]) * inv);
-            pk.z = pack_h2(__uint_as_float(o[v * 8 + 4]) * inv, __uint_as_float(o[v * 8 + 5]) * inv);
-            pk.w = pack_h2(__uint_as_float(o[v * 8 + 6]) * inv, __uint_as_float(o[v * 8 + 7]) * inv);
+            pk.x = pack_half2(__uint_as_float(o[v * 8 + 0]) * inv, __uint_as_float(o[v * 8 + 1]) * inv);
+            pk.y = pack_half2(__uint_as_float(o[v * 8 + 2]) * inv, __uint_as_float(o[v * 8 + 3]) * inv);
+            pk.z = pack_half2(__uint_as_float(o[v * 8 + 4]) * inv, __uint_as_float(o[v * 8 + 5]) * inv);
+            pk.w = pack_half2(__uint_as_float(o[v * 8 + 6]) * inv, __uint_as_float(o[v * 8 + 7]) * inv);
             *reinterpret_cast<uint4*>(orow + c + v * 8) = pk;
           }
         }

@@ -4,6 +4,7 @@
 // fixed order (no floating-point atomics), so results do not depend on what else is batched.
 #include "hb_internal.h"
 #include "pool_block.cuh"
+#include "ptx.cuh"
 
 namespace {
 
@@ -116,10 +117,12 @@ __global__ void __launch_bounds__(NORM_THREADS)
 final_pool_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
                   const PoolItem* __restrict__ items, const hb_seg* __restrict__ segs, float* __restrict__ part,
                   uint32_t* __restrict__ counters, float* __restrict__ pool_sum, uint32_t* __restrict__ pool_meta,
-                  float* __restrict__ out_emb, int d, float eps, int n_slots, uint32_t* status) {
+                  float* __restrict__ out_emb, int d, float eps, int n_slots, uint32_t* status,
+                  float* __restrict__ rowbuf, int rowbuf_rows) {
   const PoolItem it = items[blockIdx.x];
   const hb_seg sg = segs[it.seg];
-  pool_block(it, sg, x, gain, part, counters, pool_sum, pool_meta, out_emb, d, eps, n_slots, status);
+  pool_block(it, sg, x, gain, part, counters, pool_sum, pool_meta, out_emb, d, eps, n_slots, status, rowbuf,
+             rowbuf_rows);
 }
 
 // The pooler on its own: one chunk of one request, rows x[0 .. n_rows), slot 0 of a one-slot pool.
@@ -182,6 +185,18 @@ bf16_to_f16_kernel(const __nv_bfloat16* src, __half* dst, size_t n_vec, size_t n
     for (size_t i = n_vec * 8; i < n; ++i) dst[i] = __float2half_rn(sat_h(__bfloat162float(src[i])));
 }
 
+// Failure-path self-test: one thread waits, with the same bounded wait the pipelines use, on an
+// mbarrier that nothing ever arrives on.  The wait gives up after `limit_ns`, the kernel raises a
+// status bit and returns normally: no trap, no fault, the context stays usable.
+__global__ void wait_expiry_selftest_kernel(uint64_t limit_ns, uint32_t* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    mbar_init_fence();
+    if (!mbar_wait(smem_u32(&bar), 0u, nullptr, limit_ns)) atomicOr(status, HB_DEV_SELFTEST_WAIT_EXPIRED);
+  }
+}
+
 int check_launch() { return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA; }
 
 }  // namespace
@@ -200,7 +215,7 @@ int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s) {
 }
 
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta, int n_slots,
-                    float* out_emb, cudaStream_t s) {
+                    float* rowbuf, int rowbuf_rows, float* out_emb, cudaStream_t s) {
   const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(gain);
   if (c->dd.n_logit > 0) {
     final_logit_rows_kernel<<<c->dd.n_logit, NORM_THREADS, 0, s>>>(c->x, g, c->dd.logit_src, c->logit_in,
@@ -210,7 +225,7 @@ int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool
   if (c->dd.n_pool_items > 0) {
     final_pool_kernel<<<c->dd.n_pool_items, NORM_THREADS, 0, s>>>(
         c->x, g, c->dd.pool_items, c->dd.segs, c->pool_part, c->counters, pool_sum, pool_meta, out_emb,
-        c->cfg.d_model, c->cfg.rms_eps, n_slots, c->status);
+        c->cfg.d_model, c->cfg.rms_eps, n_slots, c->status, rowbuf, rowbuf_rows);
     if (check_launch() != HB_OK) return HB_ERR_CUDA;
   }
   return HB_OK;
@@ -233,6 +248,11 @@ int hb_launch_pool_chunk(hb_ctx* c, const float* x, const void* gain, int n_rows
   pool_chunk_kernel<<<blocks, NORM_THREADS, 0, s>>>(x, static_cast<const __nv_bfloat16*>(gain), n_rows, mode,
                                                     first_chunk, is_final, c->pool_part, c->counters, slot_sum,
                                                     slot_meta, out_emb, c->cfg.d_model, c->cfg.rms_eps, c->status);
+  return check_launch();
+}
+
+int hb_launch_wait_expiry_selftest(hb_ctx* c, uint64_t limit_ns, cudaStream_t s) {
+  wait_expiry_selftest_kernel<<<1, 32, 0, s>>>(limit_ns, c->status);
   return check_launch();
 }
 

@@ -22,6 +22,7 @@
 // Every mbarrier wait is bounded in time; on expiry the CTA raises a status bit, stops
 // issuing work, lets outstanding copies land, frees its TMEM and returns.
 #include "hb_internal.h"
+#include "ptx.cuh"
 
 namespace {
 
@@ -43,182 +44,6 @@ struct Tile {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(2000u)   // the thread may sleep up to ~2 us inside one try instead of spinning
-      : "memory");
-  return ok != 0;
-}
-
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false if the wait expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > WAIT_LIMIT_NS) {
-        *abort_flag = 1u;
-        return false;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int c_inner, int c_outer) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_load_2d_cg2(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                                int c_inner, int c_outer) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c_inner), "r"(c_outer)
-      : "memory");
-}
-
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-
-__device__ __forceinline__ void cluster_sync() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
-// The same shared-memory offset in the CTA of rank `rank` of this cluster.
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-
-__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
-}
-
-__device__ __forceinline__ void tcgen05_fence_before() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tcgen05_fence_after() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart,
-// 8-row groups 1024 B apart.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);        // start address
-  d |= static_cast<uint64_t>(1) << 16;                        // leading byte offset (unused with swizzle)
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;                // stride byte offset between 8-row groups
-  d |= static_cast<uint64_t>(1) << 46;                        // descriptor version (Blackwell)
-  d |= static_cast<uint64_t>(2) << 61;                        // 128-byte swizzle
-  return d;
-}
-
-// Instruction descriptor: D fp32 (bit 4), A and B fp16 (format 0 in bits 7-9 and 10-12),
-// both K-major, M = 128 * CG, N = BN.
-template <int BN, int CG>
-__device__ __forceinline__ constexpr uint32_t make_idesc() {
-  return (1u << 4) | (0u << 7) | (0u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
-         (static_cast<uint32_t>((BM * CG) >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
-                                          uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-__device__ __forceinline__ void umma_bf16_cg2(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
-                                              uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// Arrive (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs.
-__device__ __forceinline__ void umma_commit_cg2(uint32_t bar) {
-  const uint16_t mask = 3;
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(bar), "h"(mask)
-      : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Two floats -> packed fp16 pair, saturating at the largest finite half.
-__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
-  lo = fminf(fmaxf(lo, -65504.0f), 65504.0f);
-  hi = fminf(fmaxf(hi, -65504.0f), 65504.0f);
-  __half2 v = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
 
 // Store one thread's 32 consecutive accumulator columns of one row.
@@ -231,10 +56,10 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
     for (int v = 0; v < 4; ++v) {
       if (col0 + v * 8 < g.N) {
         uint4 pk;
-        pk.x = pack_f16(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-        pk.y = pack_f16(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-        pk.z = pack_f16(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-        pk.w = pack_f16(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+        pk.x = pack_half2_sat(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+        pk.y = pack_half2_sat(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+        pk.z = pack_half2_sat(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+        pk.w = pack_half2_sat(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
         *reinterpret_cast<uint4*>(out + v * 8) = pk;
       }
     }
@@ -265,7 +90,7 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
         for (int j = 0; j < 4; ++j) {
           const float g0 = __uint_as_float(r[v * 16 + j * 4 + 0]), u0 = __uint_as_float(r[v * 16 + j * 4 + 1]);
           const float g1 = __uint_as_float(r[v * 16 + j * 4 + 2]), u1 = __uint_as_float(r[v * 16 + j * 4 + 3]);
-          pk[j] = pack_f16(silu_f(g0) * u0, silu_f(g1) * u1);
+          pk[j] = pack_half2_sat(silu_f(g0) * u0, silu_f(g1) * u1);
         }
         *reinterpret_cast<uint4*>(out + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
@@ -303,7 +128,7 @@ __device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, in
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float a = __uint_as_float(r[v * 8 + e * 2]), b = __uint_as_float(r[v * 8 + e * 2 + 1]);
-        pk[v * 4 + e] = pack_f16(a * cc[e] - b * ss[e], b * cc[e] + a * ss[e]);
+        pk[v * 4 + e] = pack_half2_sat(a * cc[e] - b * ss[e], b * cc[e] + a * ss[e]);
       }
     }
     if (head < g.Hq) {
@@ -313,7 +138,7 @@ __device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, in
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < 16; ++j) pk[j] = pack_f16(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+    for (int j = 0; j < 16; ++j) pk[j] = pack_half2_sat(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
     dst = kv_slot_ptr(g, page, head - g.Hq - g.Hkv, 1, pos % g.P, off);
   }
 #pragma unroll
@@ -362,7 +187,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       mbar_init(tempty_bar(a), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
     }
     *abort_flag = 0u;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
   if (warp == 1) {
     if constexpr (CG == 2) {
@@ -377,10 +202,10 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
   }
-  tcgen05_fence_before();
+  tc_fence_before();
   __syncthreads();
   if constexpr (CG == 2) cluster_sync();  // the peer's barriers are initialised before anything signals them
-  tcgen05_fence_after();
+  tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   // Give up: raise the flag here and in the peer CTA so that every role of the group leaves its loop.
@@ -400,7 +225,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const int m0 = (tile % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
         const int n0 = (tile / m_tiles) * BN + static_cast<int>(rank) * T::B_ROWS;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; give_up(); break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
           const uint32_t a_dst = smem_base + stage * T::STAGE_BYTES;
           const uint32_t b_dst = a_dst + T::A_BYTES;
           if constexpr (CG == 2) {
@@ -425,28 +250,28 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   } else if (warp == 1) {
     // ---------------- MMA issuer (leader CTA only) ----------------
     if (lane == 0 && leader) {
-      constexpr uint32_t idesc = make_idesc<BN, CG>();
+      constexpr uint32_t idesc = make_idesc_f16(BM * CG, BN, false);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; give_up(); break; }
-        tcgen05_fence_after();
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
+        tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; give_up(); break; }
-          tcgen05_fence_after();
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
+          tc_fence_after();
           const uint32_t a_addr = smem_base + stage * T::STAGE_BYTES;
-          const uint64_t adesc = make_smem_desc(a_addr);
-          const uint64_t bdesc = make_smem_desc(a_addr + T::A_BYTES);
+          const uint64_t adesc = make_desc(a_addr, 16, 1024);
+          const uint64_t bdesc = make_desc(a_addr + T::A_BYTES, 16, 1024);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 elements along K inside the 128-byte swizzle row = +32 B = +2 in the address field
             const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
-            if constexpr (CG == 2) umma_bf16_cg2(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
-            else umma_bf16(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
+            if constexpr (CG == 2) umma_ss_cg2(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
+            else umma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
           }
           // the stage is free (in every CTA of the group) once these MMAs have read it
           if constexpr (CG == 2) umma_commit_cg2(empty_bar(stage));
@@ -469,8 +294,8 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
       const int m0 = (tile % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
       const int n0 = (tile / m_tiles) * BN;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; give_up(); break; }
-      tcgen05_fence_after();
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
+      tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(acc * BN);
       int pos = 0, page = 0;
@@ -489,12 +314,13 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       for (int c = 0; c < BN; c += 32) {
         uint32_t r[32];
         tmem_ld32(t_row + static_cast<uint32_t>(c), r);
+        tmem_ld_wait();
         if (row_ok && n0 + c < g.N) {
           if constexpr (EPI == HB_EPI_QKV_ROPE) epilogue_qkv_rope(g, row, n0 + c, r, pos, page);
           else epilogue_store<EPI>(g, row, n0 + c, r);
         }
       }
-      tcgen05_fence_before();
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) {
         if constexpr (CG == 2) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));
@@ -504,13 +330,13 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
   }
 
-  tcgen05_fence_before();
+  tc_fence_before();
   __syncthreads();
   // no CTA of a group leaves (or frees TMEM) while its peer may still read its shared memory or signal it
   if constexpr (CG == 2) cluster_sync();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(g.status, HB_DEV_GEMM_WAIT_EXPIRED);
   if (warp == 1) {
-    tcgen05_fence_after();
+    tc_fence_after();
     if constexpr (CG == 2)
       asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                    "r"(static_cast<uint32_t>(T::TMEM_COLS))

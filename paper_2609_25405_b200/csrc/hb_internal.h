@@ -18,6 +18,7 @@ enum : uint32_t {
   HB_DEV_APPEND_BAD_INDEX = 1u << 2,
   HB_DEV_POOL_BAD_INDEX = 1u << 3,
   HB_DEV_ATTN_WAIT_EXPIRED = 1u << 4,
+  HB_DEV_SELFTEST_WAIT_EXPIRED = 1u << 5,
 };
 
 // Attention work item: one (segment, kv head, row tile, key split).
@@ -91,6 +92,8 @@ struct hb_pool {
   int32_t n_slots;
   std::vector<uint8_t> used;
   int32_t n_free;
+  float* rowbuf = nullptr;    // buffered heads: [n_slots][rowbuf_rows][d] final hidden states, fp32
+  int32_t rowbuf_rows = 0;
 };
 
 // ---- GEMM -------------------------------------------------------------------
@@ -132,8 +135,9 @@ int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
 int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
 int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
-                    int n_slots, float* out_emb, cudaStream_t s);
+                    int n_slots, float* rowbuf, int rowbuf_rows, float* out_emb, cudaStream_t s);
 int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s);
+int hb_launch_wait_expiry_selftest(hb_ctx* c, uint64_t limit_ns, cudaStream_t s);
 int hb_launch_pool_chunk(hb_ctx* c, const float* x, const void* gain, int n_rows, int mode, int first_chunk,
                          int is_final, float* slot_sum, uint32_t* slot_meta, float* out_emb, cudaStream_t s);
 int hb_launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t s);

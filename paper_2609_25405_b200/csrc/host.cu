@@ -92,7 +92,7 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
 }
 
 int validate(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids, int32_t n_pages,
-             int32_t n_slots, const hb_batch_desc* d) {
+             int32_t n_slots, int32_t rowbuf_rows, const hb_batch_desc* d) {
   if (!d) return HB_ERR_BAD_ARG;
   if (d->n_tokens < 0 || d->n_segs < 0 || d->n_page_ids < 0 || d->n_logit_rows < 0 || d->n_emb_rows < 0)
     return HB_ERR_BAD_DESC;
@@ -128,7 +128,9 @@ int validate(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_
     }
     const bool embed = (s.kind == HB_KIND_EMBED_CHUNK);
     if (embed) {
-      if (s.pool_mode < HB_POOL_MEAN || s.pool_mode > HB_POOL_WMEAN) return HB_ERR_BAD_DESC;
+      if (s.pool_mode < HB_POOL_MEAN || s.pool_mode > HB_POOL_MAX) return HB_ERR_BAD_DESC;
+      // a buffered head keeps every row of the request: the whole text must fit the slot's row buffer
+      if (s.pool_mode == HB_POOL_MAX && s.pos_start + s.q_len > rowbuf_rows) return HB_ERR_BAD_DESC;
       if (s.pool_slot < 0 || s.pool_slot >= n_slots || slot_used[s.pool_slot]) return HB_ERR_BAD_DESC;
       slot_used[s.pool_slot] = 1;
       if (s.logits_row != -1) return HB_ERR_BAD_DESC;
@@ -423,6 +425,22 @@ int hb_pool_destroy(hb_pool* p) {
   return HB_OK;
 }
 
+int hb_pool_row_buffer_bytes(const hb_model_cfg* cfg, int32_t n_slots, int32_t max_rows, size_t* out_bytes) {
+  if (!cfg_ok(cfg) || n_slots < 1 || max_rows < 1 || max_rows > cfg->max_pos || !out_bytes) return HB_ERR_BAD_ARG;
+  *out_bytes = static_cast<size_t>(n_slots) * max_rows * cfg->d_model * 4;
+  return HB_OK;
+}
+
+int hb_pool_attach_row_buffer(hb_pool* p, void* buf, size_t bytes, int32_t max_rows) {
+  if (!p || !buf) return HB_ERR_BAD_ARG;
+  size_t need = 0;
+  if (hb_pool_row_buffer_bytes(&p->cfg, p->n_slots, max_rows, &need) != HB_OK) return HB_ERR_BAD_ARG;
+  if (bytes < need || (reinterpret_cast<uintptr_t>(buf) & 255u)) return HB_ERR_BAD_ARG;
+  p->rowbuf = static_cast<float*>(buf);
+  p->rowbuf_rows = max_rows;
+  return HB_OK;
+}
+
 int hb_pool_alloc_slot(hb_pool* p, int32_t* out_slot) {
   if (!p || !out_slot) return HB_ERR_BAD_ARG;
   if (p->n_free == 0) return HB_ERR_OOM_SLOTS;
@@ -448,7 +466,7 @@ int hb_pool_free_slot(hb_pool* p, int32_t slot) {
 int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids,
                      int32_t n_pages, int32_t n_slots, const hb_batch_desc* desc) {
   if (!cfg_ok(cfg)) return HB_ERR_BAD_ARG;
-  return validate(*cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, desc);
+  return validate(*cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, cfg->max_pos, desc);
 }
 
 int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv* kv, hb_pool* pool,
@@ -457,7 +475,8 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
   if (!kv->arena || !kv->has_map) return HB_ERR_BAD_ARG;
   if (memcmp(&kv->cfg, &c->cfg, sizeof(hb_model_cfg)) != 0) return HB_ERR_BAD_ARG;
   const int32_t n_slots = pool ? pool->n_slots : 0;
-  int rc = validate(c->cfg, c->max_tokens, c->max_segs, c->max_page_ids, kv->n_pages, n_slots, d);
+  int rc = validate(c->cfg, c->max_tokens, c->max_segs, c->max_page_ids, kv->n_pages, n_slots,
+                    pool ? pool->rowbuf_rows : 0, d);
   if (rc != HB_OK) return rc;
   if (d->n_logit_rows > 0 && (!out_logits || !w->lm_head)) return HB_ERR_BAD_ARG;
   if (d->n_emb_rows > 0 && !out_emb) return HB_ERR_BAD_ARG;
@@ -510,7 +529,7 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     }
     if (sg.logits_row >= 0) lsrc[sg.logits_row] = sg.q_start + sg.q_len - 1;
     if (sg.kind == HB_KIND_EMBED_CHUNK) {
-      if (sg.pool_mode == HB_POOL_MEAN || sg.pool_mode == HB_POOL_WMEAN) {
+      if (sg.pool_mode == HB_POOL_MEAN || sg.pool_mode == HB_POOL_WMEAN || sg.pool_mode == HB_POOL_MAX) {
         const int32_t nb = (sg.q_len + POOL_ROWS - 1) / POOL_ROWS;
         for (int32_t b = 0; b < nb; ++b) {
           PoolItem it{};
@@ -704,7 +723,8 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
                              : nullptr;
   {
     ProfRec* pr = prof_begin(HB_CLASS_POOL);
-    rc = hb_launch_final(c, w->final_norm, pool_sum, pool_meta, n_slots, out_emb, s);
+    rc = hb_launch_final(c, w->final_norm, pool_sum, pool_meta, n_slots, pool ? pool->rowbuf : nullptr,
+                         pool ? pool->rowbuf_rows : 0, out_emb, s);
     prof_end(pr);
     if (rc != HB_OK) return rc;
     launches += (dd.n_logit > 0) + (dd.n_pool_items > 0);
@@ -749,6 +769,11 @@ int hb_pool_chunk(hb_ctx* c, const float* x, const void* gain, int32_t n_rows, i
   if (n_rows > c->max_tokens) return HB_ERR_TOO_LARGE;
   return hb_launch_pool_chunk(c, x, gain, n_rows, mode, first_chunk != 0, is_final != 0, slot_sum, slot_meta,
                               out_emb, static_cast<cudaStream_t>(stream));
+}
+
+int hb_selftest_wait_expiry(hb_ctx* c, uint32_t limit_ms, void* stream) {
+  if (!c || limit_ms < 1 || limit_ms > 1000) return HB_ERR_BAD_ARG;
+  return hb_launch_wait_expiry_selftest(c, static_cast<uint64_t>(limit_ms) * 1000000ull, static_cast<cudaStream_t>(stream));
 }
 
 int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {

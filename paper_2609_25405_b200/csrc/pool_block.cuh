@@ -42,7 +42,7 @@ __device__ __forceinline__ PoolItem pool_chunk_item(int mode, int q_start, int n
                                                     int block, int n_blocks) {
   PoolItem it;
   it.seg = 0; it.block = block; it.n_blocks = n_blocks; it.part_base = 0; it.pad[0] = it.pad[1] = 0;
-  if (mode == HB_POOL_MEAN || mode == HB_POOL_WMEAN) {
+  if (mode == HB_POOL_MEAN || mode == HB_POOL_WMEAN || mode == HB_POOL_MAX) {
     it.row0 = q_start + block * 32;
     it.n_rows = min(32, n_rows - block * 32);
   } else if (mode == HB_POOL_CLS) {
@@ -53,6 +53,113 @@ __device__ __forceinline__ PoolItem pool_chunk_item(int mode, int q_start, int n
     it.n_rows = is_final ? 1 : 0;
   }
   return it;
+}
+
+// Buffered head (Section 3.3): a head that needs every row at once keeps A(k) = [A(k-1); H(k)], the
+// final hidden states of all rows seen so far, at O(n d) memory, and runs after the final chunk.
+// The head built in is the element-wise maximum over the n rows.  Every chunk appends its rows
+// (final RMSNorm applied, fp32) to the slot's row buffer at the rows' positions.  On the final chunk
+// the head runs over all n rows: block b of the chunk's n_blocks takes its own 32 rows straight from
+// the residual stream plus an equal share of the pos_start rows buffered by earlier steps, writes a
+// partial maximum, and the block that arrives last combines the partials, L2-normalises and emits.
+// The maximum is exact in any order, so the result does not depend on how the rows are shared out.
+__device__ __forceinline__ void pool_block_buffered(const PoolItem& it, const hb_seg& sg, const float* __restrict__ x,
+                                                    const __nv_bfloat16* __restrict__ gain, float* __restrict__ part,
+                                                    uint32_t* __restrict__ counters, uint32_t* __restrict__ meta,
+                                                    float* __restrict__ rowbuf, int rowbuf_rows,
+                                                    float* __restrict__ out_emb, int d, float eps, uint32_t* status) {
+  __shared__ float red_b[32];
+  __shared__ float rstd_b[32];
+  __shared__ uint32_t is_last_b;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nv = d >> 2;
+  if (rowbuf == nullptr || sg.pos_start + sg.q_len > rowbuf_rows) {
+    if (threadIdx.x == 0) atomicOr(status, HB_DEV_POOL_BAD_INDEX);
+    return;
+  }
+  const bool first_chunk = (sg.pos_start == 0);
+  const bool emit = (sg.is_final != 0);
+  float* A = rowbuf + static_cast<size_t>(sg.pool_slot) * rowbuf_rows * d;
+  for (int r = warp; r < it.n_rows; r += NORM_THREADS / 32) {
+    const float* xrow = x + static_cast<size_t>(it.row0 + r) * d;
+    float ss = 0.0f;
+    for (int v = lane; v < nv; v += 32) {
+      const float4 a = *reinterpret_cast<const float4*>(xrow + 4 * v);
+      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) rstd_b[r] = rsqrtf(ss / static_cast<float>(d) + eps);
+  }
+  __syncthreads();
+  // rows buffered by earlier steps that this block folds into its partial (final chunk only)
+  const int share = (sg.pos_start + it.n_blocks - 1) / it.n_blocks;
+  const int p0 = emit ? min(it.block * share, sg.pos_start) : 0;
+  const int p1 = emit ? min(p0 + share, sg.pos_start) : 0;
+  const int pos0 = sg.pos_start + (it.row0 - sg.q_start);     // position of the item's first row
+  float* my_part = part + static_cast<size_t>(it.part_base + it.block) * d;
+#pragma unroll 1
+  for (int v = threadIdx.x; v < nv; v += NORM_THREADS) {
+    float4 g;
+    bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
+    float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    for (int r = 0; r < it.n_rows; ++r) {
+      const float4 a = *reinterpret_cast<const float4*>(x + static_cast<size_t>(it.row0 + r) * d + 4 * v);
+      const float s = rstd_b[r];
+      const float4 hv = make_float4(a.x * s * g.x, a.y * s * g.y, a.z * s * g.z, a.w * s * g.w);
+      *reinterpret_cast<float4*>(A + static_cast<size_t>(pos0 + r) * d + 4 * v) = hv;
+      m.x = fmaxf(m.x, hv.x); m.y = fmaxf(m.y, hv.y); m.z = fmaxf(m.z, hv.z); m.w = fmaxf(m.w, hv.w);
+    }
+    for (int pr = p0; pr < p1; ++pr) {
+      const float4 hv = *reinterpret_cast<const float4*>(A + static_cast<size_t>(pr) * d + 4 * v);
+      m.x = fmaxf(m.x, hv.x); m.y = fmaxf(m.y, hv.y); m.z = fmaxf(m.z, hv.z); m.w = fmaxf(m.w, hv.w);
+    }
+    if (emit) *reinterpret_cast<float4*>(my_part + 4 * v) = m;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t prev = atomicAdd(counters + it.seg, 1u);
+    is_last_b = (prev + 1u == static_cast<uint32_t>(it.n_blocks)) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!is_last_b) return;
+  __threadfence();
+  const uint32_t old_count = first_chunk ? 0u : meta[0];
+  const uint32_t old_chunks = first_chunk ? 0u : meta[1];
+  if (emit) {
+    float4 e[MAX_VEC];
+    float nrm = 0.0f;
+#pragma unroll
+    for (int k = 0; k < MAX_VEC; ++k) {
+      const int v = threadIdx.x + k * NORM_THREADS;
+      e[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (v < nv) {
+        float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        for (int b = 0; b < it.n_blocks; ++b) {
+          const float4 q = __ldcg(reinterpret_cast<const float4*>(part + static_cast<size_t>(it.part_base + b) * d + 4 * v));
+          m.x = fmaxf(m.x, q.x); m.y = fmaxf(m.y, q.y); m.z = fmaxf(m.z, q.z); m.w = fmaxf(m.w, q.w);
+        }
+        e[k] = m;
+        nrm += m.x * m.x + m.y * m.y + m.z * m.z + m.w * m.w;
+      }
+    }
+    const float tot = block_sum(nrm, red_b);
+    const float inv = 1.0f / fmaxf(sqrtf(tot), 1e-12f);
+    float* o = out_emb + static_cast<size_t>(sg.emb_row) * d;
+#pragma unroll
+    for (int k = 0; k < MAX_VEC; ++k) {
+      const int v = threadIdx.x + k * NORM_THREADS;
+      if (v < nv)
+        *reinterpret_cast<float4*>(o + 4 * v) = make_float4(e[k].x * inv, e[k].y * inv, e[k].z * inv, e[k].w * inv);
+    }
+  }
+  if (threadIdx.x == 0) {
+    meta[0] = old_count + static_cast<uint32_t>(sg.q_len);
+    meta[1] = old_chunks + 1u;
+    meta[2] = static_cast<uint32_t>(sg.pool_mode);
+    meta[3] = emit ? 1u : 0u;
+    counters[it.seg] = 0u;
+  }
 }
 
 // Final RMSNorm fused with the incremental pooler (Section 3.3).  One block per work item = a block
@@ -70,7 +177,8 @@ __device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg,
                                            const __nv_bfloat16* __restrict__ gain, float* __restrict__ part,
                                            uint32_t* __restrict__ counters, float* __restrict__ pool_sum,
                                            uint32_t* __restrict__ pool_meta, float* __restrict__ out_emb, int d,
-                                           float eps, int n_slots, uint32_t* status) {
+                                           float eps, int n_slots, uint32_t* status, float* __restrict__ rowbuf = nullptr,
+                                           int rowbuf_rows = 0) {
   __shared__ float red[32];
   __shared__ float rstd_s[32];
   __shared__ uint32_t is_last_s;
@@ -78,6 +186,11 @@ __device__ __forceinline__ void pool_block(const PoolItem& it, const hb_seg& sg,
   const int nv = d >> 2;
   if (sg.pool_slot < 0 || sg.pool_slot >= n_slots) {
     if (threadIdx.x == 0) atomicOr(status, HB_DEV_POOL_BAD_INDEX);
+    return;
+  }
+  if (sg.pool_mode == HB_POOL_MAX) {
+    pool_block_buffered(it, sg, x, gain, part, counters, pool_meta + static_cast<size_t>(sg.pool_slot) * 4, rowbuf,
+                        rowbuf_rows, out_emb, d, eps, status);
     return;
   }
   const bool first_chunk = (sg.pos_start == 0);

@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
 TINY = synth.SHAPES["tiny"]
 KV_SENTINEL = 0x7F7F                                                # int16 fill pattern
 POOL_SENTINEL = 0x7FC12345                                          # a NaN bit pattern
+ROW_SENTINEL = 12345.0                                              # fill of the buffered heads' row buffer
 
 # tolerances (the benchmark spec): embeddings cosine >= 0.9995 and max-abs <= 2e-2;
 # logits max-abs <= 5e-2 and argmax agreement >= 99.5 %
@@ -171,6 +172,53 @@ def test_random_chunkings_and_chunk_size_one(weights, mode):
         eng.close()
 
 
+def test_buffered_max_head(weights):
+    """Buffered head (Section 3.3): every chunk appends its final hidden states to the slot's row
+    buffer; the final chunk emits the element-wise maximum over all rows.  Checked: the embedding
+    against the single-pass oracle for several partitions (one with a one-row final chunk, so a
+    single block folds in every buffered row), the buffered rows against the oracle's final hidden
+    states, rows past the text untouched, counters exact, and a request without a buffer rejected."""
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Request
+    W = weights[0]
+    rng = np.random.default_rng(21)
+    toks = synth.token_ids(rng, 150, TINY.V)
+    ref = T.embed(TINY, W, toks, "max")
+    hh, _ = T.forward(TINY, W, toks, logit_rows=[])
+    other = synth.token_ids(rng, 40, TINY.V)
+    for sizes in ([150], [70, 80], [33, 64, 52, 1], [1, 149]):
+        eng = _engine(weights, n_pages=96, max_tokens=512, max_pos=256)
+        rows = eng.pool.attach_row_buffer(160, fill=ROW_SENTINEL)
+        e = Request("embed", toks, B.POOL_MAX)
+        m = Request("embed", other, B.POOL_MEAN)            # shares the steps; must not disturb the buffer
+        er = {}
+        for k, c in enumerate(sizes):
+            work = [(e, c)] + ([(m, 40)] if k == 0 else [])
+            _, _, er = eng.step(work)
+            torch.cuda.synchronize()
+            meta = eng.pool.meta()[e.slot].cpu().numpy()
+            done = sum(sizes[:k + 1])
+            assert list(meta) == [done, k + 1, B.POOL_MAX, int(k == len(sizes) - 1)]
+        assert eng.ctx.status_poll() == 0
+        _check_emb(eng.out_emb[er[e]].cpu().numpy().astype(np.float64), ref)
+        buf = rows[e.slot].cpu().numpy()
+        assert np.max(np.abs(buf[:150] - hh)) <= 2e-2 * max(1.0, float(np.max(np.abs(hh))))
+        assert np.all(buf[150:] == ROW_SENTINEL)
+        assert np.all(rows[m.slot].cpu().numpy() == ROW_SENTINEL)
+        # the emitted vector is exactly the normalised maximum of what the buffer holds
+        mx = buf[:150].max(0).astype(np.float64)
+        assert np.max(np.abs(eng.out_emb[er[e]].cpu().numpy() - mx / np.linalg.norm(mx))) < 1e-6
+        eng.close()
+    eng = _engine(weights)
+    e = Request("embed", toks[:20], B.POOL_MAX)
+    with pytest.raises(B.HbError):
+        eng.step([(e, 20)])                                 # no row buffer attached
+    eng.pool.attach_row_buffer(16)
+    with pytest.raises(B.HbError):
+        eng.step([(e, 20)])                                 # text longer than the buffer's rows
+    eng.close()
+
+
 def test_long_chunks_take_the_tensor_core_attention_path(weights):
     """Chunks of more than 64 query rows run on the tcgen05 attention kernel (128-row tiles, ragged
     last tile, several key tiles, chunks that start inside a page); shorter remainders on the
@@ -257,6 +305,25 @@ def test_degenerate_batches(weights):
     torch.cuda.synchronize()
     _, ref = T.forward(TINY, W, [3, 9], logit_rows=[1])
     assert np.max(np.abs(eng.out_logits[lr[g]].cpu().numpy() - ref[0])) <= LOGIT_ABS
+    assert eng.ctx.status_poll() == 0
+    eng.close()
+
+
+def test_expired_wait_sets_status_and_context_stays_usable(weights):
+    """Failure detection without a fault: a bounded wait that runs out raises a status bit, the host
+    reads it as HB_ERR_DEVICE_STATUS, polling clears it, and the next step runs normally."""
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Request
+    W = weights[0]
+    eng = _engine(weights)
+    assert eng.ctx.status_poll() == 0
+    eng.ctx.selftest_wait_expiry(limit_ms=20)
+    assert eng.ctx.status_poll() == 32          # the self-test's bit; the poll clears the word
+    assert eng.ctx.status_poll() == 0
+    e = Request("embed", [5, 6, 7], B.POOL_MEAN)
+    _, _, er = eng.step([(e, 3)])
+    torch.cuda.synchronize()
+    _check_emb(eng.out_emb[er[e]].cpu().numpy().astype(np.float64), T.embed(TINY, W, [5, 6, 7], "mean"))
     assert eng.ctx.status_poll() == 0
     eng.close()
 

@@ -73,6 +73,22 @@ def test_slot_free_list():
     assert pool.alloc() == 0
 
 
+def test_row_buffer_size_and_argument_checks():
+    """Buffered heads keep O(n d) state: n_slots * max_rows * d floats, caller-owned."""
+    import ctypes as C
+    n = C.c_size_t()
+    assert B.lib.hb_pool_row_buffer_bytes(C.byref(CFG), 3, 100, C.byref(n)) == 0
+    assert n.value == 3 * 100 * TINY.d * 4
+    assert B.lib.hb_pool_row_buffer_bytes(C.byref(CFG), 3, 257, C.byref(n)) == -1      # more rows than max_pos
+    assert B.lib.hb_pool_row_buffer_bytes(C.byref(CFG), 0, 10, C.byref(n)) == -1
+    pool = B.Pool(CFG, 3, device=None)
+    fake = C.c_void_p(1 << 20)            # an aligned address that is only stored, never touched
+    assert B.lib.hb_pool_attach_row_buffer(pool.handle, None, 1 << 30, 100) == -1
+    assert B.lib.hb_pool_attach_row_buffer(pool.handle, fake, 3 * 100 * TINY.d * 4 - 1, 100) == -1
+    assert B.lib.hb_pool_attach_row_buffer(pool.handle, C.c_void_p((1 << 20) + 8), 1 << 30, 100) == -1
+    assert B.lib.hb_pool_attach_row_buffer(pool.handle, fake, 3 * 100 * TINY.d * 4, 100) == 0
+
+
 def _entries():
     return [
         dict(kind=B.KIND_EMBED_CHUNK, tokens=[1] * 20, pos_start=16, pages=[4, 5, 6], pool_slot=0,
