@@ -236,6 +236,52 @@ HB_API int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t
 HB_API int hb_mixed_step(hb_ctx* ctx, const hb_batch_desc* desc, const hb_weights* w, hb_kv* kv,
                   hb_pool* pool, float* out_logits, float* out_emb, void* stream);
 
+/* ---- low-rank adapters on embedding rows ------------------------------------
+ *
+ * With a shared backbone the embedding model is the generation model plus a
+ * low-rank adapter (Section 2.1 "Parameter sharing"; Section 5.1 runs both
+ * request types on one GPU "using LoRA adapters").  Inside the one forward
+ * pass, rows of EMBED_CHUNK segments compute every projection as
+ *     y = x W^T + (alpha / r) (x A^T) B^T,        A [r, in], B [out, r],
+ * and rows of DECODE / PREFILL_CHUNK segments compute y = x W^T.  The paper
+ * does not say which projections carry the adapter; here all seven of a layer
+ * do (q, k, v, o, gate, up, down).  Token embedding, norm gains and LM head
+ * are shared unchanged.
+ *
+ * Packed layout (device, fp16, row-major, 16-byte aligned; the caller packs
+ * once).  R(n) = n * r rounded up to a multiple of 64; unused rows / columns
+ * are zero.  Row orders of the B factors follow the fused weights they pair
+ * with (hb_layer_weights):
+ *   a_qkv  [R(3), d]          rows [0,r) = A_q, [r,2r) = A_k, [2r,3r) = A_v
+ *   b_qkv  [(Hq+2Hkv)Dh, R(3)] rows as wqkv (q and k rows pair-interleaved per
+ *                             head); q rows hold B_q in columns [0,r), k rows
+ *                             B_k in [r,2r), v rows B_v in [2r,3r), zero elsewhere
+ *   a_o    [R(1), Hq*Dh]      A_o;           b_o  [d, R(1)]   B_o
+ *   a_gu   [R(2), d]          A_gate, A_up;  b_gu [2F, R(2)]  rows as w_gate_up
+ *                             (gate_j, up_j interleaved): gate rows hold B_gate
+ *                             in [0,r), up rows B_up in [r,2r)
+ *   a_d    [R(1), F]          A_down;        b_d  [d, R(1)]   B_down
+ * scale = alpha / r multiplies the rank-r activations in fp32 before they are
+ * rounded to fp16.  rank in 1..64. */
+typedef struct hb_lora_layer {
+  const void *a_qkv, *b_qkv, *a_o, *b_o, *a_gu, *b_gu, *a_d, *b_d;
+} hb_lora_layer;
+
+typedef struct hb_lora {
+  int32_t rank;
+  float scale;
+  const hb_lora_layer* layers; /* host array [n_layers] */
+} hb_lora;
+
+/* hb_mixed_step with adapters on the EMBED_CHUNK rows.  lora == NULL, or a
+ * step without EMBED_CHUNK rows, is exactly hb_mixed_step.  Per layer this
+ * adds four thin GEMMs (the rank-r activations of the rows, zero for rows
+ * that carry no adapter) and extends the K loop of the four projection GEMMs
+ * by R / 64 blocks.  The context must have been created after
+ * hb_workspace_bytes (the workspace always includes the rank-r buffer). */
+HB_API int hb_mixed_step_lora(hb_ctx* ctx, const hb_batch_desc* desc, const hb_weights* w, const hb_lora* lora,
+                       hb_kv* kv, hb_pool* pool, float* out_logits, float* out_emb, void* stream);
+
 /* Repack bf16 values to fp16, element by element, on `stream` (device
  * pointers, 16-byte aligned; dst may equal src for an in-place repack, partial
  * overlap is rejected).  Exact for 2^-14 <= |w| <= 65504; smaller magnitudes
@@ -264,7 +310,8 @@ enum {
   HB_CLASS_POOL = 3,      /* final RMSNorm + pooler / logits-row preparation            */
   HB_CLASS_LM_HEAD = 4,   /* LM-head projection                                         */
   HB_CLASS_ATTENTION_TC = 5, /* chunk-row attention on the tcgen05 tensor cores         */
-  HB_N_CLASSES = 6
+  HB_CLASS_LORA = 6,      /* adapters: rank-r activations of the embedding rows         */
+  HB_N_CLASSES = 7
 };
 HB_API int hb_profile_enable(hb_ctx* ctx, int on);
 HB_API int hb_profile_read(hb_ctx* ctx, float* ms_by_class, int32_t* launches_by_class);

@@ -43,6 +43,14 @@ class Weights(C.Structure):
                 ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)]
 
 
+class LoraLayer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("a_qkv", "b_qkv", "a_o", "b_o", "a_gu", "b_gu", "a_d", "b_d")]
+
+
+class Lora(C.Structure):
+    _fields_ = [("rank", C.c_int32), ("scale", C.c_float), ("layers", C.POINTER(LoraLayer))]
+
+
 class Seg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("kind", "q_start", "q_len", "pos_start", "pt_start", "pt_len",
                                          "pool_slot", "pool_mode", "is_final", "logits_row", "emb_row",
@@ -84,6 +92,7 @@ _sig = {
     "hb_validate_desc": [C.POINTER(ModelCfg), C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                          C.POINTER(BatchDesc)],
     "hb_mixed_step": [_P, C.POINTER(BatchDesc), C.POINTER(Weights), _P, _P, _P, _P, _P],
+    "hb_mixed_step_lora": [_P, C.POINTER(BatchDesc), C.POINTER(Weights), C.POINTER(Lora), _P, _P, _P, _P, _P],
     "hb_weights_pack_f16": [_P, _P, C.c_size_t, _P],
     "hb_argmax": [_P, _P, C.c_int32, _P, _P],
     "hb_pool_chunk": [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P],
@@ -216,6 +225,109 @@ class DeviceWeights:
             lw.wo = rnd(shape.d, shape.Hq * shape.Dh)
             lw.w_gate_up = rnd(2 * shape.F, shape.d)
             lw.w_down = rnd(shape.d, shape.F)
+        return self
+
+
+def _pad64(n):
+    return (n + 63) // 64 * 64
+
+
+class DeviceLora:
+    """Adapter factors resident in HBM in the library's packed layout (fp16), plus the hb_lora
+    struct.  Packing is layout only: factors are stacked / placed in column blocks next to the fused
+    weights they pair with; the bf16 -> fp16 repack runs in the library."""
+
+    def __init__(self, n_layers, rank, scale):
+        self.tensors = []
+        self.layers = (LoraLayer * n_layers)()
+        self.struct = Lora(int(rank), float(scale), C.cast(self.layers, C.POINTER(LoraLayer)))
+        self.rank = int(rank)
+
+    def _keep(self, t):
+        self.tensors.append(t)
+        return t.data_ptr()
+
+    @staticmethod
+    def _stack_down(factors, R):
+        """A factors [r, in] stacked by rows into [R, in], zero padded."""
+        out = np.zeros((R, factors[0].shape[1]), dtype=np.float32)
+        at = 0
+        for a in factors:
+            out[at:at + a.shape[0]] = a
+            at += a.shape[0]
+        return out
+
+    @classmethod
+    def from_synth(cls, ad, device="cuda"):
+        """Upload synth.LoraAdapters."""
+        s, r = ad.shape, ad.rank
+        self = cls(s.L, r, ad.scale)
+        upw = lambda a: self._keep(pack_f16_(bf16_from_f32(a, device)))
+        R1, R2, R3 = 64, _pad64(2 * r), _pad64(3 * r)
+        for l in range(s.L):
+            f = {n: ad.factors(l, n) for n in ("wq", "wk", "wv", "wo", "wg", "wu", "wd")}
+            ll = self.layers[l]
+            ll.a_qkv = upw(self._stack_down([f["wq"][0], f["wk"][0], f["wv"][0]], R3))
+            nq, nk = s.Hq * s.Dh, s.Hkv * s.Dh
+            b = np.zeros((nq + 2 * nk, R3), dtype=np.float32)
+            b[:nq, 0:r] = rope_interleave_rows(f["wq"][1], s.Dh)
+            b[nq:nq + nk, r:2 * r] = rope_interleave_rows(f["wk"][1], s.Dh)
+            b[nq + nk:, 2 * r:3 * r] = f["wv"][1]
+            ll.b_qkv = upw(b)
+            ll.a_o = upw(self._stack_down([f["wo"][0]], R1))
+            b = np.zeros((s.d, R1), dtype=np.float32)
+            b[:, :r] = f["wo"][1]
+            ll.b_o = upw(b)
+            ll.a_gu = upw(self._stack_down([f["wg"][0], f["wu"][0]], R2))
+            b = np.zeros((2 * s.F, R2), dtype=np.float32)
+            b[0::2, 0:r] = f["wg"][1]
+            b[1::2, r:2 * r] = f["wu"][1]
+            ll.b_gu = upw(b)
+            ll.a_d = upw(self._stack_down([f["wd"][0]], R1))
+            b = np.zeros((s.d, R1), dtype=np.float32)
+            b[:, :r] = f["wd"][1]
+            ll.b_d = upw(b)
+        return self
+
+    @classmethod
+    def random_on_device(cls, shape, rank, seed=7, std=0.02, scale=2.0, device="cuda"):
+        """Random factors drawn on the device in the packed layout (benchmarks): the blocks that the
+        layout keeps at zero are zeroed after the draw."""
+        self = cls(shape.L, rank, scale)
+        g = torch.Generator(device=device)
+        g.manual_seed(seed)
+        r = rank
+        R1, R2, R3 = 64, _pad64(2 * r), _pad64(3 * r)
+        nq, nk = shape.Hq * shape.Dh, shape.Hkv * shape.Dh
+
+        def rnd(rows, cols):
+            t = torch.empty((rows, cols), dtype=torch.bfloat16, device=device)
+            t.normal_(0.0, std, generator=g)
+            return t
+
+        fin = lambda t: self._keep(pack_f16_(t.contiguous()))
+        for l in range(shape.L):
+            ll = self.layers[l]
+            a = rnd(R3, shape.d); a[3 * r:] = 0
+            ll.a_qkv = fin(a)
+            b = rnd(nq + 2 * nk, R3)
+            keep = torch.zeros_like(b, dtype=torch.bool)
+            keep[:nq, 0:r] = True; keep[nq:nq + nk, r:2 * r] = True; keep[nq + nk:, 2 * r:3 * r] = True
+            ll.b_qkv = fin(torch.where(keep, b, torch.zeros_like(b)))
+            a = rnd(R1, nq); a[r:] = 0
+            ll.a_o = fin(a)
+            b = rnd(shape.d, R1); b[:, r:] = 0
+            ll.b_o = fin(b)
+            a = rnd(R2, shape.d); a[2 * r:] = 0
+            ll.a_gu = fin(a)
+            b = rnd(2 * shape.F, R2)
+            keep = torch.zeros_like(b, dtype=torch.bool)
+            keep[0::2, 0:r] = True; keep[1::2, r:2 * r] = True
+            ll.b_gu = fin(torch.where(keep, b, torch.zeros_like(b)))
+            a = rnd(R1, shape.F); a[r:] = 0
+            ll.a_d = fin(a)
+            b = rnd(shape.d, R1); b[:, r:] = 0
+            ll.b_d = fin(b)
         return self
 
 
@@ -367,12 +479,15 @@ class Context:
         check(lib.hb_create(C.byref(cfg), max_tokens, max_segs, max_page_ids, None, 0, C.byref(self.handle)),
               "hb_create")
 
-    def mixed_step(self, batch, weights, kv, pool, out_logits, out_emb, stream=None):
-        check(lib.hb_mixed_step(self.handle, C.byref(batch.desc), C.byref(weights.struct), kv.handle,
-                                pool.handle if pool is not None else None,
-                                C.c_void_p(out_logits.data_ptr()) if out_logits is not None else None,
-                                C.c_void_p(out_emb.data_ptr()) if out_emb is not None else None,
-                                _stream_ptr(stream)), "hb_mixed_step")
+    def mixed_step(self, batch, weights, kv, pool, out_logits, out_emb, stream=None, lora=None):
+        tail = (kv.handle, pool.handle if pool is not None else None,
+                C.c_void_p(out_logits.data_ptr()) if out_logits is not None else None,
+                C.c_void_p(out_emb.data_ptr()) if out_emb is not None else None, _stream_ptr(stream))
+        if lora is None:
+            check(lib.hb_mixed_step(self.handle, C.byref(batch.desc), C.byref(weights.struct), *tail), "hb_mixed_step")
+        else:
+            check(lib.hb_mixed_step_lora(self.handle, C.byref(batch.desc), C.byref(weights.struct),
+                                         C.byref(lora.struct), *tail), "hb_mixed_step_lora")
 
     def argmax(self, logits, n_rows, out_tokens, stream=None):
         check(lib.hb_argmax(self.handle, C.c_void_p(logits.data_ptr()), n_rows,

@@ -63,6 +63,22 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
         *reinterpret_cast<uint4*>(out + v * 8) = pk;
       }
     }
+  } else if constexpr (EPI == HB_EPI_LORA_DOWN) {
+    // rank-r activations of the adapted rows: alpha * acc for rows >= first_row, zero for the rows
+    // before it (rows of request kinds that do not carry the adapter)
+    __half* out = static_cast<__half*>(g.C) + static_cast<size_t>(row) * g.ldc + col0;
+    const float a = (row >= g.first_row) ? g.alpha : 0.0f;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      if (col0 + v * 8 < g.N) {
+        uint4 pk;
+        pk.x = pack_half2_sat(a * __uint_as_float(r[v * 8 + 0]), a * __uint_as_float(r[v * 8 + 1]));
+        pk.y = pack_half2_sat(a * __uint_as_float(r[v * 8 + 2]), a * __uint_as_float(r[v * 8 + 3]));
+        pk.z = pack_half2_sat(a * __uint_as_float(r[v * 8 + 4]), a * __uint_as_float(r[v * 8 + 5]));
+        pk.w = pack_half2_sat(a * __uint_as_float(r[v * 8 + 6]), a * __uint_as_float(r[v * 8 + 7]));
+        *reinterpret_cast<uint4*>(out + v * 8) = pk;
+      }
+    }
   } else if constexpr (EPI == HB_EPI_F32 || EPI == HB_EPI_RESID_F32) {
     float* out = static_cast<float*>(g.C) + static_cast<size_t>(row) * g.ldc + col0;
 #pragma unroll
@@ -149,6 +165,7 @@ __device__ __forceinline__ void epilogue_qkv_rope(const GemmArgs& g, int row, in
 template <int BN, int EPI, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
                        const GemmArgs g) {
   using T = Tile<BN, CG>;
   extern __shared__ uint8_t smem_raw[];
@@ -175,7 +192,11 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   const int m_tiles = (g.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (g.N + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
-  const int k_blocks = (g.K + BK - 1) / BK;
+  // K runs over the columns of (A, B) and then over g.k2_blocks more 64-column blocks of a second
+  // operand pair (A2, B2): C = A B^T + A2 B2^T in one accumulation (the low-rank branch of an
+  // adapted projection, with A2 = the rows' rank-r activations and B2 = the up factor).
+  const int k1_blocks = (g.K + BK - 1) / BK;
+  const int k_blocks = k1_blocks + g.k2_blocks;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T::STAGES; ++s) {
@@ -228,15 +249,20 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
           const uint32_t a_dst = smem_base + stage * T::STAGE_BYTES;
           const uint32_t b_dst = a_dst + T::A_BYTES;
+          const bool ext = (kb >= k1_blocks);
+          const CUtensorMap* ma = ext ? &tmA2 : &tmA;
+          const CUtensorMap* mb = ext ? &tmB2 : &tmB;
+          const int ka = ext ? (kb - k1_blocks) * BK : kb * BK;
+          const int kbb = ext ? ka : (kb >> g.b_kshift) * BK;
           if constexpr (CG == 2) {
             const uint32_t bar = map_to_rank(full_bar(stage), 0u);
             if (leader) mbar_arrive_expect_tx(full_bar(stage), 2u * T::STAGE_BYTES);
-            tma_load_2d_cg2(a_dst, &tmA, bar, kb * BK, m0);
-            tma_load_2d_cg2(b_dst, &tmB, bar, (kb >> g.b_kshift) * BK, n0);
+            tma_load_2d_cg2(a_dst, ma, bar, ka, m0);
+            tma_load_2d_cg2(b_dst, mb, bar, kbb, n0);
           } else {
             mbar_arrive_expect_tx(full_bar(stage), T::STAGE_BYTES);
-            tma_load_2d(a_dst, &tmA, full_bar(stage), kb * BK, m0);
-            tma_load_2d(b_dst, &tmB, full_bar(stage), (kb >> g.b_kshift) * BK, n0);
+            tma_load_2d(a_dst, ma, full_bar(stage), ka, m0);
+            tma_load_2d(b_dst, mb, full_bar(stage), kbb, n0);
           }
           if (++stage == T::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -367,7 +393,8 @@ EncodeTiledFn get_encode_fn() {
 }
 
 template <int BN, int EPI, int CG>
-int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& a, int num_sms, cudaStream_t s) {
+int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
+               const GemmArgs& a, int num_sms, cudaStream_t s) {
   using T = Tile<BN, CG>;
   static bool configured = false;
   auto kern = hb_gemm_tcgen05_kernel<BN, EPI, CG>;
@@ -393,18 +420,21 @@ int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& a
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, a) == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+  return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmA2, tmB2, a) == cudaSuccess ? HB_OK : HB_ERR_CUDA;
 }
 
 template <int BN, int CG>
-int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, int epi, const GemmArgs& a, int num_sms,
-              cudaStream_t s) {
+int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
+              int epi, const GemmArgs& a, int num_sms, cudaStream_t s) {
   switch (epi) {
-    case HB_EPI_F16: return launch_one<BN, HB_EPI_F16, CG>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, a, num_sms, s);
-    case HB_EPI_QKV_ROPE: return launch_one<BN, HB_EPI_QKV_ROPE, CG>(tmA, tmB, a, num_sms, s);
+    case HB_EPI_F16: return launch_one<BN, HB_EPI_F16, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+    case HB_EPI_QKV_ROPE: return launch_one<BN, HB_EPI_QKV_ROPE, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+    case HB_EPI_LORA_DOWN:
+      if constexpr (BN == 128 && CG == 1) return launch_one<BN, HB_EPI_LORA_DOWN, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+      else return HB_ERR_BAD_ARG;
     default: return HB_ERR_BAD_ARG;
   }
 }
@@ -445,9 +475,13 @@ int hb_gemm_pick_bn(int M, int N, int num_sms) {
 int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : variant; }
 
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,
-                   int num_sms, cudaStream_t s) {
-  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, epi, a, num_sms, s);
-  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, epi, a, num_sms, s);
-  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, epi, a, num_sms, s);
+                   int num_sms, cudaStream_t s, const CUtensorMap* tmA2, const CUtensorMap* tmB2) {
+  if ((a.k2_blocks > 0) != (tmA2 != nullptr && tmB2 != nullptr) || a.k2_blocks < 0) return HB_ERR_BAD_ARG;
+  // without an extension the second pair is never read; pass the first so the parameters are valid maps
+  const CUtensorMap& a2 = tmA2 ? *tmA2 : tmA;
+  const CUtensorMap& b2 = tmB2 ? *tmB2 : tmB;
+  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, a2, b2, epi, a, num_sms, s);
+  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s);
+  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s);
   return HB_ERR_BAD_ARG;
 }

@@ -100,13 +100,22 @@ struct hb_pool {
 // Internal epilogue of the QKV projection: rotary embedding and KV-page append fused into the
 // accumulator read-out (not reachable through hb_gemm).
 constexpr int HB_EPI_QKV_ROPE = 4;
+// Internal epilogue of the adapters' down projection u = alpha * (x A^T): fp16 out, rows before
+// GemmArgs::first_row stored as zero (tile width 128 only).
+constexpr int HB_EPI_LORA_DOWN = 5;
+constexpr int HB_LORA_MAX_RANK = 64;
+constexpr int HB_LORA_U_COLS = 192;   // three rank-64 blocks: the fused q, k, v projection
 
 struct GemmArgs {
   void* C;
   int32_t M, N, K;      // K = columns of A; B has K >> b_kshift columns
   int32_t ldc;          // elements
   int32_t b_kshift;     // B k-block index = A k-block index >> b_kshift
+  int32_t k2_blocks;    // 64-column blocks of the second operand pair accumulated after K (0 = none)
   uint32_t* status;
+  // HB_EPI_LORA_DOWN only
+  float alpha;
+  int32_t first_row;
   // HB_EPI_QKV_ROPE only
   const int32_t* row_pos;   // [M] position of each row inside its request
   const int32_t* row_page;  // [M] physical page that holds that position
@@ -126,7 +135,8 @@ constexpr int HB_GEMM_PAIR256 = 512;
 int hb_gemm_pick_bn(int M, int N, int num_sms);
 int hb_gemm_box_rows(int variant);
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
-                   const GemmArgs& a, int num_sms, cudaStream_t s);
+                   const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,
+                   const CUtensorMap* tmB2 = nullptr);
 
 // ---- elementwise / attention launchers ---------------------------------------
 struct hb_ctx;
@@ -156,6 +166,7 @@ struct hb_ctx {
   __half* q;                // [max_tokens, Hq*Dh] rotated queries (fp16)
   __half* attn_out;         // [max_tokens, Hq*Dh] (fp16)
   __half* act;              // [max_tokens, F] (fp16)
+  __half* lora_u;           // [max_tokens, HB_LORA_U_COLS] rank-r activations of the adapted rows (fp16)
   __half* logit_in;         // [max_logit_rows, 2d] hi/lo fp16 split of final hidden rows
   float* rope_cos;          // [max_pos, Dh/2]
   float* rope_sin;
@@ -172,7 +183,7 @@ struct hb_ctx {
   int32_t max_logit_rows;
   DeviceDesc dd;
   // tensor maps over the activation buffers (A operands)
-  CUtensorMap tm_h, tm_attn_out, tm_act, tm_logit_in;
+  CUtensorMap tm_h, tm_attn_out, tm_act, tm_logit_in, tm_lora_u;
   // cached weight tensor maps
   struct WMaps {
     const void* key[4];
@@ -180,6 +191,14 @@ struct hb_ctx {
     int bn_qkv, bn_o, bn_gu, bn_down;
   };
   std::vector<WMaps> wmaps;
+  // cached adapter tensor maps: down factors (B operand of the thin GEMMs), up factors (second B
+  // operand of the projections)
+  struct LMaps {
+    const void* key[8];
+    int rank;
+    CUtensorMap a_qkv, b_qkv, a_o, b_o, a_gu, b_gu, a_d, b_d;
+  };
+  std::vector<LMaps> lmaps;
   const void* lm_key;
   CUtensorMap tm_lm;
   int32_t last_launches;

@@ -44,7 +44,7 @@ struct Carve {
 };
 
 struct Layout {
-  size_t x, h, q, attn_out, act, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
+  size_t x, h, q, attn_out, act, lora_u, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
       status, desc;
   size_t total, desc_cap, attn_part_floats, pool_part_floats;
   int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items;
@@ -63,6 +63,7 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.q = cv.take(rows * n_q * 2);
   L.attn_out = cv.take(rows * n_q * 2);
   L.act = cv.take(rows * c.d_ffn * 2);
+  L.lora_u = cv.take(rows * HB_LORA_U_COLS * 2);
   L.logit_in = cv.take(lrows * 2 * c.d_model * 2);
   L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
   L.rope_sin = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
@@ -241,6 +242,7 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->q = reinterpret_cast<__half*>(c->ws + lay.q);
   c->attn_out = reinterpret_cast<__half*>(c->ws + lay.attn_out);
   c->act = reinterpret_cast<__half*>(c->ws + lay.act);
+  c->lora_u = reinterpret_cast<__half*>(c->ws + lay.lora_u);
   c->logit_in = reinterpret_cast<__half*>(c->ws + lay.logit_in);
   c->rope_cos = reinterpret_cast<float*>(c->ws + lay.rope_cos);
   c->rope_sin = reinterpret_cast<float*>(c->ws + lay.rope_sin);
@@ -257,6 +259,11 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->max_logit_rows = lay.logit_rows_pad;
   c->wmaps.resize(cfg->n_layers);
   for (auto& w : c->wmaps) w.key[0] = w.key[1] = w.key[2] = w.key[3] = nullptr;
+  c->lmaps.resize(cfg->n_layers);
+  for (auto& m : c->lmaps) {
+    for (auto& k : m.key) k = nullptr;
+    m.rank = 0;
+  }
 
   int rc = HB_OK;
   bool cuda_ok = true;
@@ -287,6 +294,7 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
     if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_attn_out, c->attn_out, lay.rows_pad, n_q, 128);
     if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_act, c->act, lay.rows_pad, cfg->d_ffn, 128);
     if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_logit_in, c->logit_in, lay.logit_rows_pad, 2ull * cfg->d_model, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_lora_u, c->lora_u, lay.rows_pad, HB_LORA_U_COLS, 128);
   }
   cuda_ok &= cudaDeviceSynchronize() == cudaSuccess;
   if (!cuda_ok || rc != HB_OK) {
@@ -471,7 +479,14 @@ int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_se
 
 int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv* kv, hb_pool* pool,
                   float* out_logits, float* out_emb, void* stream) {
+  return hb_mixed_step_lora(c, d, w, nullptr, kv, pool, out_logits, out_emb, stream);
+}
+
+int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, const hb_lora* lora, hb_kv* kv,
+                       hb_pool* pool, float* out_logits, float* out_emb, void* stream) {
   if (!c || !d || !w || !kv || !w->layers || !w->tok_emb || !w->final_norm) return HB_ERR_BAD_ARG;
+  if (lora && (lora->rank < 1 || lora->rank > HB_LORA_MAX_RANK || !lora->layers || !(lora->scale == lora->scale)))
+    return HB_ERR_BAD_ARG;
   if (!kv->arena || !kv->has_map) return HB_ERR_BAD_ARG;
   if (memcmp(&kv->cfg, &c->cfg, sizeof(hb_model_cfg)) != 0) return HB_ERR_BAD_ARG;
   const int32_t n_slots = pool ? pool->n_slots : 0;
@@ -649,6 +664,12 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
 
   const int n_qkv = (cfg.n_heads + 2 * cfg.n_kv_heads) * cfg.head_dim;
   const int n_q = cfg.n_heads * cfg.head_dim;
+  // adapters apply to EMBED_CHUNK rows, which are the last rows of the batch (kinds are sorted)
+  int32_t first_embed_row = T;
+  for (int32_t r = 0; r < R; ++r)
+    if (d->segs[r].kind == HB_KIND_EMBED_CHUNK) { first_embed_row = d->segs[r].q_start; break; }
+  const bool use_lora = (lora != nullptr) && first_embed_row < T;
+  const int r1 = 64, r2 = use_lora ? (2 * lora->rank + 63) / 64 * 64 : 0, r3 = use_lora ? (3 * lora->rank + 63) / 64 * 64 : 0;
   int launches = 0;
   auto prof_begin = [&](int cls) -> ProfRec* {
     if (!ex->profiling) return nullptr;
@@ -691,6 +712,36 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
       if ((rc = hb_tmap_2d_bf16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
       wm.key[0] = lw.wqkv; wm.key[1] = lw.wo; wm.key[2] = lw.w_gate_up; wm.key[3] = lw.w_down;
     }
+    // adapters: tensor maps of this layer's packed factors (cached by pointer)
+    hb_ctx::LMaps* lm = nullptr;
+    if (use_lora) {
+      const hb_lora_layer& ll = lora->layers[l];
+      const void* keys[8] = {ll.a_qkv, ll.b_qkv, ll.a_o, ll.b_o, ll.a_gu, ll.b_gu, ll.a_d, ll.b_d};
+      for (const void* k : keys)
+        if (!k) return HB_ERR_BAD_ARG;
+      lm = &c->lmaps[l];
+      if (lm->rank != lora->rank || memcmp(lm->key, keys, sizeof(keys)) != 0) {
+        if ((rc = hb_tmap_2d_bf16(&lm->a_qkv, ll.a_qkv, r3, cfg.d_model, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->b_qkv, ll.b_qkv, n_qkv, r3, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->a_o, ll.a_o, r1, n_q, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->b_o, ll.b_o, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->a_gu, ll.a_gu, r2, cfg.d_model, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->b_gu, ll.b_gu, 2ull * cfg.d_ffn, r2, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->a_d, ll.a_d, r1, cfg.d_ffn, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->b_d, ll.b_d, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
+        memcpy(lm->key, keys, sizeof(keys));
+        lm->rank = lora->rank;
+      }
+    }
+    // rank-r activations of the adapted rows for the projection that reads activation map `tmX`
+    // with K columns: u = scale * (x A^T), zero for rows before the first embedding row
+    auto lora_down = [&](const CUtensorMap& tmX, const CUtensorMap& tmAfac, int R, int K) -> int {
+      GemmArgs gu = {};
+      gu.status = c->status;
+      gu.M = T; gu.N = R; gu.K = K; gu.C = c->lora_u; gu.ldc = HB_LORA_U_COLS;
+      gu.alpha = lora->scale; gu.first_row = first_embed_row;
+      return hb_gemm_launch(tmX, tmAfac, 128, HB_EPI_LORA_DOWN, gu, c->num_sms, s);
+    };
     if (l == 0) HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
     else HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.attn_norm, s));
     GemmArgs ga = {};
@@ -703,19 +754,31 @@ int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv*
     ga.q_out = c->q; ga.kv_layer = kg.arena + static_cast<int64_t>(l) * kg.layer_stride;
     ga.page_stride = kg.page_stride; ga.Hq = cfg.n_heads; ga.Hkv = cfg.n_kv_heads; ga.Dh = cfg.head_dim;
     ga.P = cfg.page_size; ga.n_pages = kg.n_pages;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s));
+    if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_qkv, r3, cfg.d_model));
+    ga.k2_blocks = use_lora ? r3 / 64 : 0;
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s,
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_qkv : nullptr));
     if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention_tc(c, kg, kv->map, l, s));
     if (dd.n_attn_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s));
+    if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_attn_out, lm->a_o, r1, n_q));
+    ga.k2_blocks = use_lora ? r1 / 64 : 0;
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s,
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_o : nullptr));
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.ffn_norm, s));
     // gate/up projection with SwiGLU
     ga.C = c->act; ga.N = 2 * cfg.d_ffn; ga.K = cfg.d_model; ga.ldc = cfg.d_ffn;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s));
+    if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_gu, r2, cfg.d_model));
+    ga.k2_blocks = use_lora ? r2 / 64 : 0;
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s,
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_gu : nullptr));
     // down projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = cfg.d_ffn; ga.ldc = cfg.d_model;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s));
+    if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_act, lm->a_d, r1, cfg.d_ffn));
+    ga.k2_blocks = use_lora ? r1 / 64 : 0;
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s,
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_d : nullptr));
   }
   float* pool_sum = pool ? static_cast<float*>(pool->arena) : nullptr;
   uint32_t* pool_meta = pool ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(pool->arena) +

@@ -71,8 +71,9 @@ def build_batch(entries, page_size):
 
 class Engine:
     def __init__(self, shape, weights, n_pages, n_slots, max_tokens, max_segs, max_pos,
-                 kv_fill=None, pool_fill=None, device="cuda"):
+                 kv_fill=None, pool_fill=None, device="cuda", lora=None):
         self.shape = shape
+        self.lora = lora                    # binding.DeviceLora applied to embedding rows, or None
         self.cfg = B.model_cfg(shape, max_pos)
         self.weights = weights
         self.max_tokens, self.max_segs = max_tokens, max_segs
@@ -113,7 +114,8 @@ class Engine:
         self.out_logits / self.out_emb once the stream is synchronised."""
         entries = [self.entry_for(r, n) for r, n in work]
         batch, order = build_batch(entries, self.shape.page_size)
-        self.ctx.mixed_step(batch, self.weights, self.kv, self.pool, self.out_logits, self.out_emb, stream)
+        self.ctx.mixed_step(batch, self.weights, self.kv, self.pool, self.out_logits, self.out_emb, stream,
+                            lora=self.lora)
         lrows, erows = {}, {}
         for si, ei in enumerate(order):
             req, n = work[ei]
