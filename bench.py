@@ -218,6 +218,44 @@ def run_trace(args):
     eng.close()
 
 
+def run_phases(args):
+    """Shifting request mix (10 % / 50 % / 90 % embedding requests) on one GPU through the IBS
+    scheduler: per-phase service rate of the same engine, nothing repartitioned between phases."""
+    import torch
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200 import synth, trace
+    from paper_2609_25405_b200.engine import Engine
+    shape = synth.SHAPES[args.workload.split("-")[1]]
+    n_req = args.sessions
+    phases = trace.make_phases(shape.V, n_requests=n_req)
+    budget, chunk = 4096, 512
+    max_pos = 128 + 512 + 8
+    P = shape.page_size
+    n_pages = n_req * ((max_pos + P - 1) // P) + 64
+    weights = B.DeviceWeights.random_on_device(shape, seed=0)
+    eng = Engine(shape, weights, n_pages=n_pages, n_slots=n_req + 8, max_tokens=budget,
+                 max_segs=n_req + budget // 16 + 8, max_pos=max_pos)
+    per_phase, rows, busy, steps = [], 0, 0.0, 0
+    for frac, sessions in zip((0.1, 0.5, 0.9), phases):
+        out = trace.replay(sessions, eng, budget, chunk)
+        per_phase.append({"embed_request_frac": frac, "rows": out["rows"], "steps": out["steps"],
+                          "busy_s": out["busy_s"], "tokens_per_s": out["rows"] / out["busy_s"],
+                          "mean_rows_per_step": out["rows"] / max(out["steps"], 1),
+                          "expected_rows": trace.trace_tokens(sessions)})
+        rows += out["rows"]; busy += out["busy_s"]; steps += out["steps"]
+    status = eng.ctx.status_poll()
+    line = {"metric": METRIC, "value": rows / busy, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": 0,
+            "ms_per_step": 1e3 * busy / max(steps, 1), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": args.workload, "shape": shape.name, "requests_per_phase": n_req,
+                       "token_budget": budget, "chunk": chunk, "scheduler": "IBS",
+                       "sizes": "embedding 128 tokens; generation 128-token prompt + 512 decode steps"},
+            "phases": per_phase, "free_pages_after": eng.kv.free_count(), "n_pages": n_pages,
+            "device_status": status}
+    print(json.dumps(line))
+    eng.close()
+
+
 # ------------------------------------------------------------------------------------------
 # the CUDA path
 # ------------------------------------------------------------------------------------------
@@ -234,6 +272,8 @@ def main():
     ap.add_argument("--decode-alias", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--sessions", type=int, default=256, help="sessions of the cfg5-trace-1b workload")
+    ap.add_argument("--lora-rank", type=int, default=0,
+                    help="rank of a random low-rank adapter applied to the embedding rows (0 = none, the headline)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -248,6 +288,9 @@ def main():
 
     if args.workload.startswith("cfg5-trace"):
         run_trace(args)
+        return
+    if args.workload.startswith("phases-"):
+        run_phases(args)
         return
 
     rank = int(os.environ.get("RANK", "0"))
@@ -278,6 +321,7 @@ def main():
     max_page_ids = spec.n_decode * ((max_pos + P - 1) // P) + (spec.budget // 16 + 8) * ((spec.emb_hi + P - 1) // P + 1)
 
     weights = B.DeviceWeights.random_on_device(shape, seed=0)
+    lora = B.DeviceLora.random_on_device(shape, args.lora_rank) if args.lora_rank else None
     kv = B.KvCache(cfg, n_pages)
     kvb = kv.arena.view(torch.float16)
     step_e = 1 << 28
@@ -302,7 +346,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def run(i):
-        ctx.mixed_step(batches[i], weights, kv, pool, out_logits, out_emb, stream)
+        ctx.mixed_step(batches[i], weights, kv, pool, out_logits, out_emb, stream, lora=lora)
 
     for i in range(args.warmup):
         run(i)
@@ -338,7 +382,7 @@ def main():
     h2d = d2h = 0
     for i in timed:
         b = build_batch(entries_all[i], P)[0]
-        ctx.mixed_step(b, weights, kv, pool, out_logits, out_emb, stream)
+        ctx.mixed_step(b, weights, kv, pool, out_logits, out_emb, stream, lora=lora)
         nl, ne = b.desc.n_logit_rows, b.desc.n_emb_rows
         if nl:
             h_logits[:nl].copy_(out_logits[:nl], non_blocking=True)
@@ -403,7 +447,7 @@ def main():
             "config": {"workload": spec.name, "shape": shape.name, "tokens_per_step": w["T"],
                        "decode_rows": spec.n_decode, "chunk": spec.chunk, "token_budget": spec.budget,
                        "l2": "inputs larger than L2 (weights and KV pages are re-streamed every step)",
-                       "replicas": world, "decode_alias": args.decode_alias},
+                       "replicas": world, "decode_alias": args.decode_alias, "lora_rank": args.lora_rank},
             "clocks": clocks, "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
                                       "h2d_bytes_per_step": h2d / K, "d2h_bytes_per_step": d2h / K},
             "gpu_launches": launches, "roofline": roofline, "step_roofline": step_roof,

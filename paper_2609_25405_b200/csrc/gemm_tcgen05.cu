@@ -114,6 +114,17 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
   }
 }
 
+// Split-K partial of the thin adapter GEMM: fp32, [split][row][N].
+__device__ __forceinline__ void store_partial(const GemmArgs& g, int split, int row, int col0, const uint32_t (&r)[32]) {
+  float* out = g.split_part + (static_cast<size_t>(split) * g.M + row) * g.N + col0;
+#pragma unroll
+  for (int v = 0; v < 8; ++v) {
+    if (col0 + v * 4 < g.N)
+      *reinterpret_cast<float4*>(out + v * 4) = make_float4(__uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
+                                                             __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+  }
+}
+
 // QKV epilogue: one thread holds 32 consecutive output columns of one token row.  The q and k rows
 // of the weight are pair-interleaved inside each head (column 2i = rotary element i, column 2i+1 =
 // element i + Dh/2), so every rotation pair sits in adjacent columns.  q goes to the query buffer,
@@ -191,12 +202,17 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 
   const int m_tiles = (g.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (g.N + BN - 1) / BN;
-  const int total_tiles = m_tiles * n_tiles;
+  // k_splits > 1 (thin adapter GEMMs only): every output tile is computed by k_splits work items,
+  // each over an equal share of the K blocks; the partial sums are combined in the epilogue.
+  const int mn_tiles = m_tiles * n_tiles;
+  const int k_splits = (EPI == HB_EPI_LORA_DOWN) ? g.k_splits : 1;
+  const int total_tiles = mn_tiles * k_splits;
   // K runs over the columns of (A, B) and then over g.k2_blocks more 64-column blocks of a second
   // operand pair (A2, B2): C = A B^T + A2 B2^T in one accumulation (the low-rank branch of an
   // adapted projection, with A2 = the rows' rank-r activations and B2 = the up factor).
   const int k1_blocks = (g.K + BK - 1) / BK;
   const int k_blocks = k1_blocks + g.k2_blocks;
+  const int k_per_split = (k_blocks + k_splits - 1) / k_splits;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T::STAGES; ++s) {
@@ -243,9 +259,11 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       bool ok = true;
       // the data of both CTAs of a group is accounted on the leader's barrier
       for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
-        const int m0 = (tile % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
-        const int n0 = (tile / m_tiles) * BN + static_cast<int>(rank) * T::B_ROWS;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int mn = tile % mn_tiles, split = tile / mn_tiles;
+        const int m0 = (mn % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
+        const int n0 = (mn / m_tiles) * BN + static_cast<int>(rank) * T::B_ROWS;
+        const int kb0 = split * k_per_split, kb1 = min(kb0 + k_per_split, k_blocks);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
           const uint32_t a_dst = smem_base + stage * T::STAGE_BYTES;
           const uint32_t b_dst = a_dst + T::A_BYTES;
@@ -286,7 +304,9 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int split = tile / mn_tiles;
+        const int kb0 = split * k_per_split, kb1 = min(kb0 + k_per_split, k_blocks);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
           tc_fence_after();
           const uint32_t a_addr = smem_base + stage * T::STAGE_BYTES;
@@ -295,7 +315,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 elements along K inside the 128-byte swizzle row = +32 B = +2 in the address field
-            const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
+            const uint32_t accum = (kb > kb0 || k > 0) ? 1u : 0u;
             if constexpr (CG == 2) umma_ss_cg2(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
             else umma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, accum);
           }
@@ -318,8 +338,9 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
-      const int m0 = (tile % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
-      const int n0 = (tile / m_tiles) * BN;
+      const int mn = tile % mn_tiles, split = tile / mn_tiles;
+      const int m0 = (mn % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
+      const int n0 = (mn / m_tiles) * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
@@ -342,8 +363,14 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         tmem_ld32(t_row + static_cast<uint32_t>(c), r);
         tmem_ld_wait();
         if (row_ok && n0 + c < g.N) {
-          if constexpr (EPI == HB_EPI_QKV_ROPE) epilogue_qkv_rope(g, row, n0 + c, r, pos, page);
-          else epilogue_store<EPI>(g, row, n0 + c, r);
+          if constexpr (EPI == HB_EPI_QKV_ROPE) {
+            epilogue_qkv_rope(g, row, n0 + c, r, pos, page);
+          } else if constexpr (EPI == HB_EPI_LORA_DOWN) {
+            if (k_splits > 1) store_partial(g, split, row, n0 + c, r);
+            else epilogue_store<EPI>(g, row, n0 + c, r);
+          } else {
+            epilogue_store<EPI>(g, row, n0 + c, r);
+          }
         }
       }
       tc_fence_before();
@@ -351,6 +378,44 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       if (lane == 0) {
         if constexpr (CG == 2) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));
         else mbar_arrive(tempty_bar(acc));
+      }
+      if constexpr (EPI == HB_EPI_LORA_DOWN) {
+        if (k_splits > 1) {
+          // The warp that arrives last for these 32 rows of the tile adds the partial sums in split
+          // order (a fixed order: the result does not depend on which work item finished when).
+          __threadfence();
+          __syncwarp();
+          uint32_t prev = 0;
+          uint32_t* ctr = g.split_counters + (static_cast<size_t>(mn) * 4 + quarter);
+          if (lane == 0) prev = atomicAdd(ctr, 1u);
+          prev = __shfl_sync(0xffffffffu, prev, 0);
+          if (prev + 1u == static_cast<uint32_t>(k_splits)) {
+            __threadfence();
+            if (row_ok) {
+              for (int c = 0; c < BN && n0 + c < g.N; c += 32) {
+                uint32_t r[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;   // +0.0f
+                for (int sp = 0; sp < k_splits; ++sp) {
+                  const float* src = g.split_part + (static_cast<size_t>(sp) * g.M + row) * g.N + n0 + c;
+#pragma unroll
+                  for (int v = 0; v < 8; ++v) {
+                    if (n0 + c + v * 4 < g.N) {
+                      const float4 p = __ldcg(reinterpret_cast<const float4*>(src + v * 4));
+                      r[v * 4 + 0] = __float_as_uint(__uint_as_float(r[v * 4 + 0]) + p.x);
+                      r[v * 4 + 1] = __float_as_uint(__uint_as_float(r[v * 4 + 1]) + p.y);
+                      r[v * 4 + 2] = __float_as_uint(__uint_as_float(r[v * 4 + 2]) + p.z);
+                      r[v * 4 + 3] = __float_as_uint(__uint_as_float(r[v * 4 + 3]) + p.w);
+                    }
+                  }
+                }
+                epilogue_store<EPI>(g, row, n0 + c, r);
+              }
+            }
+            __syncwarp();
+            if (lane == 0) *ctr = 0u;   // ready for the next launch
+          }
+        }
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -405,7 +470,7 @@ int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap
   }
   const int m_tiles = (a.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (a.N + BN - 1) / BN;
-  int workers = m_tiles * n_tiles;
+  int workers = m_tiles * n_tiles * ((EPI == HB_EPI_LORA_DOWN && a.k_splits > 1) ? a.k_splits : 1);
   if (workers > num_sms / CG) workers = num_sms / CG;
   if (workers < 1) return HB_OK;
   cudaLaunchConfig_t cfg = {};
@@ -433,7 +498,7 @@ int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap&
     case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
     case HB_EPI_QKV_ROPE: return launch_one<BN, HB_EPI_QKV_ROPE, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
     case HB_EPI_LORA_DOWN:
-      if constexpr (BN == 128 && CG == 1) return launch_one<BN, HB_EPI_LORA_DOWN, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+      if constexpr (CG == 1) return launch_one<BN, HB_EPI_LORA_DOWN, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
       else return HB_ERR_BAD_ARG;
     default: return HB_ERR_BAD_ARG;
   }
@@ -477,6 +542,8 @@ int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : va
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,
                    int num_sms, cudaStream_t s, const CUtensorMap* tmA2, const CUtensorMap* tmB2) {
   if ((a.k2_blocks > 0) != (tmA2 != nullptr && tmB2 != nullptr) || a.k2_blocks < 0) return HB_ERR_BAD_ARG;
+  if (epi == HB_EPI_LORA_DOWN && (a.k_splits < 1 || (a.k_splits > 1 && (!a.split_part || !a.split_counters))))
+    return HB_ERR_BAD_ARG;
   // without an extension the second pair is never read; pass the first so the parameters are valid maps
   const CUtensorMap& a2 = tmA2 ? *tmA2 : tmA;
   const CUtensorMap& b2 = tmB2 ? *tmB2 : tmB;

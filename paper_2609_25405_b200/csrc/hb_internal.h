@@ -103,6 +103,7 @@ constexpr int HB_EPI_QKV_ROPE = 4;
 // Internal epilogue of the adapters' down projection u = alpha * (x A^T): fp16 out, rows before
 // GemmArgs::first_row stored as zero (tile width 128 only).
 constexpr int HB_EPI_LORA_DOWN = 5;
+constexpr int HB_LORA_K_SPLITS = 4;
 constexpr int HB_LORA_MAX_RANK = 64;
 constexpr int HB_LORA_U_COLS = 192;   // three rank-64 blocks: the fused q, k, v projection
 
@@ -116,6 +117,9 @@ struct GemmArgs {
   // HB_EPI_LORA_DOWN only
   float alpha;
   int32_t first_row;
+  int32_t k_splits;          // work items per output tile (>= 1), each over an equal share of the K blocks
+  float* split_part;         // [k_splits, M, N] partial sums (k_splits > 1)
+  uint32_t* split_counters;  // [tiles * 4] arrival counters, zero between launches
   // HB_EPI_QKV_ROPE only
   const int32_t* row_pos;   // [M] position of each row inside its request
   const int32_t* row_page;  // [M] physical page that holds that position
@@ -167,6 +171,9 @@ struct hb_ctx {
   __half* attn_out;         // [max_tokens, Hq*Dh] (fp16)
   __half* act;              // [max_tokens, F] (fp16)
   __half* lora_u;           // [max_tokens, HB_LORA_U_COLS] rank-r activations of the adapted rows (fp16)
+  float* lora_part;         // [HB_LORA_K_SPLITS, max_tokens, HB_LORA_U_COLS] split-K partial sums
+  uint32_t* lora_counters;  // [n_lora_counters] arrival counters of the split-K merge
+  int32_t n_lora_counters;
   __half* logit_in;         // [max_logit_rows, 2d] hi/lo fp16 split of final hidden rows
   float* rope_cos;          // [max_pos, Dh/2]
   float* rope_sin;

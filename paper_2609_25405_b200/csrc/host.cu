@@ -44,7 +44,7 @@ struct Carve {
 };
 
 struct Layout {
-  size_t x, h, q, attn_out, act, lora_u, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
+  size_t x, h, q, attn_out, act, lora_u, lora_part, lora_counters, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
       status, desc;
   size_t total, desc_cap, attn_part_floats, pool_part_floats;
   int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items;
@@ -64,6 +64,8 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.attn_out = cv.take(rows * n_q * 2);
   L.act = cv.take(rows * c.d_ffn * 2);
   L.lora_u = cv.take(rows * HB_LORA_U_COLS * 2);
+  L.lora_part = cv.take(static_cast<size_t>(HB_LORA_K_SPLITS) * rows * HB_LORA_U_COLS * 4);
+  L.lora_counters = cv.take((rows / 128) * 2 * 4 * 4);
   L.logit_in = cv.take(lrows * 2 * c.d_model * 2);
   L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
   L.rope_sin = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
@@ -243,6 +245,9 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->attn_out = reinterpret_cast<__half*>(c->ws + lay.attn_out);
   c->act = reinterpret_cast<__half*>(c->ws + lay.act);
   c->lora_u = reinterpret_cast<__half*>(c->ws + lay.lora_u);
+  c->lora_part = reinterpret_cast<float*>(c->ws + lay.lora_part);
+  c->lora_counters = reinterpret_cast<uint32_t*>(c->ws + lay.lora_counters);
+  c->n_lora_counters = static_cast<int32_t>((lay.rows_pad / 128) * 2 * 4);
   c->logit_in = reinterpret_cast<__half*>(c->ws + lay.logit_in);
   c->rope_cos = reinterpret_cast<float*>(c->ws + lay.rope_cos);
   c->rope_sin = reinterpret_cast<float*>(c->ws + lay.rope_sin);
@@ -721,11 +726,11 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
         if (!k) return HB_ERR_BAD_ARG;
       lm = &c->lmaps[l];
       if (lm->rank != lora->rank || memcmp(lm->key, keys, sizeof(keys)) != 0) {
-        if ((rc = hb_tmap_2d_bf16(&lm->a_qkv, ll.a_qkv, r3, cfg.d_model, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->a_qkv, ll.a_qkv, r3, cfg.d_model, r3 > 128 ? 256 : 128)) != HB_OK) return rc;
         if ((rc = hb_tmap_2d_bf16(&lm->b_qkv, ll.b_qkv, n_qkv, r3, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
         if ((rc = hb_tmap_2d_bf16(&lm->a_o, ll.a_o, r1, n_q, 128)) != HB_OK) return rc;
         if ((rc = hb_tmap_2d_bf16(&lm->b_o, ll.b_o, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->a_gu, ll.a_gu, r2, cfg.d_model, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_bf16(&lm->a_gu, ll.a_gu, r2, cfg.d_model, r2 > 128 ? 256 : 128)) != HB_OK) return rc;
         if ((rc = hb_tmap_2d_bf16(&lm->b_gu, ll.b_gu, 2ull * cfg.d_ffn, r2, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
         if ((rc = hb_tmap_2d_bf16(&lm->a_d, ll.a_d, r1, cfg.d_ffn, 128)) != HB_OK) return rc;
         if ((rc = hb_tmap_2d_bf16(&lm->b_d, ll.b_d, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
@@ -740,7 +745,11 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
       gu.status = c->status;
       gu.M = T; gu.N = R; gu.K = K; gu.C = c->lora_u; gu.ldc = HB_LORA_U_COLS;
       gu.alpha = lora->scale; gu.first_row = first_embed_row;
-      return hb_gemm_launch(tmX, tmAfac, 128, HB_EPI_LORA_DOWN, gu, c->num_sms, s);
+      // split K four ways (fewer when K is short): the split depends on K alone, so a row's
+      // summation order is the same in every batch
+      gu.k_splits = std::min(HB_LORA_K_SPLITS, (K + 63) / 64);
+      gu.split_part = c->lora_part; gu.split_counters = c->lora_counters;
+      return hb_gemm_launch(tmX, tmAfac, R > 128 ? 256 : 128, HB_EPI_LORA_DOWN, gu, c->num_sms, s);
     };
     if (l == 0) HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
     else HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.attn_norm, s));
@@ -849,7 +858,8 @@ int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
     // a block that gave up may have left arrival counters mid-count: clear them with the status word
     if (cudaMemsetAsync(c->attn_counters, 0, static_cast<size_t>(c->max_segs) * c->cfg.n_kv_heads * 4, s) !=
             cudaSuccess ||
-        cudaMemsetAsync(c->counters, 0, static_cast<size_t>(c->n_counters) * 4, s) != cudaSuccess)
+        cudaMemsetAsync(c->counters, 0, static_cast<size_t>(c->n_counters) * 4, s) != cudaSuccess ||
+        cudaMemsetAsync(c->lora_counters, 0, static_cast<size_t>(c->n_lora_counters) * 4, s) != cudaSuccess)
       return HB_ERR_CUDA;
     if (cudaMemsetAsync(c->status, 0, 4, s) != cudaSuccess) return HB_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;

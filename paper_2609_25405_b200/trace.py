@@ -53,6 +53,28 @@ def make_trace(V, seed=1005, n_sessions=256, rate=20.0, rounds=(3, 5), query=(16
     return sessions
 
 
+def make_phases(V, seed=1006, n_requests=256, embed_fracs=(0.1, 0.5, 0.9), embed_len=128, prompt_len=128,
+                decode_len=512):
+    """Shifting request mix (the utilisation experiment of Section 5.3): one list of single-request
+    sessions per phase; in phase p a request is an embedding with probability embed_fracs[p], else a
+    generation.  Sizes are the paper's synthetic ones (Section 5.1: 128-token embeddings, 128-token
+    prompts with 512 generated tokens).  All requests of a phase are present from its start (a
+    saturated server); the next phase starts when the previous one has drained."""
+    rng = np.random.default_rng(seed)
+    phases = []
+    for frac in embed_fracs:
+        sessions = []
+        for _ in range(n_requests):
+            s = Session(arrival=0.0)
+            if rng.random() < frac:
+                s.requests.append(TraceRequest("embed", synth.token_ids(rng, embed_len, V)))
+            else:
+                s.requests.append(TraceRequest("gen", synth.token_ids(rng, prompt_len, V), decode_len))
+            sessions.append(s)
+        phases.append(sessions)
+    return phases
+
+
 def trace_tokens(sessions):
     """Rows the replay will process: every text / prompt token once plus one row per decode step."""
     return sum(len(r.tokens) + r.decode_steps for s in sessions for r in s.requests)

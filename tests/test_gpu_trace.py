@@ -48,3 +48,25 @@ def test_trace_replay_tiny():
     assert np.max(np.abs(row - lg[0])) <= 5e-2
     assert token == int(np.argmax(row))                      # the device argmax is the argmax of its own logits
     eng.close()
+
+
+def test_phase_workload_tiny():
+    """Shifting request mix (10 % / 50 % / 90 % embedding requests) replayed phase by phase through the
+    same engine: every phase drains, row counts are the phases' own, pages and slots all come back."""
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200 import trace
+    from paper_2609_25405_b200.engine import Engine
+    shape = synth.SHAPES["tiny"]
+    dw = B.DeviceWeights.from_synth(synth.Weights(shape, 0))
+    phases = trace.make_phases(shape.V, seed=4, n_requests=12, embed_len=40, prompt_len=24, decode_len=6)
+    n_pages = 12 * 4 + 8
+    eng = Engine(shape, dw, n_pages=n_pages, n_slots=16, max_tokens=128, max_segs=48, max_pos=64)
+    n_embed = []
+    for sessions in phases:
+        out = trace.replay(sessions, eng, budget=128, chunk=32)
+        assert out["sessions_done"] == 12 and out["rows"] == trace.trace_tokens(sessions)
+        assert out["free_pages"] == n_pages
+        n_embed.append(sum(s.requests[0].kind == "embed" for s in sessions))
+    assert eng.ctx.status_poll() == 0
+    assert n_embed[0] < n_embed[1] < n_embed[2]
+    eng.close()
