@@ -151,6 +151,8 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS)
 attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   constexpr int CH = DH / 8;                          // 16-byte chunks per row
   constexpr int TILE_BYTES = TILE_KEYS * DH * 2;
   constexpr int REC = DH + 2;                         // floats per row of a partial record
@@ -415,7 +417,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
 }
 
 template <int DH>
-int launch(const CUtensorMap& kv_map, const AttnParams& p, int n_items, int max_pos, cudaStream_t s) {
+int launch(const CUtensorMap& kv_map, const AttnParams& p, int n_items, int max_pos, cudaStream_t s, bool pdl) {
   // ring + barriers + page ids of one item (at most every page of a request) + alignment slack
   const int smem = TILE_KEYS * DH * 2 * (2 * STAGES) + 64 + (max_pos / 16 + 2) * 4 + 1024;
   static int configured = 0;
@@ -425,8 +427,7 @@ int launch(const CUtensorMap& kv_map, const AttnParams& p, int n_items, int max_
       return HB_ERR_CUDA;
     configured = smem;
   }
-  attn_kernel<DH><<<n_items, ATT_THREADS, smem, s>>>(kv_map, p);
-  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+  return hb_launch_kernel(attn_kernel<DH>, n_items, ATT_THREADS, smem, s, pdl, kv_map, p);
 }
 
 }  // namespace
@@ -446,7 +447,7 @@ int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, 
   p.Hq = c->cfg.n_heads;
   p.G = c->cfg.n_heads / c->cfg.n_kv_heads;
   p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));
-  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_attn_items, c->cfg.max_pos, s);
-  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_attn_items, c->cfg.max_pos, s);
+  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_attn_items, c->cfg.max_pos, s, c->pdl);
+  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_attn_items, c->cfg.max_pos, s, c->pdl);
   return HB_ERR_UNSUPPORTED;
 }

@@ -55,6 +55,8 @@ struct TcCfg {
 template <int DH>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams p) {
+  grid_dep_wait();
+  grid_dep_launch();
   using C = TcCfg<DH>;
   extern __shared__ uint8_t smem_raw[];
   // The kernel has no static shared memory, so the dynamic window starts at the CTA's (1 KiB
@@ -351,7 +353,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 }
 
 template <int DH>
-int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_pos, cudaStream_t s) {
+int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_pos, cudaStream_t s, bool pdl) {
   using C = TcCfg<DH>;
   (void)max_pos;
   const int smem = C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16;   // two CTAs per SM at Dh = 128
@@ -362,8 +364,7 @@ int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_po
       return HB_ERR_CUDA;
     configured = smem;
   }
-  attn_chunk_tc_kernel<DH><<<n_items, TC_THREADS, smem, s>>>(kv_map, p);
-  return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+  return hb_launch_kernel(attn_chunk_tc_kernel<DH>, n_items, TC_THREADS, smem, s, pdl, kv_map, p);
 }
 
 }  // namespace
@@ -382,7 +383,7 @@ int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_ma
   p.pages = c->dd.pages;
   p.status = c->status;
   p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));
-  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s);
-  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s);
+  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s, c->pdl);
+  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s, c->pdl);
   return HB_ERR_UNSUPPORTED;
 }

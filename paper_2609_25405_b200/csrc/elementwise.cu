@@ -33,6 +33,8 @@ __global__ void __launch_bounds__(NORM_THREADS)
 norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E,
             const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __half* __restrict__ h,
             int d, float eps) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ float red[32];
   const int t = blockIdx.x;
   const int nv = d >> 2;
@@ -76,6 +78,8 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
 __global__ void __launch_bounds__(NORM_THREADS)
 final_logit_rows_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
                         const int32_t* __restrict__ logit_src, __half* __restrict__ out, int d, float eps) {
+  grid_dep_wait();
+  grid_dep_launch();
   __shared__ float red[32];
   const int i = blockIdx.x;
   const int t = logit_src[i];
@@ -119,6 +123,8 @@ final_pool_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__
                   uint32_t* __restrict__ counters, float* __restrict__ pool_sum, uint32_t* __restrict__ pool_meta,
                   float* __restrict__ out_emb, int d, float eps, int n_slots, uint32_t* status,
                   float* __restrict__ rowbuf, int rowbuf_rows) {
+  grid_dep_wait();
+  grid_dep_launch();
   const PoolItem it = items[blockIdx.x];
   const hb_seg sg = segs[it.seg];
   pool_block(it, sg, x, gain, part, counters, pool_sum, pool_meta, out_emb, d, eps, n_slots, status, rowbuf,
@@ -202,31 +208,29 @@ int check_launch() { return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_C
 }  // namespace
 
 int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s) {
-  norm_kernel<true><<<c->dd.T, NORM_THREADS, 0, s>>>(c->dd.tok, static_cast<const __nv_bfloat16*>(tok_emb),
-                                                     static_cast<const __nv_bfloat16*>(gain), c->x, c->h,
-                                                     c->cfg.d_model, c->cfg.rms_eps);
-  return check_launch();
+  return hb_launch_kernel(norm_kernel<true>, c->dd.T, NORM_THREADS, 0, s, c->pdl, c->dd.tok,
+                          static_cast<const __nv_bfloat16*>(tok_emb), static_cast<const __nv_bfloat16*>(gain), c->x,
+                          c->h, c->cfg.d_model, c->cfg.rms_eps);
 }
 
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s) {
-  norm_kernel<false><<<c->dd.T, NORM_THREADS, 0, s>>>(nullptr, nullptr, static_cast<const __nv_bfloat16*>(gain), c->x,
-                                                      c->h, c->cfg.d_model, c->cfg.rms_eps);
-  return check_launch();
+  return hb_launch_kernel(norm_kernel<false>, c->dd.T, NORM_THREADS, 0, s, c->pdl, nullptr, nullptr,
+                          static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps);
 }
 
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta, int n_slots,
                     float* rowbuf, int rowbuf_rows, float* out_emb, cudaStream_t s) {
   const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(gain);
   if (c->dd.n_logit > 0) {
-    final_logit_rows_kernel<<<c->dd.n_logit, NORM_THREADS, 0, s>>>(c->x, g, c->dd.logit_src, c->logit_in,
-                                                                   c->cfg.d_model, c->cfg.rms_eps);
-    if (check_launch() != HB_OK) return HB_ERR_CUDA;
+    if (hb_launch_kernel(final_logit_rows_kernel, c->dd.n_logit, NORM_THREADS, 0, s, c->pdl, c->x, g, c->dd.logit_src,
+                         c->logit_in, c->cfg.d_model, c->cfg.rms_eps) != HB_OK)
+      return HB_ERR_CUDA;
   }
   if (c->dd.n_pool_items > 0) {
-    final_pool_kernel<<<c->dd.n_pool_items, NORM_THREADS, 0, s>>>(
-        c->x, g, c->dd.pool_items, c->dd.segs, c->pool_part, c->counters, pool_sum, pool_meta, out_emb,
-        c->cfg.d_model, c->cfg.rms_eps, n_slots, c->status, rowbuf, rowbuf_rows);
-    if (check_launch() != HB_OK) return HB_ERR_CUDA;
+    if (hb_launch_kernel(final_pool_kernel, c->dd.n_pool_items, NORM_THREADS, 0, s, c->pdl, c->x, g, c->dd.pool_items,
+                         c->dd.segs, c->pool_part, c->counters, pool_sum, pool_meta, out_emb, c->cfg.d_model,
+                         c->cfg.rms_eps, n_slots, c->status, rowbuf, rowbuf_rows) != HB_OK)
+      return HB_ERR_CUDA;
   }
   return HB_OK;
 }

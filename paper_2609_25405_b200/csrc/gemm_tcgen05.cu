@@ -244,6 +244,11 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   if constexpr (CG == 2) cluster_sync();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above touches only this CTA's shared memory and TMEM, so it may run while the previous
+  // kernel of the stream drains.  The order "allocate, wait, let the next kernel in" means that when a
+  // following kernel's CTAs become resident every CTA of this one already holds its TMEM columns.
+  grid_dep_wait();
+  grid_dep_launch();
 
   // Give up: raise the flag here and in the peer CTA so that every role of the group leaves its loop.
   auto give_up = [&]() {
@@ -459,7 +464,7 @@ EncodeTiledFn get_encode_fn() {
 
 template <int BN, int EPI, int CG>
 int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
-               const GemmArgs& a, int num_sms, cudaStream_t s) {
+               const GemmArgs& a, int num_sms, cudaStream_t s, bool pdl) {
   using T = Tile<BN, CG>;
   static bool configured = false;
   auto kern = hb_gemm_tcgen05_kernel<BN, EPI, CG>;
@@ -478,27 +483,29 @@ int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap
   cfg.blockDim = dim3(NUM_THREADS);
   cfg.dynamicSmemBytes = T::SMEM_BYTES;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CG;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmA2, tmB2, a) == cudaSuccess ? HB_OK : HB_ERR_CUDA;
 }
 
 template <int BN, int CG>
 int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
-              int epi, const GemmArgs& a, int num_sms, cudaStream_t s) {
+              int epi, const GemmArgs& a, int num_sms, cudaStream_t s, bool pdl) {
   switch (epi) {
-    case HB_EPI_F16: return launch_one<BN, HB_EPI_F16, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
-    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
-    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
-    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
-    case HB_EPI_QKV_ROPE: return launch_one<BN, HB_EPI_QKV_ROPE, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+    case HB_EPI_F16: return launch_one<BN, HB_EPI_F16, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s, pdl);
+    case HB_EPI_F32: return launch_one<BN, HB_EPI_F32, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s, pdl);
+    case HB_EPI_RESID_F32: return launch_one<BN, HB_EPI_RESID_F32, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s, pdl);
+    case HB_EPI_SWIGLU: return launch_one<BN, HB_EPI_SWIGLU, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s, pdl);
+    case HB_EPI_QKV_ROPE: return launch_one<BN, HB_EPI_QKV_ROPE, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s, pdl);
     case HB_EPI_LORA_DOWN:
-      if constexpr (CG == 1) return launch_one<BN, HB_EPI_LORA_DOWN, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s);
+      if constexpr (CG == 1) return launch_one<BN, HB_EPI_LORA_DOWN, CG>(tmA, tmB, tmA2, tmB2, a, num_sms, s, pdl);
       else return HB_ERR_BAD_ARG;
     default: return HB_ERR_BAD_ARG;
   }
@@ -540,15 +547,15 @@ int hb_gemm_pick_bn(int M, int N, int num_sms) {
 int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : variant; }
 
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,
-                   int num_sms, cudaStream_t s, const CUtensorMap* tmA2, const CUtensorMap* tmB2) {
+                   int num_sms, cudaStream_t s, const CUtensorMap* tmA2, const CUtensorMap* tmB2, bool pdl) {
   if ((a.k2_blocks > 0) != (tmA2 != nullptr && tmB2 != nullptr) || a.k2_blocks < 0) return HB_ERR_BAD_ARG;
   if (epi == HB_EPI_LORA_DOWN && (a.k_splits < 1 || (a.k_splits > 1 && (!a.split_part || !a.split_counters))))
     return HB_ERR_BAD_ARG;
   // without an extension the second pair is never read; pass the first so the parameters are valid maps
   const CUtensorMap& a2 = tmA2 ? *tmA2 : tmA;
   const CUtensorMap& b2 = tmB2 ? *tmB2 : tmB;
-  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, a2, b2, epi, a, num_sms, s);
-  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s);
-  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s);
+  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, a2, b2, epi, a, num_sms, s, pdl);
+  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s, pdl);
+  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s, pdl);
   return HB_ERR_BAD_ARG;
 }

@@ -140,7 +140,25 @@ int hb_gemm_pick_bn(int M, int N, int num_sms);
 int hb_gemm_box_rows(int variant);
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,
-                   const CUtensorMap* tmB2 = nullptr);
+                   const CUtensorMap* tmB2 = nullptr, bool pdl = false);
+
+// Plain launch, optionally allowed to overlap the tail of the previous kernel of the stream (the
+// kernel must then start with grid_dep_wait()).
+template <typename... KArgs, typename... Args>
+inline int hb_launch_kernel(void (*kern)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t s,
+                            bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...) == cudaSuccess ? HB_OK : HB_ERR_CUDA;
+}
 
 // ---- elementwise / attention launchers ---------------------------------------
 struct hb_ctx;
@@ -209,4 +227,5 @@ struct hb_ctx {
   const void* lm_key;
   CUtensorMap tm_lm;
   int32_t last_launches;
+  bool pdl;   // the next launch may overlap the tail of the previous kernel (set inside a step)
 };

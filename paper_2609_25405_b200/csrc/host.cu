@@ -225,6 +225,7 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->extra = ex;
   c->lm_key = nullptr;
   c->last_launches = 0;
+  c->pdl = false;
   if (workspace) {
     if (workspace_bytes < lay.total || (reinterpret_cast<uintptr_t>(workspace) & 255u)) {
       delete c; delete ex;
@@ -676,6 +677,10 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   const bool use_lora = (lora != nullptr) && first_embed_row < T;
   const int r1 = 64, r2 = use_lora ? (2 * lora->rank + 63) / 64 * 64 : 0, r3 = use_lora ? (3 * lora->rank + 63) / 64 * 64 : 0;
   int launches = 0;
+  // Kernels after the first may become resident while their predecessor drains (programmatic
+  // dependent launch); not while per-launch events are being recorded between them.
+  const bool pdl_enabled = !ex->profiling;
+  c->pdl = false;
   auto prof_begin = [&](int cls) -> ProfRec* {
     if (!ex->profiling) return nullptr;
     ProfRec r;
@@ -700,6 +705,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     prof_end(pr__);                   \
     if (rc__ != HB_OK) return rc__;   \
     ++launches;                       \
+    c->pdl = pdl_enabled;             \
   } while (0)
 
   for (int l = 0; l < cfg.n_layers; ++l) {
@@ -749,7 +755,8 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
       // summation order is the same in every batch
       gu.k_splits = std::min(HB_LORA_K_SPLITS, (K + 63) / 64);
       gu.split_part = c->lora_part; gu.split_counters = c->lora_counters;
-      return hb_gemm_launch(tmX, tmAfac, R > 128 ? 256 : 128, HB_EPI_LORA_DOWN, gu, c->num_sms, s);
+      return hb_gemm_launch(tmX, tmAfac, R > 128 ? 256 : 128, HB_EPI_LORA_DOWN, gu, c->num_sms, s, nullptr, nullptr,
+                            c->pdl);
     };
     if (l == 0) HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_embed_norm(c, w->tok_emb, lw.attn_norm, s));
     else HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.attn_norm, s));
@@ -766,7 +773,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_qkv, r3, cfg.d_model));
     ga.k2_blocks = use_lora ? r3 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s,
-                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_qkv : nullptr));
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_qkv : nullptr, c->pdl));
     if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention_tc(c, kg, kv->map, l, s));
     if (dd.n_attn_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
     // O projection, added to the residual stream
@@ -774,20 +781,20 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_attn_out, lm->a_o, r1, n_q));
     ga.k2_blocks = use_lora ? r1 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s,
-                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_o : nullptr));
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_o : nullptr, c->pdl));
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.ffn_norm, s));
     // gate/up projection with SwiGLU
     ga.C = c->act; ga.N = 2 * cfg.d_ffn; ga.K = cfg.d_model; ga.ldc = cfg.d_ffn;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_gu, r2, cfg.d_model));
     ga.k2_blocks = use_lora ? r2 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s,
-                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_gu : nullptr));
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_gu : nullptr, c->pdl));
     // down projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = cfg.d_ffn; ga.ldc = cfg.d_model;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_act, lm->a_d, r1, cfg.d_ffn));
     ga.k2_blocks = use_lora ? r1 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s,
-                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_d : nullptr));
+                                         use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_d : nullptr, c->pdl));
   }
   float* pool_sum = pool ? static_cast<float*>(pool->arena) : nullptr;
   uint32_t* pool_meta = pool ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(pool->arena) +
@@ -800,6 +807,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     prof_end(pr);
     if (rc != HB_OK) return rc;
     launches += (dd.n_logit > 0) + (dd.n_pool_items > 0);
+    c->pdl = pdl_enabled;
   }
   if (dd.n_logit > 0) {
     if (c->lm_key != w->lm_head) {
@@ -810,10 +818,12 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.status = c->status;
     ga.b_kshift = 1;  // A holds (hi, lo) 64-column blocks: each weight k-block is used twice
     ga.M = dd.n_logit; ga.N = cfg.vocab; ga.K = 2 * cfg.d_model; ga.ldc = cfg.vocab; ga.C = out_logits;
-    HB_TRY(HB_CLASS_LM_HEAD, hb_gemm_launch(c->tm_logit_in, c->tm_lm, 128, HB_EPI_F32, ga, c->num_sms, s));
+    HB_TRY(HB_CLASS_LM_HEAD, hb_gemm_launch(c->tm_logit_in, c->tm_lm, 128, HB_EPI_F32, ga, c->num_sms, s, nullptr,
+                                            nullptr, c->pdl));
   }
 #undef HB_TRY
   c->last_launches = launches;
+  c->pdl = false;
   return HB_OK;
 }
 

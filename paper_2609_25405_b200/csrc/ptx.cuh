@@ -13,6 +13,16 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// ---- programmatic dependent launch -------------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may become resident while
+// the previous kernel of the stream is still draining.  grid_dep_wait() returns once that kernel has
+// completed and its writes are visible (at once when there is no such dependency);
+// grid_dep_launch() lets the next kernel of the stream do the same with respect to this one.  Every
+// kernel of the step calls both before it reads or writes global memory; only set-up that touches
+// the CTA's own shared memory and TMEM may precede the wait.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier --------------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));

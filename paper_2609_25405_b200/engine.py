@@ -4,6 +4,8 @@ batch unit of Section 3.2 (rows sorted by type: decode, prefill chunks, embeddin
 This is bookkeeping only.  The batch-composition policy is the caller's: `Engine.step`
 takes the list of (request, rows) the scheduler chose for this iteration.
 """
+import itertools
+
 import numpy as np
 import torch
 
@@ -37,35 +39,33 @@ def build_batch(entries, page_size):
     wants_logits).  Returns (Batch, order) with segments sorted by kind (stable) and
     logits / embedding rows numbered in segment order; order[i] = index into `entries`."""
     order = sorted(range(len(entries)), key=lambda i: entries[i]["kind"])
-    segs = np.zeros(len(entries), dtype=B.SEG_DTYPE)
-    toks, pages = [], []
-    n_l = n_e = 0
-    at = 0
-    for si, ei in enumerate(order):
-        e = entries[ei]
-        q = len(e["tokens"])
-        s = segs[si]
-        s["kind"] = e["kind"]
-        s["q_start"] = at
-        s["q_len"] = q
-        s["pos_start"] = e["pos_start"]
-        s["pt_start"] = len(pages)
-        s["pt_len"] = len(e["pages"])
-        s["pool_slot"] = e.get("pool_slot", -1)
-        s["pool_mode"] = e.get("pool_mode", B.POOL_NONE)
-        s["is_final"] = 1 if e.get("is_final") else 0
-        s["logits_row"] = -1
-        s["emb_row"] = -1
-        if e["kind"] == B.KIND_EMBED_CHUNK:
-            if e.get("is_final"):
-                s["emb_row"] = n_e
-                n_e += 1
-        elif e["kind"] == B.KIND_DECODE or e.get("is_final"):
-            s["logits_row"] = n_l
-            n_l += 1
-        toks.extend(int(t) for t in e["tokens"])
-        pages.extend(int(p) for p in e["pages"])
-        at += q
+    ents = [entries[i] for i in order]
+    n = len(ents)
+    # one Python pass collects plain lists; the structured array is filled column by column
+    kind = np.fromiter((e["kind"] for e in ents), dtype=np.int32, count=n)
+    q_len = np.fromiter((len(e["tokens"]) for e in ents), dtype=np.int32, count=n)
+    pt_len = np.fromiter((len(e["pages"]) for e in ents), dtype=np.int32, count=n)
+    final = np.fromiter((1 if e.get("is_final") else 0 for e in ents), dtype=np.int32, count=n)
+    segs = np.zeros(n, dtype=B.SEG_DTYPE)
+    segs["kind"] = kind
+    segs["q_len"] = q_len
+    segs["q_start"] = np.cumsum(q_len) - q_len
+    segs["pos_start"] = np.fromiter((e["pos_start"] for e in ents), dtype=np.int32, count=n)
+    segs["pt_len"] = pt_len
+    segs["pt_start"] = np.cumsum(pt_len) - pt_len
+    segs["pool_slot"] = np.fromiter((e.get("pool_slot", -1) for e in ents), dtype=np.int32, count=n)
+    segs["pool_mode"] = np.fromiter((e.get("pool_mode", B.POOL_NONE) for e in ents), dtype=np.int32, count=n)
+    segs["is_final"] = final
+    is_emb = kind == B.KIND_EMBED_CHUNK
+    wants_emb = is_emb & (final == 1)
+    wants_lg = ~is_emb & ((kind == B.KIND_DECODE) | (final == 1))
+    segs["emb_row"] = np.where(wants_emb, np.cumsum(wants_emb) - 1, -1)
+    segs["logits_row"] = np.where(wants_lg, np.cumsum(wants_lg) - 1, -1)
+    n_e, n_l = int(wants_emb.sum()), int(wants_lg.sum())
+    toks = np.fromiter(itertools.chain.from_iterable(e["tokens"] for e in ents), dtype=np.int32,
+                       count=int(q_len.sum()))
+    pages = np.fromiter(itertools.chain.from_iterable(e["pages"] for e in ents), dtype=np.int32,
+                        count=int(pt_len.sum()))
     return B.Batch(toks, segs, pages, n_l, n_e), order
 
 
@@ -95,7 +95,7 @@ class Engine:
         assert rows >= 1 and rows <= req.remaining()
         self._ensure_pages(req, req.n_done + rows)
         toks = req.tokens[req.n_done:req.n_done + rows]
-        e = dict(tokens=toks, pos_start=req.n_done, pages=list(req.pages))
+        e = dict(tokens=toks, pos_start=req.n_done, pages=req.pages)      # read by build_batch, not kept
         last = (req.n_done + rows == len(req.tokens))
         if req.kind == "embed":
             if req.slot < 0:
@@ -117,14 +117,14 @@ class Engine:
         self.ctx.mixed_step(batch, self.weights, self.kv, self.pool, self.out_logits, self.out_emb, stream,
                             lora=self.lora)
         lrows, erows = {}, {}
+        lg, em = batch.segs["logits_row"].tolist(), batch.segs["emb_row"].tolist()
         for si, ei in enumerate(order):
             req, n = work[ei]
             req.n_done += n
-            s = batch.segs[si]
-            if s["logits_row"] >= 0:
-                lrows[req] = int(s["logits_row"])
-            if s["emb_row"] >= 0:
-                erows[req] = int(s["emb_row"])
+            if lg[si] >= 0:
+                lrows[req] = lg[si]
+            if em[si] >= 0:
+                erows[req] = em[si]
                 req.finished = True
         return batch, lrows, erows
 

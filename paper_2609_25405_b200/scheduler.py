@@ -39,7 +39,7 @@ class IBS:
         self.a_e = 0
         self.a_g = 0
         self.Qe, self.Qg = deque(), deque()
-        self.running = []                   # generation requests in their decode phase
+        self.running = {}                   # generation requests in their decode phase (insertion-ordered set)
 
     # ---- queues ----
     def submit(self, work):
@@ -47,6 +47,12 @@ class IBS:
 
     def _weight(self, Q):
         return sum(w.remaining for w in Q)
+
+    def _remove(self, Q, w):
+        if Q and Q[0] is w:                 # the usual case: requests finish in arrival order
+            Q.popleft()
+        else:
+            Q.remove(w)
 
     # ---- Algorithm 2 ----
     def _schedule_running(self, budget):
@@ -112,14 +118,14 @@ class IBS:
             if w in self.running:
                 w.decode_left -= 1
                 if w.decode_left <= 0:
-                    self.running.remove(w)
+                    del self.running[w]
                     done.append(w)
                 continue
             w.remaining -= rows
             if w.remaining == 0:
-                (self.Qe if w.kind == "embed" else self.Qg).remove(w)
+                self._remove(self.Qe if w.kind == "embed" else self.Qg, w)
                 if w.kind == "gen" and w.decode_left > 0:
-                    self.running.append(w)
+                    self.running[w] = None
                 else:
                     done.append(w)
         return done

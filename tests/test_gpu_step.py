@@ -219,6 +219,44 @@ def test_buffered_max_head(weights):
     eng.close()
 
 
+def test_chunked_versus_own_single_pass_within_the_papers_printed_bounds(weights):
+    """The paper measures how well its chunked path reproduces its own single pass (appendix "Pooling
+    Equivalence": per head and chunk size the minimum cosine and the p99 relative L2 over 250
+    samples; tests/golden/pooling_equivalence.txt).  This path must do at least as well against ITS
+    own single pass, at the same chunk sizes, for every sampled text."""
+    import os
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Request
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "pooling_equivalence.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    modes = {"mean": B.POOL_MEAN, "cls": B.POOL_CLS, "wmean": B.POOL_WMEAN}
+    rng = np.random.default_rng(31)
+    texts = [synth.token_ids(rng, n, TINY.V) for n in (300, 777, 1500, 2048)]
+    eng = _engine(weights, n_pages=2 * 130 + 8, n_slots=4, max_tokens=2048, max_segs=8, max_pos=2048)
+
+    def embed(toks, sizes, mode):
+        r = Request("embed", toks, mode)
+        er = {}
+        for c in sizes:
+            _, _, er = eng.step([(r, c)])
+        torch.cuda.synchronize()
+        out = eng.out_emb[er[r]].cpu().numpy().astype(np.float64)
+        eng.release(r)
+        return out
+
+    single = {(h, i): embed(t, [len(t)], m) for h, m in modes.items() for i, t in enumerate(texts)}
+    for head, C, cos_min, _, _, _, l2_p99 in rows:
+        for i, t in enumerate(texts):
+            if len(t) <= int(C):
+                continue                                   # one chunk: nothing to compare
+            e = embed(t, synth.nominal_chunks(len(t), int(C)), modes[head])
+            ref = single[(head, i)]
+            assert float(e @ ref) >= float(cos_min), (head, C, len(t))
+            assert np.linalg.norm(e - ref) / np.linalg.norm(ref) <= float(l2_p99), (head, C, len(t))
+    assert eng.ctx.status_poll() == 0
+    eng.close()
+
+
 def test_long_chunks_take_the_tensor_core_attention_path(weights):
     """Chunks of more than 64 query rows run on the tcgen05 attention kernel (128-row tiles, ragged
     last tile, several key tiles, chunks that start inside a page); shorter remainders on the

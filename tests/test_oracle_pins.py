@@ -500,3 +500,30 @@ def test_fp32_oracle_close_to_fp64():
     a = T.embed(TINY, W, toks, "mean", dtype=np.float64)
     b = T.embed(TINY, W, toks, "mean", dtype=np.float32)
     assert np.max(np.abs(a - b)) < 1e-5
+
+
+# --------------------------------------------------------------------------
+# values the paper prints
+# --------------------------------------------------------------------------
+
+def _golden_rows(name):
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+    return [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+
+
+def test_printed_pooling_equivalence_bounds_hold_for_the_oracle():
+    """The paper's table of chunked-versus-single-pass agreement (appendix "Pooling Equivalence": min
+    cosine and p99 relative L2 per head and chunk size) is a ceiling any exact restatement must stay
+    under: the oracle's chunked form at the same chunk sizes, on texts of several lengths."""
+    cfg, W = MICRO, _w(MICRO, 4, std=0.2)
+    rng = np.random.default_rng(12)
+    texts = [synth.token_ids(rng, n, cfg.V) for n in (300, 1100)]
+    rows = _golden_rows("pooling_equivalence.txt")
+    assert len(rows) == 9
+    for head, C, cos_min, _, _, _, l2_p99 in rows:
+        for toks in texts:
+            ref = T.embed(cfg, W, toks, head)
+            e, _ = M.embed_chunked(cfg, W, toks, synth.nominal_chunks(len(toks), int(C)), head)
+            assert float(e @ ref) >= float(cos_min)
+            assert np.linalg.norm(e - ref) / np.linalg.norm(ref) <= float(l2_p99)

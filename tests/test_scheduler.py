@@ -36,7 +36,7 @@ def test_running_decodes_are_reserved_first():
     sch.submit(Work("embed", 100))
     batch = sch.schedule()
     n_run = len(sch.running)
-    assert [w for w, _ in batch[:n_run]] == sch.running and all(r == 1 for _, r in batch[:n_run])
+    assert [w for w, _ in batch[:n_run]] == list(sch.running) and all(r == 1 for _, r in batch[:n_run])
 
 
 def test_per_type_fcfs():
@@ -127,3 +127,18 @@ def test_chunking_raises_budget_fill():
     chunked = packing_fill(256, 64, chunked=True, n_iters=3000, seed=1)
     assert chunked > atomic
     assert 0.0 < atomic < 1.0 and chunked <= 1.0
+
+
+def test_printed_packing_simulation_direction():
+    """The paper's atomic-versus-chunked table (tests/golden/packing_simulation.txt): chunking raises
+    the budget fill.  The simulator's arrival process is not stated, so the printed sizes (8.8 % and
+    85.7 %) are not reproducible; the direction is, at the same B, C and request mix, under a load
+    that does not saturate the budget."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "packing_simulation.txt")
+    rows = {ln.split()[0]: float(ln.split()[1]) for ln in open(path) if ln.strip() and not ln.startswith("#")}
+    assert rows["chunked"] > rows["atomic"]
+    for seed in (1, 2, 3):
+        atomic = packing_fill(256, 64, chunked=False, n_iters=3000, seed=seed, arrivals_per_iter=0.5)
+        chunked = packing_fill(256, 64, chunked=True, n_iters=3000, seed=seed, arrivals_per_iter=0.5)
+        assert chunked > atomic + 0.02
