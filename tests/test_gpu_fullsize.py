@@ -6,7 +6,8 @@ bit for bit on the tiny shape, and here on one request run solo and inside the b
 
 Sampled per shape: two generation requests (prompt prefilled in chunks through the library
 itself, then teacher-forced decode steps) and two embedding requests (one single-chunk, one
-multi-chunk), last-token pooling as the configurations say.  The other rows are filler: decode
+multi-chunk) with last-token pooling as the configurations say, plus one multi-chunk request with
+mean pooling.  The other rows are filler: decode
 rows over contexts of random K/V and embedding chunks of random tokens.
 """
 import os
@@ -27,9 +28,9 @@ KV_SENTINEL = 0x7F7F
 CASES = {
     # shape, decode rows, filler ctx range, budget, chunk, sampled gen prompts, sampled embed lengths
     "cfg2-1b": dict(shape="1b", n_decode=32, ctx=(128, 1024), budget=2048, chunk=256,
-                    gen=(128, 600), emb=(200, 700), seed=1002, n_steps=4),
+                    gen=(128, 600), emb=(200, 700), emb_mean=(450,), seed=1002, n_steps=4),
     "cfg3-7b": dict(shape="7b", n_decode=64, ctx=(512, 4096), budget=4096, chunk=512,
-                    gen=(512, 1100), emb=(300, 700), seed=1003, n_steps=2),
+                    gen=(512, 1100), emb=(300, 700), emb_mean=(640,), seed=1003, n_steps=2),
 }
 
 
@@ -51,7 +52,7 @@ def test_fullsize_sampled_requests_match_oracle(name):
     max_pos = c["ctx"][1] + n_steps + 8
     n_dec = c["n_decode"]
     ctxs = rng.integers(c["ctx"][0], c["ctx"][1] + 1, size=n_dec - 2)
-    n_pages = int(sum((x + n_steps + P) // P + 1 for x in ctxs)) + 4 * (max_pos // P + 2) + \
+    n_pages = int(sum((x + n_steps + P) // P + 1 for x in ctxs)) + 5 * (max_pos // P + 2) + \
         n_steps * (c["budget"] // P + 80)
     eng = Engine(shape, dw, n_pages=n_pages, n_slots=256, max_tokens=c["budget"], max_segs=n_dec + 160,
                  max_pos=max_pos)
@@ -64,6 +65,9 @@ def test_fullsize_sampled_requests_match_oracle(name):
     # ---- sampled requests ----
     gens = [Request("gen", synth.token_ids(rng, n, shape.V)) for n in c["gen"]]
     embs = [Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_LAST) for n in c["emb"]]
+    # one multi-chunk request with mean pooling (the sweep configuration's head) next to the last-token ones
+    embs += [Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_MEAN) for n in c["emb_mean"]]
+    head = {B.POOL_LAST: "last", B.POOL_MEAN: "mean"}
     sampled_pages = {}
     for r in gens + embs:
         total = len(r.tokens) + n_steps + 1
@@ -91,7 +95,7 @@ def test_fullsize_sampled_requests_match_oracle(name):
         tk, lg = T.generate(shape, W, toks, n_steps, dtype=np.float32)
         ora_tok[g], ora_lg[g] = tk, lg
         assert n0 + n_steps <= max_pos
-    ora_emb = {e: T.embed(shape, W, e.tokens, "last", dtype=np.float32) for e in embs}
+    ora_emb = {e: T.embed(shape, W, e.tokens, head[e.pool_mode], dtype=np.float32) for e in embs}
 
     # ---- run: every step is filled to the token budget ----
     got_lg = {g: [] for g in gens}
@@ -180,5 +184,5 @@ def test_fullsize_sampled_requests_match_oracle(name):
         cnt, chunks = M.pool_counters_after(synth.nominal_chunks(len(r.tokens), chunk)) if r.kind == "embed" else (0, 0)
         if r.kind == "embed":
             meta = eng.pool.meta()[r.slot].cpu().numpy()
-            assert list(meta.astype(np.int64)) == [cnt, chunks, B.POOL_LAST, 1]
+            assert list(meta.astype(np.int64)) == [cnt, chunks, r.pool_mode, 1]
     eng.close()
