@@ -90,6 +90,8 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
         o.z = __uint_as_float(r[v * 4 + 2]);
         o.w = __uint_as_float(r[v * 4 + 3]);
         if constexpr (EPI == HB_EPI_RESID_F32) {
+          // (plain load: with split K these rows were written earlier in this launch, by another SM
+          // whose stores went to L2, or by this SM itself; this SM's L1 holds no older copy of them)
           const float4 old = *reinterpret_cast<const float4*>(out + v * 4);
           o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
         }
@@ -202,10 +204,14 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 
   const int m_tiles = (g.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (g.N + BN - 1) / BN;
-  // k_splits > 1 (thin adapter GEMMs only): every output tile is computed by k_splits work items,
-  // each over an equal share of the K blocks; the partial sums are combined in the epilogue.
+  // k_splits > 1: every output tile is computed by k_splits work items, each over an equal share of
+  // the K blocks.  Thin adapter GEMMs merge fp32 partials in split order; residual-update GEMMs add
+  // their shares to x one after the other, split s after split s - 1 (a fixed order, so a row's
+  // result does not depend on timing or on the batch).  Items are ordered split-major: every
+  // split-0 item precedes every split-1 item, and a worker takes its items in increasing order, so
+  // the item a waiting epilogue depends on is never queued behind an item that itself waits.
   const int mn_tiles = m_tiles * n_tiles;
-  const int k_splits = (EPI == HB_EPI_LORA_DOWN) ? g.k_splits : 1;
+  const int k_splits = (EPI == HB_EPI_LORA_DOWN || EPI == HB_EPI_RESID_F32) ? max(g.k_splits, 1) : 1;
   const int total_tiles = mn_tiles * k_splits;
   // K runs over the columns of (A, B) and then over g.k2_blocks more 64-column blocks of a second
   // operand pair (A2, B2): C = A B^T + A2 B2^T in one accumulation (the low-rank branch of an
@@ -362,6 +368,26 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           }
         }
       }
+      uint32_t* turn = nullptr;
+      if constexpr (EPI == HB_EPI_RESID_F32) {
+        if (k_splits > 1) {
+          // one turn word per (tile, CTA of the group, warp): these 32 rows of the tile are updated by
+          // split 0, then split 1, ...; the word holds the split whose turn it is
+          turn = g.split_counters + ((static_cast<size_t>(mn) * CG + rank) * 4 + quarter);
+          if (split > 0) {
+            uint32_t okw = 1u;
+            if (lane == 0) {
+              const uint64_t t0 = global_ns();
+              while (ld_acquire_u32(turn) != static_cast<uint32_t>(split)) {
+                if (*abort_flag || global_ns() - t0 > WAIT_LIMIT_NS) { okw = 0u; break; }
+                __nanosleep(64);
+              }
+            }
+            okw = __shfl_sync(0xffffffffu, okw, 0);
+            if (!okw) { ok = false; give_up(); break; }
+          }
+        }
+      }
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         uint32_t r[32];
@@ -383,6 +409,15 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       if (lane == 0) {
         if constexpr (CG == 2) mbar_arrive_cluster(map_to_rank(tempty_bar(acc), 0u));
         else mbar_arrive(tempty_bar(acc));
+      }
+      if constexpr (EPI == HB_EPI_RESID_F32) {
+        if (turn != nullptr) {
+          // this warp's rows of x are written: pass the turn on (the last split leaves the word at 0
+          // for the next launch)
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) st_release_u32(turn, split + 1 == k_splits ? 0u : static_cast<uint32_t>(split + 1));
+        }
       }
       if constexpr (EPI == HB_EPI_LORA_DOWN) {
         if (k_splits > 1) {
@@ -475,7 +510,8 @@ int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap
   }
   const int m_tiles = (a.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (a.N + BN - 1) / BN;
-  int workers = m_tiles * n_tiles * ((EPI == HB_EPI_LORA_DOWN && a.k_splits > 1) ? a.k_splits : 1);
+  int workers = m_tiles * n_tiles *
+                (((EPI == HB_EPI_LORA_DOWN || EPI == HB_EPI_RESID_F32) && a.k_splits > 1) ? a.k_splits : 1);
   if (workers > num_sms / CG) workers = num_sms / CG;
   if (workers < 1) return HB_OK;
   cudaLaunchConfig_t cfg = {};
@@ -544,6 +580,20 @@ int hb_gemm_pick_bn(int M, int N, int num_sms) {
   return (e128 * 0.92 > e256) ? 128 : 256;
 }
 
+// Residual-update GEMMs may split K in two when that fills the last wave of CTA pairs much better
+// (7B shape at 4096 rows: 256 tiles on 74 pairs is 3.46 waves, 512 half-K items is 6.92).  The choice
+// depends on the problem shape alone, never on the batch at hand.
+int hb_gemm_pick_ksplit(int M, int N, int K, int variant, int num_sms) {
+  if (variant != HB_GEMM_PAIR256) return 1;
+  const long workers = num_sms / 2;
+  // each half must still be long enough to hide an epilogue that reads and writes the whole tile
+  if (workers < 1 || K < 128 * BK) return 1;
+  const long tiles = static_cast<long>((M + 255) / 256) * ((N + 255) / 256);
+  const double e1 = static_cast<double>(tiles) / (((tiles + workers - 1) / workers) * workers);
+  const double e2 = static_cast<double>(2 * tiles) / (((2 * tiles + workers - 1) / workers) * workers);
+  return e2 > e1 * 1.05 ? 2 : 1;
+}
+
 int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : variant; }
 
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,
@@ -551,6 +601,7 @@ int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, 
   if ((a.k2_blocks > 0) != (tmA2 != nullptr && tmB2 != nullptr) || a.k2_blocks < 0) return HB_ERR_BAD_ARG;
   if (epi == HB_EPI_LORA_DOWN && (a.k_splits < 1 || (a.k_splits > 1 && (!a.split_part || !a.split_counters))))
     return HB_ERR_BAD_ARG;
+  if (epi == HB_EPI_RESID_F32 && a.k_splits > 1 && !a.split_counters) return HB_ERR_BAD_ARG;
   // without an extension the second pair is never read; pass the first so the parameters are valid maps
   const CUtensorMap& a2 = tmA2 ? *tmA2 : tmA;
   const CUtensorMap& b2 = tmB2 ? *tmB2 : tmB;

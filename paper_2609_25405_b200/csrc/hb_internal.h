@@ -117,9 +117,10 @@ struct GemmArgs {
   // HB_EPI_LORA_DOWN only
   float alpha;
   int32_t first_row;
-  int32_t k_splits;          // work items per output tile (>= 1), each over an equal share of the K blocks
-  float* split_part;         // [k_splits, M, N] partial sums (k_splits > 1)
-  uint32_t* split_counters;  // [tiles * 4] arrival counters, zero between launches
+  // HB_EPI_LORA_DOWN and HB_EPI_RESID_F32
+  int32_t k_splits;          // work items per output tile (0 or 1 = no split), each over an equal share of the K blocks
+  float* split_part;         // LORA_DOWN: [k_splits, M, N] partial sums (k_splits > 1)
+  uint32_t* split_counters;  // LORA_DOWN: [tiles * 4] arrival counters; RESID_F32: [tiles * CG * 4] turn words; zero between launches
   // HB_EPI_QKV_ROPE only
   const int32_t* row_pos;   // [M] position of each row inside its request
   const int32_t* row_page;  // [M] physical page that holds that position
@@ -138,6 +139,7 @@ int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t 
 constexpr int HB_GEMM_PAIR256 = 512;
 int hb_gemm_pick_bn(int M, int N, int num_sms);
 int hb_gemm_box_rows(int variant);
+int hb_gemm_pick_ksplit(int M, int N, int K, int variant, int num_sms);
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,
                    const CUtensorMap* tmB2 = nullptr, bool pdl = false);
@@ -192,6 +194,8 @@ struct hb_ctx {
   float* lora_part;         // [HB_LORA_K_SPLITS, max_tokens, HB_LORA_U_COLS] split-K partial sums
   uint32_t* lora_counters;  // [n_lora_counters] arrival counters of the split-K merge
   int32_t n_lora_counters;
+  uint32_t* resid_turns;    // [n_resid_turns] turn words of the split-K residual GEMMs (zero between launches)
+  int32_t n_resid_turns;
   __half* logit_in;         // [max_logit_rows, 2d] hi/lo fp16 split of final hidden rows
   float* rope_cos;          // [max_pos, Dh/2]
   float* rope_sin;
@@ -214,6 +218,7 @@ struct hb_ctx {
     const void* key[4];
     CUtensorMap qkv, o, gu, down;
     int bn_qkv, bn_o, bn_gu, bn_down;
+    int ks_o, ks_down;
   };
   std::vector<WMaps> wmaps;
   // cached adapter tensor maps: down factors (B operand of the thin GEMMs), up factors (second B

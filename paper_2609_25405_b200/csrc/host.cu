@@ -44,10 +44,10 @@ struct Carve {
 };
 
 struct Layout {
-  size_t x, h, q, attn_out, act, lora_u, lora_part, lora_counters, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
+  size_t x, h, q, attn_out, act, lora_u, lora_part, lora_counters, resid_turns, logit_in, rope_cos, rope_sin, attn_part, pool_part, counters, attn_counters,
       status, desc;
   size_t total, desc_cap, attn_part_floats, pool_part_floats;
-  int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items;
+  int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items, n_resid_turns;
 };
 
 Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids) {
@@ -66,6 +66,8 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.lora_u = cv.take(rows * HB_LORA_U_COLS * 2);
   L.lora_part = cv.take(static_cast<size_t>(HB_LORA_K_SPLITS) * rows * HB_LORA_U_COLS * 4);
   L.lora_counters = cv.take((rows / 128) * 2 * 4 * 4);
+  L.n_resid_turns = static_cast<int32_t>((rows / 128) * ((static_cast<size_t>(c.d_model) + 255) / 256) * 4);
+  L.resid_turns = cv.take(static_cast<size_t>(L.n_resid_turns) * 4);
   L.logit_in = cv.take(lrows * 2 * c.d_model * 2);
   L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
   L.rope_sin = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
@@ -252,6 +254,8 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->lora_part = reinterpret_cast<float*>(c->ws + lay.lora_part);
   c->lora_counters = reinterpret_cast<uint32_t*>(c->ws + lay.lora_counters);
   c->n_lora_counters = static_cast<int32_t>((lay.rows_pad / 128) * 2 * 4);
+  c->resid_turns = reinterpret_cast<uint32_t*>(c->ws + lay.resid_turns);
+  c->n_resid_turns = lay.n_resid_turns;
   c->logit_in = reinterpret_cast<__half*>(c->ws + lay.logit_in);
   c->rope_cos = reinterpret_cast<float*>(c->ws + lay.rope_cos);
   c->rope_sin = reinterpret_cast<float*>(c->ws + lay.rope_sin);
@@ -729,6 +733,8 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
       wm.bn_o = hb_gemm_pick_bn(c->max_tokens, cfg.d_model, c->num_sms);
       wm.bn_gu = hb_gemm_pick_bn(c->max_tokens, 2 * cfg.d_ffn, c->num_sms);
       wm.bn_down = wm.bn_o;
+      wm.ks_o = hb_gemm_pick_ksplit(c->max_tokens, cfg.d_model, n_q, wm.bn_o, c->num_sms);
+      wm.ks_down = hb_gemm_pick_ksplit(c->max_tokens, cfg.d_model, cfg.d_ffn, wm.bn_down, c->num_sms);
       if ((rc = hb_tmap_2d_bf16(&wm.qkv, lw.wqkv, n_qkv, cfg.d_model, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
       if ((rc = hb_tmap_2d_bf16(&wm.o, lw.wo, cfg.d_model, n_q, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
       if ((rc = hb_tmap_2d_bf16(&wm.gu, lw.w_gate_up, 2ull * cfg.d_ffn, cfg.d_model, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
@@ -803,6 +809,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     }
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
+    ga.k_splits = wm.ks_o; ga.split_counters = c->resid_turns;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_attn_out, lm->a_o, r1, n_q));
     ga.k2_blocks = use_lora ? r1 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s,
@@ -810,12 +817,14 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.ffn_norm, s));
     // gate/up projection with SwiGLU
     ga.C = c->act; ga.N = 2 * cfg.d_ffn; ga.K = cfg.d_model; ga.ldc = cfg.d_ffn;
+    ga.k_splits = 1;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_gu, r2, cfg.d_model));
     ga.k2_blocks = use_lora ? r2 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s,
                                          use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_gu : nullptr, c->pdl));
     // down projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = cfg.d_ffn; ga.ldc = cfg.d_model;
+    ga.k_splits = wm.ks_down; ga.split_counters = c->resid_turns;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_act, lm->a_d, r1, cfg.d_ffn));
     ga.k2_blocks = use_lora ? r1 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s,
@@ -894,7 +903,8 @@ int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
     if (cudaMemsetAsync(c->attn_counters, 0, static_cast<size_t>(c->max_segs) * c->cfg.n_kv_heads * 4, s) !=
             cudaSuccess ||
         cudaMemsetAsync(c->counters, 0, static_cast<size_t>(c->n_counters) * 4, s) != cudaSuccess ||
-        cudaMemsetAsync(c->lora_counters, 0, static_cast<size_t>(c->n_lora_counters) * 4, s) != cudaSuccess)
+        cudaMemsetAsync(c->lora_counters, 0, static_cast<size_t>(c->n_lora_counters) * 4, s) != cudaSuccess ||
+        cudaMemsetAsync(c->resid_turns, 0, static_cast<size_t>(c->n_resid_turns) * 4, s) != cudaSuccess)
       return HB_ERR_CUDA;
     if (cudaMemsetAsync(c->status, 0, 4, s) != cudaSuccess) return HB_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;
@@ -945,6 +955,14 @@ int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t
   GemmArgs ga = {};
   ga.C = C; ga.M = M; ga.N = N; ga.K = K; ga.b_kshift = 0; ga.status = c->status;
   ga.ldc = (epilogue == HB_EPI_SWIGLU) ? N / 2 : N;
+  if (epilogue == HB_EPI_RESID_F32) {
+    const int ks = hb_gemm_pick_ksplit(M, N, K, bn, c->num_sms);
+    const long turns = static_cast<long>((M + 255) / 256) * ((N + 255) / 256) * 2 * 4;
+    if (ks > 1 && turns <= c->n_resid_turns) {
+      ga.k_splits = ks;
+      ga.split_counters = c->resid_turns;
+    }
+  }
   return hb_gemm_launch(ta, tb, bn, epilogue, ga, c->num_sms, static_cast<cudaStream_t>(stream));
 }
 

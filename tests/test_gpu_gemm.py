@@ -79,6 +79,35 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
         assert np.all(got[M] == 768.0)
 
 
+@pytest.mark.parametrize("M", [4096, 3900])
+def test_residual_gemm_with_split_k_is_exact_to_tolerance_and_deterministic(M):
+    """At the 7B projection shape the residual-update GEMM splits K in two (512 half-K work items fill
+    the 74 CTA pairs far better than 256 tiles); the halves add to x in a fixed order.  Checked against
+    the oracle's definition, the untouched row after the last one, and bitwise equality of two runs."""
+    from paper_2609_25405_b200 import binding as B
+    shape = synth.SHAPES["7b"]
+    c = B.Context(B.model_cfg(shape, 64), 4096, 8, 64)
+    N, K = 4096, 8192
+    rng = np.random.default_rng(M)
+    A = _f16_exact(rng, (M, K), 1.0)
+    Bm = _bf16_exact(rng, (N, K), 0.05)
+    dA, dB = torch.from_numpy(A.astype(np.float16)).cuda(), B.pack_f16_(B.bf16_from_f32(Bm))
+    C0 = rng.standard_normal((M + 1, N), dtype=np.float32)
+    outs = []
+    for _ in range(2):
+        out = torch.from_numpy(C0.copy()).cuda()
+        c.gemm(dA, dB, out, M, N, K, B.EPI_RESID_F32)
+        assert c.status_poll() == 0
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1])
+    got = outs[0].cpu().numpy().astype(np.float64)
+    ref = ops.projection(A, Bm, "resid", C0[:M])
+    scale = 0.05 * np.sqrt(K)
+    assert np.max(np.abs(got[:M] - ref)) <= 2e-5 * scale * np.sqrt(K) + 1e-5
+    assert np.array_equal(got[M], C0[M].astype(np.float64))
+    c.close()
+
+
 def test_weights_pack_f16_matches_round_to_nearest(ctx):
     """bf16 -> fp16 repack: exact in the fp16 normal range, round-to-nearest on the subnormal grid,
     saturating above 65504; in place."""
