@@ -29,8 +29,9 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) per launch of the projection GEMM at the 7B shape, T = 4096, mean of the four
 # projections of a layer, from the ncu capture summarised in profiles/gemm_tcgen05_cfg3-7b_layers2.md
-# (QKV 128.4 MB, O 169.5 MB, gate/up 403.1 MB, down 736.2 MB; algorithmic 134 / 201 / 386 / 369 MB)
-NCU_GEMM_TRAFFIC_BYTES = {"7b": 359.3e6}
+# (QKV 126.5 MB, O 171.7 MB, gate/up 420.7 MB, down 807.6 MB; algorithmic 134 / 201 / 386 / 497 MB, the last
+# with the second pass over x that the split-K down projection makes)
+NCU_GEMM_TRAFFIC_BYTES = {"7b": 381.6e6}
 
 
 def load_peaks():
