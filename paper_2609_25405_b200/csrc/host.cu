@@ -800,8 +800,10 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
       c->pdl = false;
       if ((rc = hb_launch_attention_tc(c, kg, kv->map, l, ex->side)) != HB_OK) return rc;
       if (cudaEventRecord(ex->ev_join, ex->side) != cudaSuccess) return HB_ERR_CUDA;
-      if ((rc = hb_launch_attention(c, kg, kv->map, l, s)) != HB_OK) return rc;
+      rc = hb_launch_attention(c, kg, kv->map, l, s);
+      // join even if the second launch failed: nothing later on `s` may overtake the side stream
       if (cudaStreamWaitEvent(s, ex->ev_join, 0) != cudaSuccess) return HB_ERR_CUDA;
+      if (rc != HB_OK) return rc;
       launches += 2;
     } else {
       if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention_tc(c, kg, kv->map, l, s));
