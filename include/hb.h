@@ -346,6 +346,13 @@ enum {
 HB_API int hb_gemm(hb_ctx* ctx, const void* A, const void* B, void* C, int32_t M, int32_t N,
             int32_t K, int32_t epilogue, void* stream);
 
+/* hb_gemm with a second operand pair accumulated after the first:
+ * C = epilogue(A * B^T + A2 * B2^T), A2 fp16 [M,K2], B2 fp16 [N,K2], K2 a
+ * multiple of 64.  This is how an adapted projection adds its low-rank branch
+ * (hb_mixed_step_lora): A2 = the rows' rank-r activations, B2 = the up factor. */
+HB_API int hb_gemm_pair(hb_ctx* ctx, const void* A, const void* B, const void* A2, const void* B2, void* C,
+                 int32_t M, int32_t N, int32_t K, int32_t K2, int32_t epilogue, void* stream);
+
 /* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
  * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of
  * the chunk's rows, then

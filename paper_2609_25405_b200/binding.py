@@ -98,6 +98,7 @@ _sig = {
     "hb_pool_chunk": [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P],
     "hb_pool_chunk_noalloc": [_P, _P, C.c_int32, C.c_int32, C.c_float, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P,
                               _P],
+    "hb_gemm_pair": [_P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
     "hb_status_poll": [_P, _P, C.POINTER(C.c_uint32)],
     "hb_last_launch_count": [_P, C.POINTER(C.c_int32)],
     "hb_selftest_wait_expiry": [_P, C.c_uint32, _P],
@@ -492,6 +493,11 @@ class Context:
     def argmax(self, logits, n_rows, out_tokens, stream=None):
         check(lib.hb_argmax(self.handle, C.c_void_p(logits.data_ptr()), n_rows,
                             C.c_void_p(out_tokens.data_ptr()), _stream_ptr(stream)), "hb_argmax")
+
+    def gemm_pair(self, A, B, A2, B2, Cout, M, N, K, K2, epilogue, stream=None):
+        check(lib.hb_gemm_pair(self.handle, C.c_void_p(A.data_ptr()), C.c_void_p(B.data_ptr()),
+                               C.c_void_p(A2.data_ptr()), C.c_void_p(B2.data_ptr()), C.c_void_p(Cout.data_ptr()),
+                               M, N, K, K2, epilogue, _stream_ptr(stream)), "hb_gemm_pair")
 
     def gemm(self, A, B, Cout, M, N, K, epilogue, stream=None):
         check(lib.hb_gemm(self.handle, C.c_void_p(A.data_ptr()), C.c_void_p(B.data_ptr()),

@@ -944,18 +944,29 @@ int hb_last_launch_count(const hb_ctx* c, int32_t* out_count) {
 
 int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int32_t epilogue,
             void* stream) {
+  return hb_gemm_pair(c, A, B, nullptr, nullptr, C, M, N, K, 0, epilogue, stream);
+}
+
+int hb_gemm_pair(hb_ctx* c, const void* A, const void* B, const void* A2, const void* B2, void* C, int32_t M,
+                 int32_t N, int32_t K, int32_t K2, int32_t epilogue, void* stream) {
   if (!c || !A || !B || !C || M < 1 || N < 8 || K < 8 || (N & 7) || (K & 7)) return HB_ERR_BAD_ARG;
   if (epilogue < HB_EPI_F16 || epilogue > HB_EPI_SWIGLU) return HB_ERR_BAD_ARG;
   if (epilogue == HB_EPI_SWIGLU && (N & 15)) return HB_ERR_BAD_ARG;
   if (reinterpret_cast<uintptr_t>(C) & 15u) return HB_ERR_BAD_ARG;
+  if (K2 < 0 || (K2 & 63) || ((K2 > 0) != (A2 != nullptr && B2 != nullptr))) return HB_ERR_BAD_ARG;
   const int bn = hb_gemm_pick_bn(M, N, c->num_sms);
-  CUtensorMap ta, tb;
+  CUtensorMap ta, tb, ta2, tb2;
   int rc = hb_tmap_2d_bf16(&ta, A, M, K, 128);
   if (rc != HB_OK) return rc;
   rc = hb_tmap_2d_bf16(&tb, B, N, K, hb_gemm_box_rows(bn));
   if (rc != HB_OK) return rc;
+  if (K2 > 0) {
+    if ((rc = hb_tmap_2d_bf16(&ta2, A2, M, K2, 128)) != HB_OK) return rc;
+    if ((rc = hb_tmap_2d_bf16(&tb2, B2, N, K2, hb_gemm_box_rows(bn))) != HB_OK) return rc;
+  }
   GemmArgs ga = {};
   ga.C = C; ga.M = M; ga.N = N; ga.K = K; ga.b_kshift = 0; ga.status = c->status;
+  ga.k2_blocks = K2 / 64;
   ga.ldc = (epilogue == HB_EPI_SWIGLU) ? N / 2 : N;
   if (epilogue == HB_EPI_RESID_F32) {
     const int ks = hb_gemm_pick_ksplit(M, N, K, bn, c->num_sms);
@@ -965,7 +976,8 @@ int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t
       ga.split_counters = c->resid_turns;
     }
   }
-  return hb_gemm_launch(ta, tb, bn, epilogue, ga, c->num_sms, static_cast<cudaStream_t>(stream));
+  return hb_gemm_launch(ta, tb, bn, epilogue, ga, c->num_sms, static_cast<cudaStream_t>(stream),
+                        K2 > 0 ? &ta2 : nullptr, K2 > 0 ? &tb2 : nullptr);
 }
 
 }  // extern "C"

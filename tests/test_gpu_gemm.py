@@ -79,6 +79,51 @@ def test_gemm_matches_oracle(ctx, M, N, K, epi):
         assert np.all(got[M] == 768.0)
 
 
+@pytest.mark.parametrize("M,N,K,K2", [(300, 328, 200, 64), (68, 768, 256, 192), (2500, 3072, 256, 128), (1030, 4160, 128, 64)])
+@pytest.mark.parametrize("epi", ["f32", "resid", "swiglu"])
+def test_gemm_with_second_operand_pair(ctx, M, N, K, K2, epi):
+    """C = epilogue(A B^T + A2 B2^T): the second pair runs as extra K blocks into the same accumulator
+    (the adapters' low-rank branch).  The definition is one product over the concatenated K."""
+    from paper_2609_25405_b200 import binding as B
+    if epi == "swiglu" and N % 16:
+        pytest.skip("swiglu needs N % 16 == 0")
+    rng = np.random.default_rng(M + N + K + K2)
+    A, A2 = _f16_exact(rng, (M, K), 1.0), _f16_exact(rng, (M, K2), 1.0)
+    Bm, B2 = _bf16_exact(rng, (N, K), 0.05), _bf16_exact(rng, (N, K2), 0.05)
+    dA, dA2 = torch.from_numpy(A.astype(np.float16)).cuda(), torch.from_numpy(A2.astype(np.float16)).cuda()
+    dB, dB2 = B.pack_f16_(B.bf16_from_f32(Bm)), B.pack_f16_(B.bf16_from_f32(B2))
+    Ac, Bc = np.concatenate([A, A2], axis=1), np.concatenate([Bm, B2], axis=1)
+    scale = 0.05 * np.sqrt(K + K2)
+    if epi == "f32":
+        out = torch.full((M + 1, N), 768.0, dtype=torch.float32, device="cuda")
+        ctx.gemm_pair(dA, dB, dA2, dB2, out, M, N, K, K2, B.EPI_F32)
+        ref, tol = ops.projection(Ac, Bc, "plain"), 2e-5 * scale * np.sqrt(K + K2) + 1e-6
+    elif epi == "resid":
+        C0 = rng.standard_normal((M + 1, N), dtype=np.float32)
+        out = torch.from_numpy(C0.copy()).cuda()
+        ctx.gemm_pair(dA, dB, dA2, dB2, out, M, N, K, K2, B.EPI_RESID_F32)
+        ref, tol = ops.projection(Ac, Bc, "resid", C0[:M]), 2e-5 * scale * np.sqrt(K + K2) + 1e-5
+    else:
+        out = torch.full((M + 1, N // 2), 768.0, dtype=torch.float16, device="cuda")
+        ctx.gemm_pair(dA, dB, dA2, dB2, out, M, N, K, K2, B.EPI_SWIGLU)
+        ref, tol = ops.projection(Ac, Bc, "swiglu"), None
+    assert ctx.status_poll() == 0
+    got = out.float().cpu().numpy().astype(np.float64)
+    if tol is None:
+        err = np.abs(got[:M] - ref)
+        assert np.all(err <= np.abs(ref) * 2.0 ** -10 + 2e-5 * scale * np.sqrt(K + K2) + 1e-6), err.max()
+    else:
+        assert np.max(np.abs(got[:M] - ref)) <= tol
+    # the second pair must matter, and a zero second operand must reproduce the plain GEMM bit for bit
+    base = torch.zeros_like(out) if epi != "resid" else torch.from_numpy(C0.copy()).cuda()
+    ctx.gemm(dA, dB, base, M, N, K, {"f32": B.EPI_F32, "resid": B.EPI_RESID_F32, "swiglu": B.EPI_SWIGLU}[epi])
+    zero = torch.zeros_like(dA2)
+    again = torch.zeros_like(out) if epi != "resid" else torch.from_numpy(C0.copy()).cuda()
+    ctx.gemm_pair(dA, dB, zero, dB2, again, M, N, K, K2, {"f32": B.EPI_F32, "resid": B.EPI_RESID_F32, "swiglu": B.EPI_SWIGLU}[epi])
+    torch.cuda.synchronize()
+    assert torch.equal(base[:M], again[:M]) and not torch.equal(base[:M], out[:M])
+
+
 @pytest.mark.parametrize("M", [4096, 3900])
 def test_residual_gemm_with_split_k_is_exact_to_tolerance_and_deterministic(M):
     """At the 7B projection shape the residual-update GEMM splits K in two (512 half-K work items fill
