@@ -71,8 +71,10 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   auto kv_full = [&](int s) { return bar_s + 8u * s; };
   auto kv_empty = [&](int s) { return bar_s + 8u * (C::STAGES + s); };
   const uint32_t s_full = bar_s + 8u * (2 * C::STAGES), s_empty = bar_s + 8u * (2 * C::STAGES + 1);
-  const uint32_t q_ready = bar_s + 8u * (2 * C::STAGES + 2), p_ready = bar_s + 8u * (2 * C::STAGES + 4),
-                 pv_done = bar_s + 8u * (2 * C::STAGES + 5);
+  // P is handed over in two halves (keys 0-31, then 32-63) so that the first half of P V is issued
+  // while the softmax threads are still producing the second
+  const uint32_t q_ready = bar_s + 8u * (2 * C::STAGES + 2), p_ready2 = bar_s + 8u * (2 * C::STAGES + 3),
+                 p_ready = bar_s + 8u * (2 * C::STAGES + 4), pv_done = bar_s + 8u * (2 * C::STAGES + 5);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -88,6 +90,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
     mbar_init(s_empty, 4);
     mbar_init(q_ready, 4);
     mbar_init(p_ready, 4);
+    mbar_init(p_ready2, 4);
     mbar_init(pv_done, 1);
     *abort_flag = 0u;
     mbar_init_fence();
@@ -175,16 +178,20 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
         // S_{j+1} may start as soon as the softmax warps have read S_j out of TMEM
         if (j + 1 < n_tiles) ok = issue_s(j + 1);
         if (!ok) break;
-        if (!mbar_wait(p_ready, static_cast<uint32_t>(j & 1), abort_flag, WAIT_NS)) break;
-        tc_fence_after();
         const uint32_t kv_tile = ring_s + (j % C::STAGES) * 2 * C::KV_HALF;
+        bool got = true;
 #pragma unroll
         for (int ks = 0; ks < BN / 16; ++ks) {   // one page (16 keys = two 8-key groups) per k-step
+          if (ks == 0 || ks == BN / 32) {        // each half of P has its own barrier
+            if (!mbar_wait(ks == 0 ? p_ready : p_ready2, static_cast<uint32_t>(j & 1), abort_flag, WAIT_NS)) { got = false; break; }
+            tc_fence_after();
+          }
           const uint64_t ad = make_desc(p_s + ks * 32, 16, 1024);
           // V is the MN-major B operand: 64-column halves 1024 B apart, 8-key groups GROUP_BYTES apart
           const uint64_t bd = make_desc(kv_tile + ks * C::PAGE_BYTES + C::V_OFF, 1024, C::GROUP_BYTES);
           umma_ss(tmem + static_cast<uint32_t>(C::O_COL), ad, bd, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
         }
+        if (!got) break;
         umma_commit(kv_empty(j % C::STAGES));
         umma_commit(pv_done);
       }
@@ -236,12 +243,16 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
       if (lane == 0) mbar_arrive(s_empty);
       // row maximum of the raw scores; masking only on tiles that touch the diagonal or the end of the keys
       const bool need_mask = (key_base + BN - 1 > pos) || (key_base + BN > it.key1);
-      float mx = -INFINITY;
+      // (eight independent running maxima: a single chain of 64 dependent compares costs ~250 cycles
+      // on a warp that has its scheduler to itself)
+      float mx8[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) mx8[q] = -INFINITY;
       if (!need_mask) {
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[h][i]));
+          for (int i = 0; i < 32; ++i) mx8[i & 7] = fmaxf(mx8[i & 7], __uint_as_float(sr[h][i]));
       } else {
         const int last = min(pos, it.key1 - 1) - key_base;   // last visible column of this row in the tile
 #pragma unroll
@@ -249,9 +260,10 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             if (h * 32 + i > last) sr[h][i] = 0xff800000u;   // -inf
-            mx = fmaxf(mx, __uint_as_float(sr[h][i]));
+            mx8[i & 7] = fmaxf(mx8[i & 7], __uint_as_float(sr[h][i]));
           }
       }
+      float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])), fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
       mx *= p.scale_log2;   // scores enter the exponent as s * log2(e) / sqrt(Dh)
       const float m_new = fmaxf(m_used, mx);
       const bool grow = (m_new > m_used + 8.0f) || (m_used == -INFINITY && m_new > -INFINITY);
@@ -277,23 +289,8 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
       }
       const float neg_ms = (m_used == -INFINITY) ? 0.0f : -m_used;
       // probabilities p = 2^(s * scale - m) -> fp16 P row in shared memory (K-major, 128-byte swizzle)
-      uint8_t* prow = smem + C::RING + rr * 128;
-      float sum = 0.0f;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        uint32_t pk[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int i = c * 8 + e * 2;
-          const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i >> 5][i & 31]), p.scale_log2, neg_ms));
-          const float p1 = ex2_approx(fmaf(__uint_as_float(sr[(i + 1) >> 5][(i + 1) & 31]), p.scale_log2, neg_ms));
-          sum += p0 + p1;
-          pk[e] = pack_half2(p0, p1);
-        }
-        *reinterpret_cast<uint4*>(prow + ((c ^ (rr & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      }
-      l += sum;
       // keys past the end of the request hold stale bytes: zero those V rows (0 * garbage must stay 0)
+      // before any part of P is handed over
       const int valid_keys = it.key1 - key_base;
       if (valid_keys < BN) {
         uint8_t* kv_gen = smem + (j % C::STAGES) * 2 * C::KV_HALF;
@@ -305,10 +302,28 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
               make_uint4(0u, 0u, 0u, 0u);
         }
       }
-      fence_async_smem();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(p_ready);
+      uint8_t* prow = smem + C::RING + rr * 128;
+      float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};   // fixed association, four short chains
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int i = c * 8 + e * 2;
+          const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i >> 5][i & 31]), p.scale_log2, neg_ms));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(sr[(i + 1) >> 5][(i + 1) & 31]), p.scale_log2, neg_ms));
+          sum4[e] += p0 + p1;
+          pk[e] = pack_half2(p0, p1);
+        }
+        *reinterpret_cast<uint4*>(prow + ((c ^ (rr & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        if (c == 3 || c == 7) {   // keys 0-31 (then 32-63) of this warp's rows are in shared memory
+          fence_async_smem();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(c == 3 ? p_ready : p_ready2);
+        }
+      }
+      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
     }
     // ---- epilogue: O / l -> fp16 ----
     if (ok && n_tiles > 0 && wait_w(pv_done, static_cast<uint32_t>((n_tiles - 1) & 1))) {
