@@ -23,7 +23,8 @@
 
 namespace {
 
-constexpr int ATT_THREADS = 128;
+constexpr int ATT_THREADS = 160;   // four compute warps + one warp whose lane 0 drives TMA
+constexpr int ATT_COMPUTE = 128;
 constexpr int TILE_KEYS = 64;
 constexpr int TILE_ROWS = 64;
 constexpr int STAGES = 3;
@@ -198,8 +199,13 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     for (int pi = 0; pi < TILE_KEYS / 16; ++pi) ids[pi] = (pi0 + pi < n_blk) ? pg_s[pi0 + pi] : 0;
     issue_pages(kt, ids);
   };
+  // The thread that talks to TMA sits in a warp of its own: requesting a tile (page ids, four copies,
+  // the proxy fence) takes ~650 cycles, which on a compute warp made that warp the one every block
+  // barrier waited for.
+  const bool prod = (tid == ATT_COMPUTE);
+  const bool compute = (warp < ATT_COMPUTE / 32);
   int issued = 0, bad = 0;
-  if (tid == 0) {
+  if (prod) {
     for (int st = 0; st < STAGES; ++st) mbar_init(bar_s + 8u * st, 1);
     mbar_init_fence();
     // the first tiles are requested right away, with page ids read straight from global memory, so
@@ -235,7 +241,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   }
   cp_async_commit();
   if (__syncthreads_or(bad)) {  // also publishes the barrier initialisation and the page ids
-    if (tid == 0) {
+    if (prod) {
       atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
       for (int st = 0; st < issued; ++st) mbar_wait(bar_s + 8u * st, 0u, nullptr, ATT_WAIT_NS);   // copies already requested must land
     }
@@ -269,11 +275,11 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   cp_async_wait<0>();
   for (int kt = 0; kt < n_tiles; ++kt) {
     if (__syncthreads_or(failed)) { failed = 1; break; }   // everyone is done with tile kt - 1 (and Q landed)
-    if (tid == 0 && kt > 0) {   // at kt = 0 the last stage still holds Q
+    if (prod && kt > 0) {   // at kt = 0 the last stage still holds Q
       fence_async_smem();  // stages were read / patched by generic accesses
       for (; issued < n_tiles && issued < kt + STAGES; ++issued) issue_tile(issued);
     }
-    if (kt == 0) {
+    if (kt == 0 && compute) {
       const int j = lane >> 3, rr = lane & 7;
 #pragma unroll
       for (int ks = 0; ks < DH / 16; ++ks)
@@ -281,19 +287,24 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     }
     const uint32_t k_tile = kv_s + (kt % STAGES) * 2 * TILE_BYTES;
     const int key_base = it.key0 + kt * TILE_KEYS;
-    if (!mbar_wait(bar_s + 8u * (kt % STAGES), static_cast<uint32_t>((kt / STAGES) & 1), nullptr, ATT_WAIT_NS)) failed = 1;
+    if (compute &&
+        !mbar_wait(bar_s + 8u * (kt % STAGES), static_cast<uint32_t>((kt / STAGES) & 1), nullptr, ATT_WAIT_NS))
+      failed = 1;
     const int valid_rows = it.key1 - key_base;
     if (valid_rows < TILE_KEYS) {
       // rows past the last key hold stale bytes (rest of the last page, pages not requested): zero the
       // V rows so that a zero probability times garbage cannot produce NaN (K rows are masked anyway)
       uint8_t* kv_gen = smem + (kt % STAGES) * 2 * TILE_BYTES;
-      for (int u = tid; u < (TILE_KEYS - valid_rows) * CH; u += ATT_THREADS) {
+      // (compute warps only: they have seen the tile land; the TMA warp has not waited for it)
+      for (int u = tid; compute && u < (TILE_KEYS - valid_rows) * CH; u += ATT_COMPUTE) {
         const int rr = valid_rows + u / CH, c = u % CH;
         *reinterpret_cast<uint4*>(kv_gen + kv_off<DH>(rr, c, 1)) = make_uint4(0u, 0u, 0u, 0u);
       }
       __syncthreads();
     }
-    if (decode) {
+    if (!compute) {
+      // the TMA warp has nothing to compute
+    } else if (decode) {
       if (key_base + warp * 16 < it.key1)
         warp_attend<DH, 2>(qf, k_tile, warp * 16, key_base, it.key1, pos_a, pos_b, p.scale_log2, m, l, oacc);
     } else {
@@ -302,7 +313,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
     }
   }
   if (__syncthreads_or(failed)) {
-    if (tid == 0) {
+    if (prod) {
       atomicOr(p.status, HB_DEV_ATTN_WAIT_EXPIRED);
       for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block retires
     }
@@ -317,6 +328,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   }
 
   if (!decode) {
+    if (!compute) return;
     // ---- chunk item: normalise, stage the warp's 16 rows in shared memory, store 16-byte vectors ----
     const float inv_a = (l[0] > 0.0f) ? 1.0f / l[0] : 0.0f, inv_b = (l[1] > 0.0f) ? 1.0f / l[1] : 0.0f;
     uint8_t* stage = smem;  // the ring is idle now; this warp touches its own 16 rows of the first tile only
@@ -343,7 +355,7 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   // ---- decode item: merge the four warps' partials in shared memory ----
   __syncthreads();  // every warp is done reading the K/V ring
   float* mbuf = reinterpret_cast<float*>(smem);  // [4 warps][16 rows][REC], over the idle ring
-  {
+  if (compute) {
     float* mine = mbuf + warp * 16 * REC;
 #pragma unroll
     for (int dn = 0; dn < DH / 8; ++dn) {
