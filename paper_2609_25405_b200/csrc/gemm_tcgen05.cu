@@ -41,7 +41,11 @@ struct Tile {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = (2 * BN <= 256) ? 256 : 512;  // two accumulators, rounded to a power of two
   static constexpr int BAR_BYTES = 256;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
+  // staging tiles of the residual epilogue: per epilogue warp 32 rows x 32 floats, rows 36 floats apart
+  static constexpr int STG_PITCH = 36;
+  static constexpr int STG_WARP_BYTES = 32 * STG_PITCH * 4;
+  static constexpr int STG_OFF = STAGES * STAGE_BYTES + BAR_BYTES;
+  static constexpr int SMEM_BYTES = STG_OFF + 4 * STG_WARP_BYTES + 1024;  // + alignment slack
 };
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
@@ -114,6 +118,44 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
       }
     }
   }
+}
+
+// Residual update x += acc for one 32 x 32 block (this warp's 32 rows, 32 columns from col0).  In
+// TMEM a thread owns a row, so storing straight from registers makes every warp-level access touch
+// 32 different rows (one 16-byte piece of 32 cache lines): measured 44-49 k cycles per 256 x 256
+// tile, longer than the 64-k-block main loop it should hide behind.  The block goes through a
+// shared-memory tile instead and comes back with eight lanes per row, so each access covers whole
+// 128-byte lines of four rows.
+__device__ __forceinline__ void resid_block_store(const GemmArgs& g, float* stg, int pitch, int lane, int row0,
+                                                  int col0, const uint32_t (&r)[32]) {
+  float* mine = stg + lane * pitch;
+#pragma unroll
+  for (int v = 0; v < 8; ++v)
+    *reinterpret_cast<float4*>(mine + v * 4) = make_float4(__uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
+                                                           __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+  __syncwarp();
+  const int sub = lane >> 3, cq = (lane & 7) * 4;
+  if (col0 + cq < g.N) {   // N is a multiple of 8: a group of four columns is valid or not as a whole
+    // all eight loads of x are issued before the first store: interleaved, the compiler has to keep
+    // each load behind the previous store (they could alias) and the round trips add up
+    float* base = static_cast<float*>(g.C) + static_cast<size_t>(row0 + sub) * g.ldc + col0 + cq;
+    float4 old[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // (plain load: with split K these rows were written earlier in this launch, by another SM
+      // whose stores went to L2, or by this SM itself; this SM's L1 holds no older copy of them)
+      if (row0 + i * 4 + sub < g.M) old[i] = *reinterpret_cast<const float4*>(base + static_cast<size_t>(i) * 4 * g.ldc);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (row0 + i * 4 + sub < g.M) {
+        const float4 a = *reinterpret_cast<const float4*>(stg + (i * 4 + sub) * pitch + cq);
+        *reinterpret_cast<float4*>(base + static_cast<size_t>(i) * 4 * g.ldc) =
+            make_float4(old[i].x + a.x, old[i].y + a.y, old[i].z + a.z, old[i].w + a.w);
+      }
+    }
+  }
+  __syncwarp();   // the tile may be rewritten by the next block
 }
 
 // Split-K partial of the thin adapter GEMM: fp32, [split][row][N].
@@ -393,7 +435,13 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         uint32_t r[32];
         tmem_ld32(t_row + static_cast<uint32_t>(c), r);
         tmem_ld_wait();
-        if (row_ok && n0 + c < g.N) {
+        if constexpr (EPI == HB_EPI_RESID_F32) {
+          // every lane takes part (the block is exchanged through shared memory); rows and columns
+          // past the edges are masked inside
+          if (n0 + c < g.N)
+            resid_block_store(g, reinterpret_cast<float*>(smem_gen + T::STG_OFF + quarter * T::STG_WARP_BYTES),
+                              T::STG_PITCH, lane, m0 + quarter * 32, n0 + c, r);
+        } else if (row_ok && n0 + c < g.N) {
           if constexpr (EPI == HB_EPI_QKV_ROPE) {
             epilogue_qkv_rope(g, row, n0 + c, r, pos, page);
           } else if constexpr (EPI == HB_EPI_LORA_DOWN) {
