@@ -27,9 +27,10 @@ __device__ __forceinline__ void f16x4_to_float4(uint2 raw, float4& o) {
 }
 
 // x[t,:] = E[tok[t],:] (kept in fp32 as the residual stream); h[t,:] = fp16(rmsnorm(x) * gain).
-// GATHER = false: x is read instead.
-template <bool GATHER>
-__global__ void __launch_bounds__(NORM_THREADS)
+// GATHER = false: x is read instead.  NV = 16-byte vectors a thread holds: 4 covers d_model <= 4096 in
+// few enough registers for eight blocks per SM (more rows in flight per SM), 8 covers d_model <= 8192.
+template <bool GATHER, int NV>
+__global__ void __launch_bounds__(NORM_THREADS, NV == 4 ? 8 : 4)
 norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E,
             const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __half* __restrict__ h,
             int d, float eps) {
@@ -38,12 +39,12 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
   __shared__ float red[32];
   const int t = blockIdx.x;
   const int nv = d >> 2;
-  float4 buf[MAX_VEC];
+  float4 buf[NV];
   float ss = 0.0f;
   float* xrow = x + static_cast<size_t>(t) * d;
   const __nv_bfloat16* erow = GATHER ? E + static_cast<size_t>(tok[t]) * d : nullptr;
 #pragma unroll
-  for (int i = 0; i < MAX_VEC; ++i) {
+  for (int i = 0; i < NV; ++i) {
     const int v = threadIdx.x + i * NORM_THREADS;
     if (v < nv) {
       if (GATHER) {
@@ -59,7 +60,7 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
   const float rstd = rsqrtf(tot / static_cast<float>(d) + eps);
   __half* hrow = h + static_cast<size_t>(t) * d;
 #pragma unroll
-  for (int i = 0; i < MAX_VEC; ++i) {
+  for (int i = 0; i < NV; ++i) {
     const int v = threadIdx.x + i * NORM_THREADS;
     if (v < nv) {
       float4 g;
@@ -208,13 +209,20 @@ int check_launch() { return cudaGetLastError() == cudaSuccess ? HB_OK : HB_ERR_C
 }  // namespace
 
 int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s) {
-  return hb_launch_kernel(norm_kernel<true>, c->dd.T, NORM_THREADS, 0, s, c->pdl, c->dd.tok,
+  if (c->cfg.d_model <= 4 * 4 * NORM_THREADS)
+    return hb_launch_kernel(norm_kernel<true, 4>, c->dd.T, NORM_THREADS, 0, s, c->pdl, c->dd.tok,
+                            static_cast<const __nv_bfloat16*>(tok_emb), static_cast<const __nv_bfloat16*>(gain), c->x,
+                            c->h, c->cfg.d_model, c->cfg.rms_eps);
+  return hb_launch_kernel(norm_kernel<true, MAX_VEC>, c->dd.T, NORM_THREADS, 0, s, c->pdl, c->dd.tok,
                           static_cast<const __nv_bfloat16*>(tok_emb), static_cast<const __nv_bfloat16*>(gain), c->x,
                           c->h, c->cfg.d_model, c->cfg.rms_eps);
 }
 
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s) {
-  return hb_launch_kernel(norm_kernel<false>, c->dd.T, NORM_THREADS, 0, s, c->pdl, nullptr, nullptr,
+  if (c->cfg.d_model <= 4 * 4 * NORM_THREADS)
+    return hb_launch_kernel(norm_kernel<false, 4>, c->dd.T, NORM_THREADS, 0, s, c->pdl, nullptr, nullptr,
+                            static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps);
+  return hb_launch_kernel(norm_kernel<false, MAX_VEC>, c->dd.T, NORM_THREADS, 0, s, c->pdl, nullptr, nullptr,
                           static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps);
 }
 
