@@ -29,7 +29,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;   // TMA warp, MMA warp, eight epilogue warps
+constexpr int EPI_WARPS = 8;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
 template <int BN, int CG>
@@ -41,11 +42,11 @@ struct Tile {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = (2 * BN <= 256) ? 256 : 512;  // two accumulators, rounded to a power of two
   static constexpr int BAR_BYTES = 256;
-  // staging tiles of the residual epilogue: per epilogue warp 32 rows x 32 floats, rows 36 floats apart
-  static constexpr int STG_PITCH = 36;
+  // staging tiles of the residual epilogue: per epilogue warp 32 rows x 16 floats, rows 20 floats apart
+  static constexpr int STG_PITCH = 20;
   static constexpr int STG_WARP_BYTES = 32 * STG_PITCH * 4;
   static constexpr int STG_OFF = STAGES * STAGE_BYTES + BAR_BYTES;
-  static constexpr int SMEM_BYTES = STG_OFF + 4 * STG_WARP_BYTES + 1024;  // + alignment slack
+  static constexpr int SMEM_BYTES = STG_OFF + EPI_WARPS * STG_WARP_BYTES + 1024;  // + alignment slack
 };
 
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
@@ -122,40 +123,45 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
 
 // Residual update x += acc for one 32 x 32 block (this warp's 32 rows, 32 columns from col0).  In
 // TMEM a thread owns a row, so storing straight from registers makes every warp-level access touch
-// 32 different rows (one 16-byte piece of 32 cache lines): measured 44-49 k cycles per 256 x 256
-// tile, longer than the 64-k-block main loop it should hide behind.  The block goes through a
-// shared-memory tile instead and comes back with eight lanes per row, so each access covers whole
-// 128-byte lines of four rows.
+// 32 different rows (one 16-byte piece of 32 cache lines), and with each load of x followed by its
+// store the compiler has to keep every load behind the previous store (they could alias): measured
+// 44-49 k cycles per 256 x 256 tile, longer than the 64-k-block main loop it should hide behind.
+// The block goes through a shared-memory tile instead, 16 columns at a time, and comes back with
+// four lanes per row (64-byte row segments of eight rows per access); all loads of x are issued
+// before the first store.
 __device__ __forceinline__ void resid_block_store(const GemmArgs& g, float* stg, int pitch, int lane, int row0,
                                                   int col0, const uint32_t (&r)[32]) {
   float* mine = stg + lane * pitch;
+  const int sub = lane >> 2, cq = (lane & 3) * 4;
 #pragma unroll
-  for (int v = 0; v < 8; ++v)
-    *reinterpret_cast<float4*>(mine + v * 4) = make_float4(__uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
-                                                           __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
-  __syncwarp();
-  const int sub = lane >> 3, cq = (lane & 7) * 4;
-  if (col0 + cq < g.N) {   // N is a multiple of 8: a group of four columns is valid or not as a whole
-    // all eight loads of x are issued before the first store: interleaved, the compiler has to keep
-    // each load behind the previous store (they could alias) and the round trips add up
-    float* base = static_cast<float*>(g.C) + static_cast<size_t>(row0 + sub) * g.ldc + col0 + cq;
-    float4 old[8];
+  for (int hcol = 0; hcol < 2; ++hcol) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      // (plain load: with split K these rows were written earlier in this launch, by another SM
-      // whose stores went to L2, or by this SM itself; this SM's L1 holds no older copy of them)
-      if (row0 + i * 4 + sub < g.M) old[i] = *reinterpret_cast<const float4*>(base + static_cast<size_t>(i) * 4 * g.ldc);
-    }
+    for (int v = 0; v < 4; ++v)
+      *reinterpret_cast<float4*>(mine + v * 4) =
+          make_float4(__uint_as_float(r[hcol * 16 + v * 4 + 0]), __uint_as_float(r[hcol * 16 + v * 4 + 1]),
+                      __uint_as_float(r[hcol * 16 + v * 4 + 2]), __uint_as_float(r[hcol * 16 + v * 4 + 3]));
+    __syncwarp();
+    const int cb = col0 + hcol * 16 + cq;
+    if (cb < g.N) {   // N is a multiple of 8: a group of four columns is valid or not as a whole
+      float* base = static_cast<float*>(g.C) + static_cast<size_t>(row0 + sub) * g.ldc + cb;
+      float4 old[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (row0 + i * 4 + sub < g.M) {
-        const float4 a = *reinterpret_cast<const float4*>(stg + (i * 4 + sub) * pitch + cq);
-        *reinterpret_cast<float4*>(base + static_cast<size_t>(i) * 4 * g.ldc) =
-            make_float4(old[i].x + a.x, old[i].y + a.y, old[i].z + a.z, old[i].w + a.w);
+      for (int i = 0; i < 4; ++i) {
+        // (plain load: with split K these rows were written earlier in this launch, by another SM
+        // whose stores went to L2, or by this SM itself; this SM's L1 holds no older copy of them)
+        if (row0 + i * 8 + sub < g.M) old[i] = *reinterpret_cast<const float4*>(base + static_cast<size_t>(i) * 8 * g.ldc);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (row0 + i * 8 + sub < g.M) {
+          const float4 a = *reinterpret_cast<const float4*>(stg + (i * 8 + sub) * pitch + cq);
+          *reinterpret_cast<float4*>(base + static_cast<size_t>(i) * 8 * g.ldc) =
+              make_float4(old[i].x + a.x, old[i].y + a.y, old[i].z + a.z, old[i].w + a.w);
+        }
       }
     }
+    __syncwarp();   // the tile may be rewritten
   }
-  __syncwarp();   // the tile may be rewritten by the next block
 }
 
 // Split-K partial of the thin adapter GEMM: fp32, [split][row][N].
@@ -269,7 +275,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4 * CG);  // one arrival per epilogue warp of every CTA of the group
+      mbar_init(tempty_bar(a), EPI_WARPS * CG);  // one arrival per epilogue warp of every CTA of the group
     }
     *abort_flag = 0u;
     mbar_init_fence();
@@ -385,8 +391,13 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     }
     __syncwarp();
   } else {
-    // ---------------- epilogue (warps 2..5) ----------------
+    // ---------------- epilogue (warps 2..9) ----------------
+    // Two warps share each group of 32 TMEM lanes (rows): warps 2-5 take the left half of the tile's
+    // columns, warps 6-9 the right half, so a tile's epilogue - and with it the one after a CTA's
+    // last tile, which nothing hides - takes half as long.
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    const int half = (warp - 2) >> 2;
+    const int epi_slot = half * 4 + quarter;   // 0..7
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -415,7 +426,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         if (k_splits > 1) {
           // one turn word per (tile, CTA of the group, warp): these 32 rows of the tile are updated by
           // split 0, then split 1, ...; the word holds the split whose turn it is
-          turn = g.split_counters + ((static_cast<size_t>(mn) * CG + rank) * 4 + quarter);
+          turn = g.split_counters + ((static_cast<size_t>(mn) * CG + rank) * EPI_WARPS + epi_slot);
           if (split > 0) {
             uint32_t okw = 1u;
             if (lane == 0) {
@@ -431,7 +442,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         }
       }
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = half * (BN / 2); c < (half + 1) * (BN / 2); c += 32) {
         uint32_t r[32];
         tmem_ld32(t_row + static_cast<uint32_t>(c), r);
         tmem_ld_wait();
@@ -439,7 +450,7 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           // every lane takes part (the block is exchanged through shared memory); rows and columns
           // past the edges are masked inside
           if (n0 + c < g.N)
-            resid_block_store(g, reinterpret_cast<float*>(smem_gen + T::STG_OFF + quarter * T::STG_WARP_BYTES),
+            resid_block_store(g, reinterpret_cast<float*>(smem_gen + T::STG_OFF + epi_slot * T::STG_WARP_BYTES),
                               T::STG_PITCH, lane, m0 + quarter * 32, n0 + c, r);
         } else if (row_ok && n0 + c < g.N) {
           if constexpr (EPI == HB_EPI_QKV_ROPE) {
@@ -474,13 +485,13 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           __threadfence();
           __syncwarp();
           uint32_t prev = 0;
-          uint32_t* ctr = g.split_counters + (static_cast<size_t>(mn) * 4 + quarter);
+          uint32_t* ctr = g.split_counters + (static_cast<size_t>(mn) * EPI_WARPS + epi_slot);
           if (lane == 0) prev = atomicAdd(ctr, 1u);
           prev = __shfl_sync(0xffffffffu, prev, 0);
           if (prev + 1u == static_cast<uint32_t>(k_splits)) {
             __threadfence();
             if (row_ok) {
-              for (int c = 0; c < BN && n0 + c < g.N; c += 32) {
+              for (int c = half * (BN / 2); c < (half + 1) * (BN / 2) && n0 + c < g.N; c += 32) {
                 uint32_t r[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = 0u;   // +0.0f

@@ -120,7 +120,7 @@ struct GemmArgs {
   // HB_EPI_LORA_DOWN and HB_EPI_RESID_F32
   int32_t k_splits;          // work items per output tile (0 or 1 = no split), each over an equal share of the K blocks
   float* split_part;         // LORA_DOWN: [k_splits, M, N] partial sums (k_splits > 1)
-  uint32_t* split_counters;  // LORA_DOWN: [tiles * 4] arrival counters; RESID_F32: [tiles * CG * 4] turn words; zero between launches
+  uint32_t* split_counters;  // LORA_DOWN: [tiles * 8] arrival counters; RESID_F32: [tiles * CG * 8] turn words (one per epilogue warp); zero between launches
   // HB_EPI_QKV_ROPE only
   const int32_t* row_pos;   // [M] position of each row inside its request
   const int32_t* row_page;  // [M] physical page that holds that position

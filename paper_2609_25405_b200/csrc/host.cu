@@ -65,8 +65,8 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.act = cv.take(rows * c.d_ffn * 2);
   L.lora_u = cv.take(rows * HB_LORA_U_COLS * 2);
   L.lora_part = cv.take(static_cast<size_t>(HB_LORA_K_SPLITS) * rows * HB_LORA_U_COLS * 4);
-  L.lora_counters = cv.take((rows / 128) * 2 * 4 * 4);
-  L.n_resid_turns = static_cast<int32_t>((rows / 128) * ((static_cast<size_t>(c.d_model) + 255) / 256) * 4);
+  L.lora_counters = cv.take((rows / 128) * 2 * 8 * 4);
+  L.n_resid_turns = static_cast<int32_t>((rows / 128) * ((static_cast<size_t>(c.d_model) + 255) / 256) * 8);
   L.resid_turns = cv.take(static_cast<size_t>(L.n_resid_turns) * 4);
   L.logit_in = cv.take(lrows * 2 * c.d_model * 2);
   L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
@@ -253,7 +253,7 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   c->lora_u = reinterpret_cast<__half*>(c->ws + lay.lora_u);
   c->lora_part = reinterpret_cast<float*>(c->ws + lay.lora_part);
   c->lora_counters = reinterpret_cast<uint32_t*>(c->ws + lay.lora_counters);
-  c->n_lora_counters = static_cast<int32_t>((lay.rows_pad / 128) * 2 * 4);
+  c->n_lora_counters = static_cast<int32_t>((lay.rows_pad / 128) * 2 * 8);
   c->resid_turns = reinterpret_cast<uint32_t*>(c->ws + lay.resid_turns);
   c->n_resid_turns = lay.n_resid_turns;
   c->logit_in = reinterpret_cast<__half*>(c->ws + lay.logit_in);
@@ -970,7 +970,7 @@ int hb_gemm_pair(hb_ctx* c, const void* A, const void* B, const void* A2, const 
   ga.ldc = (epilogue == HB_EPI_SWIGLU) ? N / 2 : N;
   if (epilogue == HB_EPI_RESID_F32) {
     const int ks = hb_gemm_pick_ksplit(M, N, K, bn, c->num_sms);
-    const long turns = static_cast<long>((M + 255) / 256) * ((N + 255) / 256) * 2 * 4;
+    const long turns = static_cast<long>((M + 255) / 256) * ((N + 255) / 256) * 2 * 8;
     if (ks > 1 && turns <= c->n_resid_turns) {
       ga.k_splits = ks;
       ga.split_counters = c->resid_turns;
