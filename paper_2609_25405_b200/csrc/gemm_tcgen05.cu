@@ -6,14 +6,15 @@
 // the forward "applies attention and feed-forward layers" to every row of the mixed
 // batch): QKV, O, gate/up, down and the LM head.
 //
-// Structure (one persistent CTA per SM, 192 threads):
+// Structure (one persistent CTA per SM, 320 threads):
 //   warp 0   TMA producer: cp.async.bulk.tensor 2-D tiles (128B swizzle) into a ring of
 //            shared-memory stages, completion on mbarriers
 //   warp 1   MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=16) from shared
 //            memory descriptors into one of two TMEM accumulators; tcgen05.commit
 //            releases stages and publishes finished accumulators
-//   warps 2-5 epilogue: tcgen05.ld the accumulator (each warp owns 32 TMEM lanes), apply
-//            the epilogue, store with 16-byte vectors; overlaps the next tile's main loop
+//   warps 2-9 epilogue: tcgen05.ld the accumulator (two warps per group of 32 TMEM lanes, half of
+//            the tile's columns each), apply the epilogue, store with 16-byte vectors; overlaps
+//            the next tile's main loop
 // Two variants share the code.  CG = 1: one CTA per 128 x BN tile.  CG = 2: a cluster of two CTAs
 // works on one 256 x 256 tile with tcgen05 cta_group::2: each CTA loads its own 128 rows of A and
 // its own 128 rows of B (no multicast), the leader CTA issues MMAs that read both CTAs' shared
