@@ -239,8 +239,8 @@ HB_API int hb_mixed_step(hb_ctx* ctx, const hb_batch_desc* desc, const hb_weight
 /* ---- low-rank adapters on embedding rows ------------------------------------
  *
  * With a shared backbone the embedding model is the generation model plus a
- * low-rank adapter (Section 2.1 "Parameter sharing"; Section 5.1 runs both
- * request types on one GPU "using LoRA adapters").  Inside the one forward
+ * low-rank adapter (Section 2.1, paragraph on parameter sharing; in Section
+ * 5.1 both request types share one GPU through such adapters).  Inside the one forward
  * pass, rows of EMBED_CHUNK segments compute every projection as
  *     y = x W^T + (alpha / r) (x A^T) B^T,        A [r, in], B [out, r],
  * and rows of DECODE / PREFILL_CHUNK segments compute y = x W^T.  The paper
@@ -331,7 +331,7 @@ HB_API int hb_last_launch_count(const hb_ctx* ctx, int32_t* out_count);
 /* ---- kernel-level entry points (used by the parity tests) ----------------- */
 
 /* Epilogues of the projection GEMM (the dense contractions of the forward,
- * Section 3.1 "attention and feed-forward layers"). */
+ * Section 3.1: the attention and feed-forward projections every row passes through). */
 enum {
   HB_EPI_F16 = 0,       /* C fp16 [M,N] = A * B^T                               */
   HB_EPI_F32 = 1,       /* C float [M,N] = A * B^T                              */

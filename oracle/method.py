@@ -5,7 +5,7 @@ own steps in the paper's order and notation, so the method's invariants can be
 brute-forced on small shapes:
 
 * a request is executed as K chunks of sizes c_1..c_K over successive
-  iterations (Section 3.2 "chunked embedding", Section 3.3 first paragraph);
+  iterations (chunked embedding, Section 3.2; Section 3.3, first paragraph);
   chunk k attends causally over the K/V its request produced in chunks 1..k-1
   plus its own rows;
 * the incremental pooler keeps S and W per request and applies
@@ -20,7 +20,7 @@ brute-forced on small shapes:
   (Section 2.1 "Parameter sharing", Section 5.1): taken here as the
   unmerged two-branch product per request;
 * a decode token is a chunk of one row whose logits are wanted
-  (Section 3.2: "decode tokens process exactly one token per request").
+  (Section 3.2: a decode step contributes a single token of its request).
 
 GPU results are never compared with this module's floating-point outputs;
 they are compared with `transformer`.  The integer helpers at the bottom

@@ -83,7 +83,7 @@ def forward(cfg, W, tokens, logit_rows=None, dtype=np.float64, pos_offset=0,
     """Whole-sequence forward of one request.
 
     Returns (Hhat [n,d], logits [len(logit_rows), V]).  Hhat is the output of
-    the final RMSNorm ("final hidden states", Section 2.1); logits are computed
+    the final RMSNorm (the hidden states of the last layer that Section 2.1 pools); logits are computed
     for `logit_rows` only (all rows if None, none if empty).  `pos_offset`
     shifts every position by a constant (used by a rotary-invariance pin).
     With return_kv=True also returns per-layer (k_rotated, v) lists.

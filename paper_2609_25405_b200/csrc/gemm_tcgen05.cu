@@ -3,8 +3,8 @@
 // operands), both K-major, fp32 accumulation in tensor memory.
 //
 // These are the dense contractions of the shared forward pass (Section 3.1 of the paper:
-// the forward "applies attention and feed-forward layers" to every row of the mixed
-// batch): QKV, O, gate/up, down and the LM head.
+// every row of the mixed batch goes through the same attention and feed-forward projections):
+// QKV, O, gate/up, down and the LM head.
 //
 // Structure (one persistent CTA per SM, 320 threads):
 //   warp 0   TMA producer: cp.async.bulk.tensor 2-D tiles (128B swizzle) into a ring of
