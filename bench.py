@@ -437,6 +437,8 @@ def main():
                  "bound": "tensor" if t_gemm_burst > t_mem else "hbm",
                  "frac_of_burst_roof": max(t_gemm_burst, t_mem) * 1e3 / step_ms,
                  "frac_of_sustained_roof": max(t_gemm_sust, t_mem) * 1e3 / step_ms,
+                 # nominal dense bf16 rate and HBM3e bandwidth of the part, for context only
+                 "frac_of_datasheet_roof": max(w["gemm_flops"] / 2250e12, bytes_step / 8.0e12) * 1e3 / step_ms,
                  "peak_kind": peak_kind}
     breakdown = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in prof.items()}
     line = {"metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
