@@ -1,7 +1,7 @@
 """Full-size parity: the 1B-class and 7B-class shapes at their full depth and width, in the launch
-configuration the benchmark times (full token budget per step, decode rows over long synthetic
-contexts plus embedding chunks), checked on sampled requests the CPU oracle can recompute one
-by one.  Legitimate because a request's outputs do not depend on its batch mates (checked
+configurations the benchmark times (full token budget per step, decode rows over long synthetic
+contexts plus embedding chunks; for the 7B shape also one point of the embedding-fraction sweep with
+2048 decode rows), checked on sampled requests the CPU oracle can recompute one by one.  Legitimate because a request's outputs do not depend on its batch mates (checked
 bit for bit on the tiny shape, and here on one request run solo and inside the batch).
 
 Sampled per shape: two generation requests (prompt prefilled in chunks through the library
@@ -31,6 +31,13 @@ CASES = {
                     gen=(128, 600), emb=(200, 700), emb_mean=(450,), seed=1002, n_steps=4),
     "cfg3-7b": dict(shape="7b", n_decode=64, ctx=(512, 4096), budget=4096, chunk=512,
                     gen=(512, 1100), emb=(300, 700), emb_mean=(640,), seed=1003, n_steps=2),
+    # one point of the embedding-fraction sweep (f = 0.5): 2048 decode rows at context 2048 next to
+    # 2048 rows of mean-pooled embedding chunks.  Unaliased, the decode contexts alone would need
+    # 550 GB of KV, so (as in the benchmark) filler row i reads the context pages of row i mod `alias`
+    # and appends to a private tail page; 64 distinct contexts here (256 in the benchmark).
+    "cfg4-7b-f0.5": dict(shape="7b", n_decode=2048, ctx=(2048, 2048), budget=4096, chunk=512,
+                         gen=(2048,), emb=(), emb_mean=(1500,), seed=1004, n_steps=2, alias=64,
+                         fill_len=(128, 2048), fill_mean=True),
 }
 
 
@@ -38,7 +45,7 @@ def _threads():
     return max(4, min(32, os.cpu_count() or 8))
 
 
-@pytest.mark.parametrize("name", ["cfg2-1b", "cfg3-7b"])
+@pytest.mark.parametrize("name", ["cfg2-1b", "cfg3-7b", "cfg4-7b-f0.5"])
 def test_fullsize_sampled_requests_match_oracle(name):
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
@@ -51,9 +58,11 @@ def test_fullsize_sampled_requests_match_oracle(name):
     n_steps = c["n_steps"]       # logits rows compared per generation request (prefill row + decode rows)
     max_pos = c["ctx"][1] + n_steps + 8
     n_dec = c["n_decode"]
-    ctxs = rng.integers(c["ctx"][0], c["ctx"][1] + 1, size=n_dec - 2)
-    n_pages = int(sum((x + n_steps + P) // P + 1 for x in ctxs)) + 5 * (max_pos // P + 2) + \
-        n_steps * (c["budget"] // P + 80)
+    alias = c.get("alias", 0)
+    ctxs = rng.integers(c["ctx"][0], c["ctx"][1] + 1, size=n_dec - len(c["gen"]))
+    own = ctxs if not alias else ctxs[:alias]
+    n_pages = int(sum((x + n_steps + P) // P + 1 for x in own)) + 5 * (max_pos // P + 2) + \
+        (n_steps + 4) * (c["budget"] // P + 80) + (2 * (len(ctxs) - alias) if alias else 0)
     eng = Engine(shape, dw, n_pages=n_pages, n_slots=256, max_tokens=c["budget"], max_segs=n_dec + 160,
                  max_pos=max_pos)
     # synthetic cached context for the filler rows: N(0,1) K/V everywhere, then sentinel on the pages
@@ -78,11 +87,15 @@ def test_fullsize_sampled_requests_match_oracle(name):
         view[:, torch.tensor(r.pages)] = KV_SENTINEL
     # ---- filler ----
     fill_dec = []
-    for x in ctxs:
+    for i, x in enumerate(ctxs):
         r = Request("gen", synth.token_ids(rng, int(x) + 1, shape.V))
         r.n_prompt = int(x)
         r.n_done = int(x)
-        r.pages = eng.kv.alloc((int(x) + P - 1) // P)
+        if alias and i >= alias:
+            assert int(x) % P == 0                      # whole context pages are shared, read-only
+            r.pages = list(fill_dec[i % alias].pages[:int(x) // P])
+        else:
+            r.pages = eng.kv.alloc((int(x) + P - 1) // P)
         fill_dec.append(r)
 
     # ---- oracle (one whole-sequence forward per sampled request; fp32 as the benchmark spec says) ----
@@ -102,7 +115,7 @@ def test_fullsize_sampled_requests_match_oracle(name):
     got_emb = {}
     chunk = c["chunk"]
     inflight_fill = []
-    for step in range(n_steps + 3):
+    for step in range(n_steps + 3 + max(c["gen"]) // chunk):
         work = []
         rows = 0
         for r in fill_dec:
@@ -131,8 +144,9 @@ def test_fullsize_sampled_requests_match_oracle(name):
             if f.remaining() - max(q, 0) > 0:
                 nxt.append(f)
         while rows < c["budget"]:
-            n = int(rng.integers(16, 2 * chunk))
-            f = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_LAST)
+            lo, hi = c.get("fill_len", (16, 2 * chunk - 1))
+            n = int(rng.integers(lo, hi + 1))
+            f = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_MEAN if c.get("fill_mean") else B.POOL_LAST)
             q = min(chunk, n, c["budget"] - rows)
             work.append((f, q)); rows += q
             if q < n:
@@ -153,6 +167,16 @@ def test_fullsize_sampled_requests_match_oracle(name):
                 eng.release(f)
         if all(len(got_lg[g]) >= n_steps for g in gens) and len(got_emb) == len(embs):
             break
+    assert eng.ctx.status_poll() == 0
+
+    # ---- one sampled embedding request again, alone in its steps (same chunking): bit for bit the
+    # result it had inside the full batches
+    solo = Request("embed", list(embs[0].tokens), embs[0].pool_mode)
+    while solo.remaining() > 0:
+        _, _, er = eng.step([(solo, min(chunk, solo.remaining()))])
+    torch.cuda.synchronize()
+    assert np.array_equal(eng.out_emb[er[solo]].cpu().numpy().astype(np.float64), got_emb[embs[0]])
+    eng.release(solo)
     assert eng.ctx.status_poll() == 0
 
     # ---- compare ----
