@@ -29,9 +29,9 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) per launch of the projection GEMM at the 7B shape, T = 4096, mean of the four
 # projections of a layer, from the ncu capture summarised in profiles/gemm_tcgen05_cfg3-7b_layers2.md
-# (QKV 126.5 MB, O 188.3 MB, gate/up 411.6 MB, down 829.2 MB; algorithmic 134 / 201 / 386 / 497 MB, the last
+# (QKV 126.3 MB, O 188.5 MB, gate/up 406.2 MB, down 836.8 MB; algorithmic 134 / 201 / 386 / 497 MB, the last
 # with the second pass over x that the split-K down projection makes)
-NCU_GEMM_TRAFFIC_BYTES = {"7b": 388.9e6}
+NCU_GEMM_TRAFFIC_BYTES = {"7b": 389.4e6}
 
 
 def load_peaks():
