@@ -654,6 +654,28 @@ int hb_gemm_pick_ksplit(int M, int N, int K, int variant, int num_sms) {
   return e2 > e1 * 1.05 ? 2 : 1;
 }
 
+// CTA-pair 256 x 256 tiles and single-CTA 128 x 128 tiles read B through the same 128-row boxes and
+// accumulate every output element over K in the same order, so their results are bit-identical
+// (checked in the tests) and a launch may use whichever is faster for its own row count without a
+// request's result depending on its batch.  K splits are not part of this choice: they change the
+// summation order and stay fixed per context.  The estimate is waves x time per wave with figures
+// measured on the 1B- and 7B-class projections (microseconds; k = 64-column K blocks per work item):
+// pair tile 4 + 0.33 k, single tile 1.5 + 0.275 k.  The pair tile does four times the flops of the
+// single one, so it wins whenever both variants have more than a wave of work; the single tile wins
+// when a small step leaves most CTA pairs without a tile.
+int hb_gemm_pick_step_variant(int map_variant, int rows, int N, int k_blocks, int k_splits, int num_sms) {
+  if (map_variant != HB_GEMM_PAIR256 && map_variant != 128) return map_variant;
+  if (rows <= 128) return 128;   // one row tile: the pair's second CTA would hold no rows
+  const int ks = k_splits > 1 ? k_splits : 1;
+  const double k = static_cast<double>((k_blocks + ks - 1) / ks);
+  const long pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
+  const long u_pair = static_cast<long>((rows + 255) / 256) * ((N + 255) / 256) * ks;
+  const long u_single = static_cast<long>((rows + 127) / 128) * ((N + 127) / 128) * ks;
+  const double t_pair = static_cast<double>((u_pair + pairs - 1) / pairs) * (4.0 + 0.33 * k);
+  const double t_single = static_cast<double>((u_single + num_sms - 1) / num_sms) * (1.5 + 0.275 * k);
+  return t_single * 1.05 < t_pair ? 128 : HB_GEMM_PAIR256;
+}
+
 int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : variant; }
 
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,

@@ -140,6 +140,9 @@ constexpr int HB_GEMM_PAIR256 = 512;
 int hb_gemm_pick_bn(int M, int N, int num_sms);
 int hb_gemm_box_rows(int variant);
 int hb_gemm_pick_ksplit(int M, int N, int K, int variant, int num_sms);
+// Variant for one launch of `rows` rows when the B map was built for `map_variant` (the choice made
+// for the context's row capacity): a step much smaller than the capacity may run single-CTA tiles.
+int hb_gemm_pick_step_variant(int map_variant, int rows, int N, int k_blocks, int k_splits, int num_sms);
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,
                    const CUtensorMap* tmB2 = nullptr, bool pdl = false);

@@ -66,7 +66,8 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.lora_u = cv.take(rows * HB_LORA_U_COLS * 2);
   L.lora_part = cv.take(static_cast<size_t>(HB_LORA_K_SPLITS) * rows * HB_LORA_U_COLS * 4);
   L.lora_counters = cv.take((rows / 128) * 2 * 8 * 4);
-  L.n_resid_turns = static_cast<int32_t>((rows / 128) * ((static_cast<size_t>(c.d_model) + 255) / 256) * 8);
+  // one word per (128-row block, column tile, epilogue warp); the narrowest column tile is 128 wide
+  L.n_resid_turns = static_cast<int32_t>((rows / 128) * ((static_cast<size_t>(c.d_model) + 127) / 128) * 8);
   L.resid_turns = cv.take(static_cast<size_t>(L.n_resid_turns) * 4);
   L.logit_in = cv.take(lrows * 2 * c.d_model * 2);
   L.rope_cos = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
@@ -782,6 +783,12 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.status = c->status;
     ga.b_kshift = 0;
     ga.M = T;
+    // tile variant of this step's launches (the maps serve both; see hb_gemm_pick_step_variant)
+    const int kb_d = (cfg.d_model + 63) / 64, kb_q = (n_q + 63) / 64, kb_f = (cfg.d_ffn + 63) / 64;
+    const int v_qkv = hb_gemm_pick_step_variant(wm.bn_qkv, T, n_qkv, kb_d + (use_lora ? r3 / 64 : 0), 1, c->num_sms);
+    const int v_o = hb_gemm_pick_step_variant(wm.bn_o, T, cfg.d_model, kb_q + (use_lora ? r1 / 64 : 0), wm.ks_o, c->num_sms);
+    const int v_gu = hb_gemm_pick_step_variant(wm.bn_gu, T, 2 * cfg.d_ffn, kb_d + (use_lora ? r2 / 64 : 0), 1, c->num_sms);
+    const int v_down = hb_gemm_pick_step_variant(wm.bn_down, T, cfg.d_model, kb_f + (use_lora ? r1 / 64 : 0), wm.ks_down, c->num_sms);
     // QKV projection; its epilogue rotates q, k and appends k, v to the pages
     ga.C = nullptr; ga.N = n_qkv; ga.K = cfg.d_model; ga.ldc = n_qkv;
     ga.row_pos = dd.row_pos; ga.row_page = dd.row_page; ga.rope_cos = c->rope_cos; ga.rope_sin = c->rope_sin;
@@ -790,7 +797,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.P = cfg.page_size; ga.n_pages = kg.n_pages;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_qkv, r3, cfg.d_model));
     ga.k2_blocks = use_lora ? r3 / 64 : 0;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, wm.bn_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s,
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, v_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s,
                                          use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_qkv : nullptr, c->pdl));
     if (fork_attention) {
       // The two attention kernels read the same q and pages and write disjoint rows of attn_out:
@@ -814,7 +821,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.k_splits = wm.ks_o; ga.split_counters = c->resid_turns;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_attn_out, lm->a_o, r1, n_q));
     ga.k2_blocks = use_lora ? r1 / 64 : 0;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, wm.bn_o, HB_EPI_RESID_F32, ga, c->num_sms, s,
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_attn_out, wm.o, v_o, HB_EPI_RESID_F32, ga, c->num_sms, s,
                                          use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_o : nullptr, c->pdl));
     HB_TRY(HB_CLASS_NORM_ROPE, hb_launch_rmsnorm(c, lw.ffn_norm, s));
     // gate/up projection with SwiGLU
@@ -822,14 +829,14 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.k_splits = 1;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_h, lm->a_gu, r2, cfg.d_model));
     ga.k2_blocks = use_lora ? r2 / 64 : 0;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, wm.bn_gu, HB_EPI_SWIGLU, ga, c->num_sms, s,
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.gu, v_gu, HB_EPI_SWIGLU, ga, c->num_sms, s,
                                          use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_gu : nullptr, c->pdl));
     // down projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = cfg.d_ffn; ga.ldc = cfg.d_model;
     ga.k_splits = wm.ks_down; ga.split_counters = c->resid_turns;
     if (use_lora) HB_TRY(HB_CLASS_LORA, lora_down(c->tm_act, lm->a_d, r1, cfg.d_ffn));
     ga.k2_blocks = use_lora ? r1 / 64 : 0;
-    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, wm.bn_down, HB_EPI_RESID_F32, ga, c->num_sms, s,
+    HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_act, wm.down, v_down, HB_EPI_RESID_F32, ga, c->num_sms, s,
                                          use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_d : nullptr, c->pdl));
   }
   float* pool_sum = pool ? static_cast<float*>(pool->arena) : nullptr;

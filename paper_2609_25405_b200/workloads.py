@@ -39,6 +39,8 @@ SPECS = {
     # sigma 1) clipped to [32,4096], chunk 512, last-token pooling, 4096-token budget
     "cfg3-7b": MixSpec("cfg3-7b", "7b", 64, 512, 4096, 4096, 512, "lognormal", 512, 32, 4096, B.POOL_LAST, 1003),
     # small decode-heavy case for profiler captures (use with --layers and --decode-alias)
+    # a small decode-heavy step of the 1B shape, the size the trace replay's steps have on average
+    "dec-1b": MixSpec("dec-1b", "1b", 400, 128, 1024, 448, 256, "uniform", 128, 16, 256, B.POOL_LAST, 1011),
     "dec-7b": MixSpec("dec-7b", "7b", 256, 2048, 2048, 512, 256, "uniform", 128, 128, 1024, B.POOL_MEAN, 1010),
 }
 

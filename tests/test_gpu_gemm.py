@@ -153,6 +153,31 @@ def test_residual_gemm_with_split_k_is_exact_to_tolerance_and_deterministic(M):
     c.close()
 
 
+@pytest.mark.parametrize("epi", ["f32", "swiglu"])
+def test_tile_variants_give_identical_bits(epi):
+    """The same rows computed inside a 4096-row launch (CTA-pair 256 x 256 tiles) and as a launch of
+    their own (single-CTA tiles) are equal bit for bit: every output element is accumulated over K in
+    the same order whatever the tile shape.  The step relies on this when it picks the tile variant
+    from its own row count."""
+    from paper_2609_25405_b200 import binding as B
+    c = B.Context(B.model_cfg(synth.SHAPES["tiny"], 64), 4096, 8, 64)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    code = B.EPI_F32 if epi == "f32" else B.EPI_SWIGLU
+    for N, K in [(4096, 2048), (3072, 4096), (2048, 8192)]:
+        A = torch.randn((4096, K), generator=g, device="cuda").to(torch.float16)
+        Bw = (torch.randn((N, K), generator=g, device="cuda") * 0.05).to(torch.float16)
+        width, dt = (N, torch.float32) if epi == "f32" else (N // 2, torch.float16)
+        big = torch.zeros((4096, width), dtype=dt, device="cuda")
+        c.gemm(A, Bw, big, 4096, N, K, code)
+        for M in (100, 128, 448, 1000):
+            small = torch.zeros((M, width), dtype=dt, device="cuda")
+            c.gemm(A[:M].contiguous(), Bw, small, M, N, K, code)
+            torch.cuda.synchronize()
+            assert torch.equal(small, big[:M]), (N, K, M)
+    assert c.status_poll() == 0
+    c.close()
+
+
 def test_weights_pack_f16_matches_round_to_nearest(ctx):
     """bf16 -> fp16 repack: exact in the fp16 normal range, round-to-nearest on the subnormal grid,
     saturating above 65504; in place."""
