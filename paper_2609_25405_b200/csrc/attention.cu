@@ -150,7 +150,7 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
 }
 
 template <int DH>
-__global__ void __launch_bounds__(ATT_THREADS)
+__global__ void __launch_bounds__(ATT_THREADS, 2)
 attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   grid_dep_wait();
   grid_dep_launch();
@@ -205,22 +205,38 @@ attn_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   const bool prod = (tid == ATT_COMPUTE);
   const bool compute = (warp < ATT_COMPUTE / 32);
   int issued = 0, bad = 0;
-  if (prod) {
-    for (int st = 0; st < STAGES; ++st) mbar_init(bar_s + 8u * st, 1);
-    mbar_init_fence();
-    // the first tiles are requested right away, with page ids read straight from global memory, so
-    // that their latency overlaps the rest of the set-up
-    for (; issued < STAGES - 1 && issued < n_tiles && !bad; ++issued) {
-      int ids[TILE_KEYS / 16];
-      const int pi0 = issued * (TILE_KEYS / 16);
-#pragma unroll
-      for (int pi = 0; pi < TILE_KEYS / 16; ++pi) {
-        const int blk = first_blk + pi0 + pi;
-        ids[pi] = (pi0 + pi < n_blk) ? ((blk < it.pt_len) ? __ldg(p.pages + it.pt_start + blk) : -1) : 0;
-        bad |= (ids[pi] < 0 || ids[pi] >= p.kv.n_pages);
+  if (warp == ATT_COMPUTE / 32) {
+    if (lane == 0) {
+      for (int st = 0; st < STAGES; ++st) mbar_init(bar_s + 8u * st, 1);
+      mbar_init_fence();
+    }
+    __syncwarp();
+    // The first tiles are requested right away, with page ids read straight from global memory, so
+    // that their latency overlaps the rest of the set-up; one lane per page (a single thread needs
+    // ~650 cycles per tile, which for a short item is most of its start-up).
+    static_assert((STAGES - 1) * (TILE_KEYS / 16) <= 32, "one lane per page of the first tiles");
+    const int n_init = min(STAGES - 1, n_tiles);
+    const int t0 = lane / (TILE_KEYS / 16), pi = lane % (TILE_KEYS / 16);
+    const bool act = (t0 < n_init) && (lane < n_blk);
+    int id = 0;
+    if (act) {
+      const int blk = first_blk + lane;
+      id = (blk < it.pt_len) ? __ldg(p.pages + it.pt_start + blk) : -1;
+      bad = (id < 0 || id >= p.kv.n_pages);
+    }
+    bad = __any_sync(0xffffffffu, bad);
+    if (!bad) {
+      const uint32_t bar = bar_s + 8u * t0;
+      if (t0 < n_init && pi == 0) {
+        const int n_pg = min(TILE_KEYS / 16, (it.key1 - (it.key0 + t0 * TILE_KEYS) + 15) / 16);
+        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n_pg) * PAGE_BYTES);
       }
-      if (bad) break;
-      issue_pages(issued, ids);
+      __syncwarp();
+      if (act) {
+        const int row = static_cast<int>(((static_cast<int64_t>(p.layer) * p.kv.n_pages + id) * p.kv.Hkv + hk) * (DH / 2));
+        tma_load_2d(kv_s + t0 * 2 * TILE_BYTES + pi * PAGE_BYTES, &kv_map, bar, 0, row);
+      }
+      issued = n_init;
     }
   }
   // page ids of the keys this item reads -> shared memory (checked once)
