@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhb.so")
-SOURCES = ["host.cu", "gemm_tcgen05.cu", "elementwise.cu", "attention.cu", "attention_tc.cu", "pool_static.cu"]
+SOURCES = ["host.cu", "gemm_tcgen05.cu", "elementwise.cu", "attention.cu", "pool_static.cu"]
 
 
 def _stale():

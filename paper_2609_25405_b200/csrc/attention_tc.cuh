@@ -16,10 +16,14 @@
 //             (probabilities stay below 256, exact in fp16/fp32); the final 1/sum absorbs it.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status bit and leaves without
 // storing.  The work split depends on the segment's own lengths only.
+//
+// This file is the body of one CTA; attention.cu includes it and calls it from the one attention
+// kernel of the step for the blocks that hold a chunk item.
+#pragma once
 #include "hb_internal.h"
 #include "ptx.cuh"
 
-namespace {
+namespace hb_tc {
 
 constexpr int TC_THREADS = 192;
 constexpr int BM = 128;        // query rows per CTA
@@ -52,11 +56,14 @@ struct TcCfg {
   static constexpr int O_COL = 128;                      // O: DH columns (fp32)
 };
 
+// Dynamic shared memory one chunk item needs.
 template <int DH>
-__global__ void __launch_bounds__(TC_THREADS, 2)
-attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams p) {
-  grid_dep_wait();
-  grid_dep_launch();
+constexpr int smem_bytes() { return TcCfg<DH>::BAR_OFF + 8 * (2 * TcCfg<DH>::STAGES + 6) + 16; }
+
+// One CTA of TC_THREADS threads, item `item` of p.items.  `kv_map` points at the kernel's
+// __grid_constant__ tensor map.
+template <int DH>
+__device__ __forceinline__ void chunk_item(const CUtensorMap* kv_map, const TcParams& p, int item) {
   using C = TcCfg<DH>;
   extern __shared__ uint8_t smem_raw[];
   // The kernel has no static shared memory, so the dynamic window starts at the CTA's (1 KiB
@@ -78,7 +85,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
-  const AttnItem it = p.items[blockIdx.x];
+  const AttnItem it = p.items[item];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, Hq = p.Hq, hk = it.kv_head;
   const int n_tiles = (it.key1 + BN - 1) / BN;           // key0 is 0 for chunk items
@@ -143,7 +150,7 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
           if (pi < n_pg) {
             const int64_t page = cur[pi];
             const int row = static_cast<int>(((static_cast<int64_t>(p.layer) * p.n_pages + page) * p.Hkv + hk) * (DH / 2));
-            tma_load_2d(k_dst + pi * C::PAGE_BYTES, &kv_map, kv_full(st), 0, row);   // K and V of this head, one copy
+            tma_load_2d(k_dst + pi * C::PAGE_BYTES, kv_map, kv_full(st), 0, row);   // K and V of this head, one copy
           }
         }
       }
@@ -367,25 +374,8 @@ attn_chunk_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const TcParams 
   }
 }
 
-template <int DH>
-int launch(const CUtensorMap& kv_map, const TcParams& p, int n_items, int max_pos, cudaStream_t s, bool pdl) {
-  using C = TcCfg<DH>;
-  (void)max_pos;
-  const int smem = C::BAR_OFF + 8 * (2 * C::STAGES + 6) + 16;   // two CTAs per SM at Dh = 128
-  static int configured = 0;
-  if (smem > 227 * 1024) return HB_ERR_UNSUPPORTED;
-  if (configured < smem) {
-    if (cudaFuncSetAttribute(attn_chunk_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return HB_ERR_CUDA;
-    configured = smem;
-  }
-  return hb_launch_kernel(attn_chunk_tc_kernel<DH>, n_items, TC_THREADS, smem, s, pdl, kv_map, p);
-}
-
-}  // namespace
-
-int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s) {
-  if (c->dd.n_tc_items <= 0) return HB_OK;
+// Parameters of the chunk items of one layer.
+inline TcParams make_params(hb_ctx* c, const KvGeom& kv, int layer) {
   TcParams p;
   p.q = c->q;
   p.out = c->attn_out;
@@ -398,7 +388,7 @@ int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_ma
   p.pages = c->dd.pages;
   p.status = c->status;
   p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(c->cfg.head_dim));
-  if (c->cfg.head_dim == 64) return launch<64>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s, c->pdl);
-  if (c->cfg.head_dim == 128) return launch<128>(kv_map, p, c->dd.n_tc_items, c->cfg.max_pos, s, c->pdl);
-  return HB_ERR_UNSUPPORTED;
+  return p;
 }
+
+}  // namespace hb_tc

@@ -169,8 +169,12 @@ inline int hb_launch_kernel(void (*kern)(KArgs...), unsigned grid, unsigned bloc
 struct hb_ctx;
 int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaStream_t s);
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
-int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
-int hb_launch_attention_tc(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s);
+// The step's attention launch of one layer.  `which` selects the item lists it serves (both in the
+// step itself; one at a time when launches are timed per class).
+constexpr int HB_ATTN_CHUNK_TILES = 1;   // chunk items of 65-128 rows (tcgen05 body)
+constexpr int HB_ATTN_SMALL_ITEMS = 2;   // decode items and chunk items of at most 64 rows (mma.sync body)
+constexpr int HB_ATTN_ALL = 3;
+int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s, int which);
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,
                     int n_slots, float* rowbuf, int rowbuf_rows, float* out_emb, cudaStream_t s);
 int hb_launch_argmax(const float* logits, int n_rows, int V, int32_t* out, cudaStream_t s);

@@ -187,9 +187,6 @@ struct CtxExtra {
   Layout lay;
   bool profiling = false;
   std::vector<ProfRec> free_recs, used_recs;
-  // side stream on which the chunk-attention kernel runs next to the decode-attention kernel
-  cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 CtxExtra* extra_of(hb_ctx* c) { return static_cast<CtxExtra*>(c->extra); }
@@ -302,9 +299,6 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
     cuda_ok &= cudaMallocHost(reinterpret_cast<void**>(&ex->ring[i].host), lay.desc_cap) == cudaSuccess;
     cuda_ok &= cudaEventCreateWithFlags(&ex->ring[i].ev, cudaEventDisableTiming) == cudaSuccess;
   }
-  cuda_ok &= cudaStreamCreateWithFlags(&ex->side, cudaStreamNonBlocking) == cudaSuccess;
-  cuda_ok &= cudaEventCreateWithFlags(&ex->ev_fork, cudaEventDisableTiming) == cudaSuccess;
-  cuda_ok &= cudaEventCreateWithFlags(&ex->ev_join, cudaEventDisableTiming) == cudaSuccess;
   if (cuda_ok) {
     const uint64_t n_q = static_cast<uint64_t>(cfg->n_heads) * cfg->head_dim;
     rc = hb_tmap_2d_bf16(&c->tm_h, c->h, lay.rows_pad, cfg->d_model, 128);
@@ -331,9 +325,6 @@ int hb_destroy(hb_ctx* c) {
       if (ex->ring[i].host) cudaFreeHost(ex->ring[i].host);
       if (ex->ring[i].ev) cudaEventDestroy(ex->ring[i].ev);
     }
-    if (ex->side) cudaStreamDestroy(ex->side);
-    if (ex->ev_fork) cudaEventDestroy(ex->ev_fork);
-    if (ex->ev_join) cudaEventDestroy(ex->ev_join);
     for (auto* v : {&ex->free_recs, &ex->used_recs})
       for (ProfRec& r : *v) {
         cudaEventDestroy(r.a);
@@ -694,9 +685,6 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   // Kernels after the first may become resident while their predecessor drains (programmatic
   // dependent launch); not while per-launch events are being recorded between them.
   const bool pdl_enabled = !ex->profiling;
-  // with enough work of both kinds the two attention kernels run side by side (measured 0.6-0.8 ms
-  // per 7B step); small steps stay on one stream, where the extra event calls would cost more
-  const bool fork_attention = !ex->profiling && dd.n_tc_items >= 64 && dd.n_attn_items >= 64;
   c->pdl = false;
   auto prof_begin = [&](int cls) -> ProfRec* {
     if (!ex->profiling) return nullptr;
@@ -799,22 +787,14 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.k2_blocks = use_lora ? r3 / 64 : 0;
     HB_TRY(HB_CLASS_GEMM, hb_gemm_launch(c->tm_h, wm.qkv, v_qkv, HB_EPI_QKV_ROPE, ga, c->num_sms, s,
                                          use_lora ? &c->tm_lora_u : nullptr, use_lora ? &lm->b_qkv : nullptr, c->pdl));
-    if (fork_attention) {
-      // The two attention kernels read the same q and pages and write disjoint rows of attn_out:
-      // run them side by side so that each fills the SMs the other's ragged last wave leaves idle.
-      if (cudaEventRecord(ex->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ex->side, ex->ev_fork, 0) != cudaSuccess)
-        return HB_ERR_CUDA;
-      c->pdl = false;
-      if ((rc = hb_launch_attention_tc(c, kg, kv->map, l, ex->side)) != HB_OK) return rc;
-      if (cudaEventRecord(ex->ev_join, ex->side) != cudaSuccess) return HB_ERR_CUDA;
-      rc = hb_launch_attention(c, kg, kv->map, l, s);
-      // join even if the second launch failed: nothing later on `s` may overtake the side stream
-      if (cudaStreamWaitEvent(s, ex->ev_join, 0) != cudaSuccess) return HB_ERR_CUDA;
-      if (rc != HB_OK) return rc;
-      launches += 2;
-    } else {
-      if (dd.n_tc_items > 0) HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention_tc(c, kg, kv->map, l, s));
-      if (dd.n_attn_items > 0) HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s));
+    if (ex->profiling) {
+      // timed per class: one launch per item list (the same kernel over one list)
+      if (dd.n_tc_items > 0)
+        HB_TRY(HB_CLASS_ATTENTION_TC, hb_launch_attention(c, kg, kv->map, l, s, HB_ATTN_CHUNK_TILES));
+      if (dd.n_attn_items > 0)
+        HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s, HB_ATTN_SMALL_ITEMS));
+    } else if (dd.n_tc_items + dd.n_attn_items > 0) {
+      HB_TRY(HB_CLASS_ATTENTION, hb_launch_attention(c, kg, kv->map, l, s, HB_ATTN_ALL));
     }
     // O projection, added to the residual stream
     ga.C = c->x; ga.N = cfg.d_model; ga.K = n_q; ga.ldc = cfg.d_model;
