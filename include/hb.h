@@ -302,14 +302,16 @@ HB_API int hb_status_poll(hb_ctx* ctx, void* stream, uint32_t* out_code);
 /* Per-kernel-class device timing.  While enabled, hb_mixed_step brackets every launch with a
  * pair of CUDA events on the step's stream; hb_profile_read synchronises them, adds the
  * elapsed milliseconds and launch counts per class into the two arrays of HB_N_CLASSES
- * entries, and clears the record.  Classes: */
+ * entries, and clears the record.  While enabled, launches do not overlap one another and
+ * the layer's one attention launch is issued once per item list (classes 1 and 5), so the
+ * launch count of a step is higher than in normal operation.  Classes: */
 enum {
   HB_CLASS_GEMM = 0,      /* QKV, O, gate/up, down projections                          */
-  HB_CLASS_ATTENTION = 1, /* paged attention: decode splits and short chunk tiles       */
+  HB_CLASS_ATTENTION = 1, /* attention launch (when timed: decode splits, short chunk tiles) */
   HB_CLASS_NORM_ROPE = 2, /* gather + RMSNorm, RMSNorm, RoPE + KV append                */
   HB_CLASS_POOL = 3,      /* final RMSNorm + pooler / logits-row preparation            */
   HB_CLASS_LM_HEAD = 4,   /* LM-head projection                                         */
-  HB_CLASS_ATTENTION_TC = 5, /* chunk-row attention on the tcgen05 tensor cores         */
+  HB_CLASS_ATTENTION_TC = 5, /* when timed: the attention launch's tcgen05 chunk tiles alone */
   HB_CLASS_LORA = 6,      /* adapters: rank-r activations of the embedding rows         */
   HB_N_CLASSES = 7
 };
