@@ -841,7 +841,10 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     ga.status = c->status;
     ga.b_kshift = 1;  // A holds (hi, lo) 64-column blocks: each weight k-block is used twice
     ga.M = dd.n_logit; ga.N = cfg.vocab; ga.K = 2 * cfg.d_model; ga.ldc = cfg.vocab; ga.C = out_logits;
-    HB_TRY(HB_CLASS_LM_HEAD, hb_gemm_launch(c->tm_logit_in, c->tm_lm, 128, HB_EPI_F32, ga, c->num_sms, s, nullptr,
+    // a few logits rows stream the weights through single-CTA tiles; hundreds of them (decode-heavy
+    // steps) are a real contraction and take the pair tiles (same boxes, same bits)
+    const int v_lm = hb_gemm_pick_step_variant(128, dd.n_logit, cfg.vocab, (2 * cfg.d_model + 63) / 64, 1, c->num_sms);
+    HB_TRY(HB_CLASS_LM_HEAD, hb_gemm_launch(c->tm_logit_in, c->tm_lm, v_lm, HB_EPI_F32, ga, c->num_sms, s, nullptr,
                                             nullptr, c->pdl));
   }
 #undef HB_TRY
