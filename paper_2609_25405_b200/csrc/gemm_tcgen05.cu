@@ -267,7 +267,10 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   // adapted projection, with A2 = the rows' rank-r activations and B2 = the up factor).
   const int k1_blocks = (g.K + BK - 1) / BK;
   const int k_blocks = k1_blocks + g.k2_blocks;
-  const int k_per_split = (k_blocks + k_splits - 1) / k_splits;
+  // Splits share the main K blocks evenly; the second pair's blocks all go to the last split, so
+  // that where a row's sum is cut does not depend on whether the launch carries a second pair (a
+  // generation row's bits must not change when embedding rows with an adapter join its batch).
+  const int k_per_split = (k1_blocks + k_splits - 1) / k_splits;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T::STAGES; ++s) {
@@ -322,7 +325,8 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const int mn = tile % mn_tiles, split = tile / mn_tiles;
         const int m0 = (mn % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
         const int n0 = (mn / m_tiles) * BN + static_cast<int>(rank) * T::B_ROWS;
-        const int kb0 = split * k_per_split, kb1 = min(kb0 + k_per_split, k_blocks);
+        const int kb0 = split * k_per_split;
+        const int kb1 = (split + 1 == k_splits) ? k_blocks : min(kb0 + k_per_split, k1_blocks);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
           const uint32_t a_dst = smem_base + stage * T::STAGE_BYTES;
@@ -365,7 +369,8 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         const int split = tile / mn_tiles;
-        const int kb0 = split * k_per_split, kb1 = min(kb0 + k_per_split, k_blocks);
+        const int kb0 = split * k_per_split;
+        const int kb1 = (split + 1 == k_splits) ? k_blocks : min(kb0 + k_per_split, k1_blocks);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
           tc_fence_after();

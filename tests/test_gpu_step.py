@@ -312,6 +312,57 @@ def test_batch_composition_independence(weights):
     assert torch.equal(e_batch, e_solo)
 
 
+@pytest.mark.parametrize("lora_rank", [0, 16])
+def test_batch_composition_independence_across_step_sizes_full_width(lora_rank):
+    """7B-class width, two layers, random weights drawn on the device, a 4096-row context: a
+    generation and an embedding request run alone, every piece of work a step of its own (300, 512, 1
+    and 188 rows, most of which take single-CTA GEMM tiles), equal bit for bit the same requests inside
+    full 4096-row steps (CTA-pair tiles; the down projection's K is split in two in both).  No oracle
+    here: the point is that tile variants and K splits chosen per step or per context never change a
+    row's bits."""
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Engine, Request
+    shape = synth.SHAPES["7b"].with_layers(2)
+    dw = B.DeviceWeights.random_on_device(shape, seed=3)
+    lora = B.DeviceLora.random_on_device(shape, lora_rank) if lora_rank else None
+    rng = np.random.default_rng(77)
+    emb_toks = synth.token_ids(rng, 700, shape.V)
+    gen_toks = synth.token_ids(rng, 300, shape.V)
+
+    def run(fill):
+        eng = Engine(shape, dw, n_pages=1024, n_slots=64, max_tokens=4096, max_segs=64, max_pos=1024, lora=lora)
+        e, g = Request("embed", list(emb_toks), B.POOL_MEAN), Request("gen", list(gen_toks))
+        outs, extra = [], []
+        for step in range(2):
+            work = [(g, 300)] if step == 0 else [(g, 1)]
+            if step == 1:
+                g.tokens.append(7)
+            work.append((e, 512 if step == 0 else 188))
+            rows = sum(n for _, n in work)
+            while fill and rows < 4096:
+                n = min(512, 4096 - rows)
+                f = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_LAST)
+                work.append((f, n)); extra.append(f); rows += n
+            for part in ([work] if fill else [[w] for w in work]):
+                _, l1, e1 = eng.step(part)
+                torch.cuda.synchronize()
+                if g in l1:
+                    outs.append(eng.out_logits[l1[g]].clone())
+                if e in e1:
+                    outs.append(eng.out_emb[e1[e]].clone())
+            for f in extra:
+                eng.release(f)
+            extra = []
+        assert eng.ctx.status_poll() == 0
+        eng.close()
+        return outs
+
+    solo, batch = run(False), run(True)
+    assert len(solo) == len(batch) == 3
+    for a, b in zip(solo, batch):
+        assert torch.isfinite(a).all() and torch.equal(a, b)
+
+
 def test_argmax_kernel_lowest_index_on_ties(weights):
     eng = _engine(weights)
     lg = torch.randn(5, TINY.V, device="cuda")
