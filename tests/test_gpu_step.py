@@ -330,7 +330,7 @@ def test_batch_composition_independence_across_step_sizes_full_width(lora_rank):
     gen_toks = synth.token_ids(rng, 300, shape.V)
 
     def run(fill):
-        eng = Engine(shape, dw, n_pages=1024, n_slots=64, max_tokens=4096, max_segs=64, max_pos=1024, lora=lora)
+        eng = Engine(shape, dw, n_pages=1024, n_slots=64, max_tokens=4096, max_segs=256, max_pos=1024, lora=lora)
         e, g = Request("embed", list(emb_toks), B.POOL_MEAN), Request("gen", list(gen_toks))
         outs, extra = [], []
         for step in range(2):
@@ -339,6 +339,9 @@ def test_batch_composition_independence_across_step_sizes_full_width(lora_rank):
                 g.tokens.append(7)
             work.append((e, 512 if step == 0 else 188))
             rows = sum(n for _, n in work)
+            for _ in range(200 if fill else 0):      # 200 more logits rows: the LM head takes pair tiles
+                f = Request("gen", synth.token_ids(rng, 4, shape.V))
+                work.append((f, 4)); extra.append(f); rows += 4
             while fill and rows < 4096:
                 n = min(512, 4096 - rows)
                 f = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_LAST)
