@@ -312,9 +312,10 @@ def test_batch_composition_independence(weights):
     assert torch.equal(e_batch, e_solo)
 
 
+@pytest.mark.parametrize("width", ["7b", "1b"])
 @pytest.mark.parametrize("lora_rank", [0, 16])
-def test_batch_composition_independence_across_step_sizes_full_width(lora_rank):
-    """7B-class width, two layers, random weights drawn on the device, a 4096-row context: a
+def test_batch_composition_independence_across_step_sizes_full_width(lora_rank, width):
+    """7B-class (and 1B-class) width, two layers, random weights drawn on the device, a 4096-row context: a
     generation and an embedding request run alone, every piece of work a step of its own (300, 512, 1
     and 188 rows, most of which take single-CTA GEMM tiles), equal bit for bit the same requests inside
     full 4096-row steps (CTA-pair tiles; the down projection's K is split in two in both).  No oracle
@@ -322,7 +323,7 @@ def test_batch_composition_independence_across_step_sizes_full_width(lora_rank):
     row's bits."""
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
-    shape = synth.SHAPES["7b"].with_layers(2)
+    shape = synth.SHAPES[width].with_layers(2)
     dw = B.DeviceWeights.random_on_device(shape, seed=3)
     lora = B.DeviceLora.random_on_device(shape, lora_rank) if lora_rank else None
     rng = np.random.default_rng(77)
