@@ -503,6 +503,59 @@ def test_fp32_oracle_close_to_fp64():
 
 
 # --------------------------------------------------------------------------
+# the single projection with its epilogues (oracle/ops.py), which the GEMM unit tests rest on
+# --------------------------------------------------------------------------
+
+def test_projection_epilogues_match_torch_linear_with_separate_gate_and_up():
+    """ops.projection against torch: the plain product against F.linear, the residual form against
+    C0 + F.linear, and the SwiGLU form against silu(F.linear(x, Wg)) * F.linear(x, Wu) with gate
+    and up given as SEPARATE matrices that this test interleaves itself (row 2j = gate row j, row
+    2j + 1 = up row j, the layout the library documents for w_gate_up).  Swapping gate and up,
+    dropping the residual or transposing an operand in ops.projection fails here."""
+    from oracle import ops
+    import torch.nn.functional as Fn
+    rng = np.random.default_rng(3)
+    M_, K, F_ = 5, 12, 7
+    x = rng.standard_normal((M_, K))
+    wg, wu = rng.standard_normal((F_, K)), rng.standard_normal((F_, K))
+    c0 = rng.standard_normal((M_, F_))
+    tx, tg, tu = (torch.from_numpy(a) for a in (x, wg, wu))
+    assert np.allclose(ops.projection(x, wg, "plain"), Fn.linear(tx, tg).numpy(), atol=1e-12)
+    assert np.allclose(ops.projection(x, wg, "resid", c0), c0 + Fn.linear(tx, tg).numpy(), atol=1e-12)
+    inter = np.empty((2 * F_, K))
+    inter[0::2], inter[1::2] = wg, wu
+    ref = (Fn.silu(Fn.linear(tx, tg)) * Fn.linear(tx, tu)).numpy()
+    got = ops.projection(x, inter, "swiglu")
+    assert got.shape == (M_, F_) and np.allclose(got, ref, atol=1e-12)
+    swapped = np.empty_like(inter)
+    swapped[0::2], swapped[1::2] = wu, wg
+    assert not np.allclose(ops.projection(x, swapped, "swiglu"), ref, atol=1e-3)   # the order matters
+    # the same inside the whole model: one FFN block of transformer.forward is this projection chain
+    h = rng.standard_normal((M_, K))
+    wd = rng.standard_normal((K, F_))
+    ffn = ops.projection(ops.projection(h, inter, "swiglu"), wd, "resid", x)
+    assert np.allclose(ffn, x + (T.silu(h @ wg.T) * (h @ wu.T)) @ wd.T, atol=1e-12)
+
+
+def test_projection_two_by_two_by_hand():
+    """A 2 x 2 case worked by hand.  A = [[1, 2], [0, -1]], B rows = (gate, up) = ([1, 0], [0, 1]):
+    A B^T = A itself, so plain = A, resid with C0 = 10 everywhere = A + 10, and swiglu has one
+    output column: silu(gate) * up = silu(1) * 2 and silu(0) * (-1) = 0 (silu(0) = 0,
+    silu(1) = 1 / (1 + e^-1))."""
+    from oracle import ops
+    A = np.array([[1.0, 2.0], [0.0, -1.0]])
+    Bm = np.array([[1.0, 0.0], [0.0, 1.0]])
+    assert np.array_equal(ops.projection(A, Bm, "plain"), A)
+    assert np.array_equal(ops.projection(A, Bm, "resid", np.full((2, 2), 10.0)), A + 10.0)
+    sw = ops.projection(A, Bm, "swiglu")
+    assert sw.shape == (2, 1)
+    assert abs(sw[0, 0] - 2.0 / (1.0 + np.exp(-1.0))) < 1e-15 and sw[1, 0] == 0.0
+    # a non-symmetric B tells A B^T from A B: B = [[1, 1], [0, 1]] gives rows (a0 + a1, a1)
+    B2 = np.array([[1.0, 1.0], [0.0, 1.0]])
+    assert np.array_equal(ops.projection(A, B2, "plain"), np.array([[3.0, 2.0], [-1.0, -1.0]]))
+
+
+# --------------------------------------------------------------------------
 # values the paper prints
 # --------------------------------------------------------------------------
 
