@@ -14,7 +14,12 @@
  *  - "host" / "device" is stated for every pointer; device pointers are plain
  *    CUDA device addresses on the current device; `stream` is a cudaStream_t
  *    passed as void* (NULL = the legacy default stream);
- *  - the library never frees caller memory; hb_mixed_step allocates nothing;
+ *  - the library never frees caller memory; hb_mixed_step allocates no device
+ *    memory, and its host scratch (work lists, validation marks, the pinned
+ *    descriptor staging) belongs to the context: it is reserved by hb_create
+ *    for the context's limits and only grows if a step meets a KV cache or
+ *    pool with more pages / slots than any step before (per-class timing,
+ *    hb_profile_enable, creates its CUDA events on demand);
  *  - all work is enqueued on `stream`; outputs are valid once the caller has
  *    synchronised that stream;
  *  - there is no CPU path: without a CUDA device every compute call fails.
@@ -49,8 +54,8 @@ enum {
 };
 
 /* Row kinds of the batch unit (Section 3.2).  Rows of one kind are contiguous
- * and kinds appear in this order (the scheduler "outputs batches sorted by
- * request type"). */
+ * and kinds appear in this order (Section 3.2 has the scheduler hand over each
+ * batch already grouped by kind, so every output head reads one slice). */
 enum { HB_KIND_DECODE = 0, HB_KIND_PREFILL_CHUNK = 1, HB_KIND_EMBED_CHUNK = 2 };
 
 /* Pooling heads (Section 3.3).  Additive (Eq. 1-2): mean (w = 1) and weighted
@@ -231,8 +236,10 @@ HB_API int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t
  *   out_emb     device float [>= n_emb_rows, d_model]; row seg.emb_row gets the
  *               L2-normalised embedding of a request whose final chunk ran
  * Rows of the outputs not named by a segment are left untouched.  Returns
- * after enqueueing; no synchronisation, no allocation.  A failed validation
- * enqueues nothing. */
+ * after enqueueing; no synchronisation, no device allocation.  A failed
+ * validation enqueues nothing.  Alignment (checked, HB_ERR_BAD_ARG): out_logits,
+ * out_emb and tok_emb 16 bytes, every norm gain 8 bytes (the kernels use
+ * 16-byte and 8-byte vector accesses); projection weights 16 bytes. */
 HB_API int hb_mixed_step(hb_ctx* ctx, const hb_batch_desc* desc, const hb_weights* w, hb_kv* kv,
                   hb_pool* pool, float* out_logits, float* out_emb, void* stream);
 
@@ -295,8 +302,20 @@ HB_API int hb_argmax(hb_ctx* ctx, const float* logits, int32_t n_rows, int32_t* 
               void* stream);
 
 /* Read (and clear) the device status word; synchronises `stream`.  0 = clean.
- * Non-zero: a bounded wait inside a kernel expired or an index check failed;
- * *out_code holds the kernel-specific code.  Returns HB_ERR_DEVICE_STATUS then. */
+ * Non-zero: *out_code holds the OR of the bits below and the call returns
+ * HB_ERR_DEVICE_STATUS.  Bits 0-5 mean a kernel gave up (a bounded wait expired,
+ * an index check failed: outputs of that step are not valid); bit 6 is a value
+ * report: the step ran, but an activation did not fit fp16. */
+enum {
+  HB_STATUS_GEMM_WAIT = 1,        /* projection GEMM: a pipeline wait expired                 */
+  HB_STATUS_ATTN_INDEX = 2,       /* attention: page id out of range                          */
+  HB_STATUS_APPEND_INDEX = 4,     /* KV append: page id out of range (row not written)        */
+  HB_STATUS_POOL_INDEX = 8,       /* pooler: slot / row buffer out of range                   */
+  HB_STATUS_ATTN_WAIT = 16,       /* attention: a pipeline wait expired                       */
+  HB_STATUS_SELFTEST_WAIT = 32,   /* hb_selftest_wait_expiry                                  */
+  HB_STATUS_F16_RANGE = 64        /* a normed row or a SwiGLU output was NaN or beyond +-65504:
+                                     finite values were stored saturated, NaN was stored as NaN */
+};
 HB_API int hb_status_poll(hb_ctx* ctx, void* stream, uint32_t* out_code);
 
 /* Per-kernel-class device timing.  While enabled, hb_mixed_step brackets every launch with a
@@ -370,7 +389,9 @@ HB_API int hb_gemm_pair(hb_ctx* ctx, const void* A, const void* B, const void* A
  *   slot_sum   device float [d_model], slot_meta device uint32 [4] =
  *              {count, chunks, mode, state}: the request's pool slot (in/out)
  *   out_emb    device float [d_model] (written when is_final != 0)
- * n_rows <= the context's max_tokens.  Uses the context's scratch. */
+ * n_rows <= the context's max_tokens.  Uses the context's scratch.  x,
+ * slot_sum and out_emb must be 16-byte aligned, gain 8-byte aligned (vector
+ * accesses); a misaligned pointer is HB_ERR_BAD_ARG and nothing is launched. */
 HB_API int hb_pool_chunk(hb_ctx* ctx, const float* x, const void* gain, int32_t n_rows, int32_t mode,
                          int32_t first_chunk, int32_t is_final, float* slot_sum, uint32_t* slot_meta,
                          float* out_emb, void* stream);
@@ -407,7 +428,17 @@ HB_API int hb_pool_chunk(hb_ctx* ctx, const float* x, const void* gain, int32_t 
  *    Two calls whose kernels can run at the same time on that device -- from
  *    different streams or threads -- race on it: serialise them;
  *  - the caller still owns and passes every input and output (x, gain,
- *    slot_sum, slot_meta, out_emb: device pointers as in hb_pool_chunk). */
+ *    slot_sum, slot_meta, out_emb: device pointers as in hb_pool_chunk), with
+ *    the same alignment rule: x, slot_sum, out_emb 16 bytes, gain 8 bytes.  A
+ *    view cut out of a larger arena at an odd offset is refused with
+ *    HB_ERR_BAD_ARG before anything is launched;
+ *  - the looked-up address is cached for the life of the process.  After
+ *    cudaDeviceReset on that device it is stale: do not call this entry again
+ *    in a process that reset the device;
+ *  - there is no context, so no hb_status_poll: the status word the kernel
+ *    keeps in the array's tail is write-only for callers.  The only device
+ *    check behind it (pool slot in range) cannot fail here, because this entry
+ *    always runs on a one-slot pool it builds itself. */
 HB_API int hb_pool_chunk_noalloc(const float* x, const void* gain, int32_t n_rows, int32_t d_model,
                                  float rms_eps, int32_t mode, int32_t first_chunk, int32_t is_final,
                                  float* slot_sum, uint32_t* slot_meta, float* out_emb, void* stream);

@@ -332,20 +332,32 @@ class DeviceLora:
         return self
 
 
-class KvCache:
-    """Caller-owned KV arena (torch) + the library's page free list."""
+def kv_arena_bytes(cfg, n_pages):
+    nbytes = C.c_size_t()
+    check(lib.hb_kv_arena_bytes(C.byref(cfg), n_pages, C.byref(nbytes)), "hb_kv_arena_bytes")
+    return nbytes.value
 
-    def __init__(self, cfg, n_pages, device="cuda", fill=None):
+
+class KvCache:
+    """Caller-owned KV arena (torch) + the library's page free list.  `arena`: an int16 tensor to
+    use instead of allocating one (it must hold n_pages; several caches may be laid over one
+    buffer one after the other)."""
+
+    def __init__(self, cfg, n_pages, device="cuda", fill=None, arena=None):
         self.cfg = cfg
         self.n_pages = n_pages
-        nbytes = C.c_size_t()
-        check(lib.hb_kv_arena_bytes(C.byref(cfg), n_pages, C.byref(nbytes)), "hb_kv_arena_bytes")
+        nbytes = C.c_size_t(kv_arena_bytes(cfg, n_pages))
         self.handle = C.c_void_p()
         if device is None:      # bookkeeping only (host tests): no arena
             self.arena = None
             check(lib.hb_kv_create(C.byref(cfg), None, 0, n_pages, C.byref(self.handle)), "hb_kv_create")
             return
-        self.arena = torch.empty(nbytes.value // 2, dtype=torch.int16, device=device)
+        if arena is not None:
+            if arena.dtype != torch.int16 or arena.numel() * 2 < nbytes.value:
+                raise ValueError("arena too small for n_pages")
+            self.arena = arena[: nbytes.value // 2]
+        else:
+            self.arena = torch.empty(nbytes.value // 2, dtype=torch.int16, device=device)
         if fill is not None:
             self.arena.fill_(fill)
         check(lib.hb_kv_create(C.byref(cfg), C.c_void_p(self.arena.data_ptr()), nbytes.value, n_pages,

@@ -45,15 +45,11 @@ template <int DH>
 int launch(const CUtensorMap& kv_map, const hb_tc::TcParams& tp, const hb_dec::AttnParams& dp, int n_tc, int n_small,
            int max_pos, cudaStream_t s, bool pdl) {
   const int smem = std::max(n_tc > 0 ? hb_tc::smem_bytes<DH>() : 0, n_small > 0 ? hb_dec::smem_bytes<DH>(max_pos) : 0);
-  static int configured[2] = {0, 0};
+  static DynSmemState configured[2];   // per instantiation and per device
   if (smem > 227 * 1024) return HB_ERR_UNSUPPORTED;
   const int v = n_tc > 0 ? 1 : 0;
   auto kern = v ? attn_varlen_kernel<DH, true> : attn_varlen_kernel<DH, false>;
-  if (configured[v] < smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return HB_ERR_CUDA;
-    configured[v] = smem;
-  }
+  if (hb_ensure_dyn_smem(reinterpret_cast<const void*>(kern), configured[v], smem) != HB_OK) return HB_ERR_CUDA;
   return hb_launch_kernel(kern, n_tc + n_small, ATTN_THREADS, smem, s, pdl, kv_map, tp, dp, n_tc, n_small);
 }
 

@@ -8,9 +8,9 @@
 
 namespace {
 
-// Activations leave these kernels as fp16 (three more mantissa bits than bf16), saturating at
-// the largest finite half.
-__device__ __forceinline__ float sat_h(float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); }
+// Activations leave these kernels as fp16 (three more mantissa bits than bf16); finite values
+// saturate at the largest finite half, NaN stays NaN.
+__device__ __forceinline__ float sat_h(float v) { return sat_half_range(v); }
 
 __device__ __forceinline__ uint2 float4_to_f16x4(float4 v) {
   __half2 a = __floats2half2_rn(sat_h(v.x), sat_h(v.y)), b = __floats2half2_rn(sat_h(v.z), sat_h(v.w));
@@ -33,7 +33,7 @@ template <bool GATHER, int NV>
 __global__ void __launch_bounds__(NORM_THREADS, NV == 4 ? 8 : 4)
 norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E,
             const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __half* __restrict__ h,
-            int d, float eps) {
+            int d, float eps, uint32_t* __restrict__ status) {
   grid_dep_wait();
   grid_dep_launch();
   __shared__ float red[32];
@@ -59,6 +59,7 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
   const float tot = block_sum(ss, red);
   const float rstd = rsqrtf(tot / static_cast<float>(d) + eps);
   __half* hrow = h + static_cast<size_t>(t) * d;
+  bool range = false;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     const int v = threadIdx.x + i * NORM_THREADS;
@@ -67,9 +68,12 @@ norm_kernel(const int32_t* __restrict__ tok, const __nv_bfloat16* __restrict__ E
       bf16x4_to_float4(*reinterpret_cast<const uint2*>(gain + 4 * v), g);
       float4 o = make_float4(buf[i].x * rstd * g.x, buf[i].y * rstd * g.y, buf[i].z * rstd * g.z,
                              buf[i].w * rstd * g.w);
+      range |= outside_half_range(o.x) | outside_half_range(o.y) | outside_half_range(o.z) | outside_half_range(o.w);
       *reinterpret_cast<uint2*>(hrow + 4 * v) = float4_to_f16x4(o);
     }
   }
+  // a normed row that does not fit fp16 (a NaN in the residual stream, a gain far above 1) is reported
+  if (range) atomicOr(status, HB_DEV_F16_RANGE);
 }
 
 // Final RMSNorm of the rows that feed the LM head, written as a (hi, lo) fp16 pair:
@@ -212,18 +216,20 @@ int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaS
   if (c->cfg.d_model <= 4 * 4 * NORM_THREADS)
     return hb_launch_kernel(norm_kernel<true, 4>, c->dd.T, NORM_THREADS, 0, s, c->pdl, c->dd.tok,
                             static_cast<const __nv_bfloat16*>(tok_emb), static_cast<const __nv_bfloat16*>(gain), c->x,
-                            c->h, c->cfg.d_model, c->cfg.rms_eps);
+                            c->h, c->cfg.d_model, c->cfg.rms_eps, c->status);
   return hb_launch_kernel(norm_kernel<true, MAX_VEC>, c->dd.T, NORM_THREADS, 0, s, c->pdl, c->dd.tok,
                           static_cast<const __nv_bfloat16*>(tok_emb), static_cast<const __nv_bfloat16*>(gain), c->x,
-                          c->h, c->cfg.d_model, c->cfg.rms_eps);
+                          c->h, c->cfg.d_model, c->cfg.rms_eps, c->status);
 }
 
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s) {
   if (c->cfg.d_model <= 4 * 4 * NORM_THREADS)
     return hb_launch_kernel(norm_kernel<false, 4>, c->dd.T, NORM_THREADS, 0, s, c->pdl, nullptr, nullptr,
-                            static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps);
+                            static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps,
+                            c->status);
   return hb_launch_kernel(norm_kernel<false, MAX_VEC>, c->dd.T, NORM_THREADS, 0, s, c->pdl, nullptr, nullptr,
-                          static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps);
+                          static_cast<const __nv_bfloat16*>(gain), c->x, c->h, c->cfg.d_model, c->cfg.rms_eps,
+                          c->status);
 }
 
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta, int n_slots,

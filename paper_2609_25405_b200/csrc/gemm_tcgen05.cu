@@ -110,13 +110,18 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int row, int c
     for (int v = 0; v < 2; ++v) {
       if (col0 + v * 16 < g.N) {
         uint32_t pk[4];
+        bool range = false;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const float g0 = __uint_as_float(r[v * 16 + j * 4 + 0]), u0 = __uint_as_float(r[v * 16 + j * 4 + 1]);
           const float g1 = __uint_as_float(r[v * 16 + j * 4 + 2]), u1 = __uint_as_float(r[v * 16 + j * 4 + 3]);
-          pk[j] = pack_half2_sat(silu_f(g0) * u0, silu_f(g1) * u1);
+          const float a0 = silu_f(g0) * u0, a1 = silu_f(g1) * u1;
+          range |= outside_half_range(a0) | outside_half_range(a1);
+          pk[j] = pack_half2_sat(a0, a1);
         }
         *reinterpret_cast<uint4*>(out + v * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        // the FFN's inner activation is the widest-ranging fp16 value of the step: report, do not hide
+        if (range) atomicOr(g.status, HB_DEV_F16_RANGE);
       }
     }
   }
@@ -566,13 +571,9 @@ template <int BN, int EPI, int CG>
 int launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
                const GemmArgs& a, int num_sms, cudaStream_t s, bool pdl) {
   using T = Tile<BN, CG>;
-  static bool configured = false;
+  static DynSmemState configured;   // per device: a second GPU in the process needs the attribute too
   auto kern = hb_gemm_tcgen05_kernel<BN, EPI, CG>;
-  if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM_BYTES) != cudaSuccess)
-      return HB_ERR_CUDA;
-    configured = true;
-  }
+  if (hb_ensure_dyn_smem(reinterpret_cast<const void*>(kern), configured, T::SMEM_BYTES) != HB_OK) return HB_ERR_CUDA;
   const int m_tiles = (a.M + BM * CG - 1) / (BM * CG);
   const int n_tiles = (a.N + BN - 1) / BN;
   int workers = m_tiles * n_tiles *
@@ -614,7 +615,7 @@ int launch_bn(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap&
 
 }  // namespace
 
-int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+int hb_tmap_2d_f16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return HB_ERR_CUDA;
   if ((reinterpret_cast<uintptr_t>(base) & 15u) || (cols & 7u) || rows == 0 || cols == 0) return HB_ERR_BAD_ARG;
@@ -622,7 +623,7 @@ int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t 
   const cuuint64_t strides[1] = {cols * 2};
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK), box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+  const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box,
                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? HB_OK : HB_ERR_CUDA;

@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <vector>
 
 #include "../../include/hb.h"
@@ -19,6 +20,7 @@ enum : uint32_t {
   HB_DEV_POOL_BAD_INDEX = 1u << 3,
   HB_DEV_ATTN_WAIT_EXPIRED = 1u << 4,
   HB_DEV_SELFTEST_WAIT_EXPIRED = 1u << 5,
+  HB_DEV_F16_RANGE = 1u << 6,   // a normed row or a SwiGLU output was NaN or beyond the largest finite half
 };
 
 // Attention work item: one (segment, kv head, row tile, key split).
@@ -132,8 +134,28 @@ struct GemmArgs {
   int32_t Hq, Hkv, Dh, P, n_pages;
 };
 
-int hb_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
-                    uint32_t box_rows);
+// 2-D tensor map over a row-major 16-bit matrix (fp16 everywhere in this library), 64-column boxes,
+// 128-byte swizzle.
+int hb_tmap_2d_f16(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
+                   uint32_t box_rows);
+
+// Dynamic shared memory above 48 KiB has to be enabled per kernel ON EVERY DEVICE the kernel runs
+// on.  One of these per kernel instantiation remembers, per device, the largest size enabled so
+// far; hb_ensure_dyn_smem raises it on the current device when a launch needs more.
+constexpr int HB_MAX_DEVICES = 64;
+struct DynSmemState {
+  std::atomic<int> bytes[HB_MAX_DEVICES];
+};
+inline int hb_ensure_dyn_smem(const void* kern, DynSmemState& st, int bytes) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= HB_MAX_DEVICES) return HB_ERR_CUDA;
+  if (st.bytes[dev].load(std::memory_order_acquire) >= bytes) return HB_OK;
+  // two threads may both get here: the attribute call is idempotent
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return HB_ERR_CUDA;
+  int seen = st.bytes[dev].load(std::memory_order_relaxed);
+  while (seen < bytes && !st.bytes[dev].compare_exchange_weak(seen, bytes, std::memory_order_release)) {}
+  return HB_OK;
+}
 // GEMM variants: 128 / 256 = one CTA per 128 x BN tile; HB_GEMM_PAIR256 = a CTA pair per 256 x 256 tile.
 // The B tensor map's box must have hb_gemm_box_rows(variant) rows.
 constexpr int HB_GEMM_PAIR256 = 512;

@@ -19,6 +19,8 @@ constexpr int N_STAGING = 4;    // pinned descriptor staging ring
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+bool misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
 bool cfg_ok(const hb_model_cfg* c) {
   if (!c) return false;
   if (c->n_layers < 1 || c->d_model < 64 || c->n_heads < 1 || c->n_kv_heads < 1 || c->d_ffn < 64 || c->vocab < 8)
@@ -97,8 +99,18 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   return L;
 }
 
+// Marks the validation needs (one byte per page / slot / output row).  A context keeps one and
+// reuses it, so that a step allocates host memory only when it meets a larger cache than any before.
+struct ValidateScratch {
+  std::vector<uint8_t> page_written, slot_used, lrow, erow;
+  static void zeroed(std::vector<uint8_t>& v, size_t n) {
+    if (v.size() < n) v.resize(n);
+    memset(v.data(), 0, n);
+  }
+};
+
 int validate(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids, int32_t n_pages,
-             int32_t n_slots, int32_t rowbuf_rows, const hb_batch_desc* d) {
+             int32_t n_slots, int32_t rowbuf_rows, const hb_batch_desc* d, ValidateScratch& vs) {
   if (!d) return HB_ERR_BAD_ARG;
   if (d->n_tokens < 0 || d->n_segs < 0 || d->n_page_ids < 0 || d->n_logit_rows < 0 || d->n_emb_rows < 0)
     return HB_ERR_BAD_DESC;
@@ -111,10 +123,14 @@ int validate(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_
   for (int32_t i = 0; i < d->n_page_ids; ++i)
     if (d->page_ids[i] < 0 || d->page_ids[i] >= n_pages) return HB_ERR_BAD_DESC;
   const int P = c.page_size;
-  std::vector<uint8_t> page_written(static_cast<size_t>(std::max(n_pages, 1)), 0);
-  std::vector<uint8_t> slot_used(static_cast<size_t>(std::max(n_slots, 1)), 0);
-  std::vector<uint8_t> lrow(static_cast<size_t>(std::max(d->n_logit_rows, 1)), 0);
-  std::vector<uint8_t> erow(static_cast<size_t>(std::max(d->n_emb_rows, 1)), 0);
+  ValidateScratch::zeroed(vs.page_written, static_cast<size_t>(std::max(n_pages, 1)));
+  ValidateScratch::zeroed(vs.slot_used, static_cast<size_t>(std::max(n_slots, 1)));
+  ValidateScratch::zeroed(vs.lrow, static_cast<size_t>(std::max(d->n_logit_rows, 1)));
+  ValidateScratch::zeroed(vs.erow, static_cast<size_t>(std::max(d->n_emb_rows, 1)));
+  uint8_t* page_written = vs.page_written.data();
+  uint8_t* slot_used = vs.slot_used.data();
+  uint8_t* lrow = vs.lrow.data();
+  uint8_t* erow = vs.erow.data();
   int32_t at = 0, prev_kind = 0, n_l = 0, n_e = 0;
   for (int32_t r = 0; r < d->n_segs; ++r) {
     const hb_seg& s = d->segs[r];
@@ -187,6 +203,11 @@ struct CtxExtra {
   Layout lay;
   bool profiling = false;
   std::vector<ProfRec> free_recs, used_recs;
+  // host scratch of a step, reserved at hb_create for the context's limits and reused by every call
+  ValidateScratch vscratch;
+  std::vector<PoolItem> pitems;
+  std::vector<AttnItem> aitems, titems;
+  std::vector<uint64_t> sort_keys;
 };
 
 CtxExtra* extra_of(hb_ctx* c) { return static_cast<CtxExtra*>(c->extra); }
@@ -219,6 +240,12 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   CtxExtra* ex = new (std::nothrow) CtxExtra();
   if (!c || !ex) { delete c; delete ex; return HB_ERR_BAD_ARG; }
   ex->lay = lay;
+  ex->pitems.reserve(static_cast<size_t>(lay.max_pool_items));
+  ex->aitems.reserve(static_cast<size_t>(lay.max_attn_items));
+  ex->titems.reserve(static_cast<size_t>(lay.max_attn_items));
+  ex->sort_keys.reserve(static_cast<size_t>(lay.max_attn_items));
+  ex->vscratch.lrow.resize(static_cast<size_t>(max_segs));
+  ex->vscratch.erow.resize(static_cast<size_t>(max_segs));
   c->cfg = *cfg;
   c->max_tokens = max_tokens;
   c->max_segs = max_segs;
@@ -301,11 +328,11 @@ int hb_create(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int
   }
   if (cuda_ok) {
     const uint64_t n_q = static_cast<uint64_t>(cfg->n_heads) * cfg->head_dim;
-    rc = hb_tmap_2d_bf16(&c->tm_h, c->h, lay.rows_pad, cfg->d_model, 128);
-    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_attn_out, c->attn_out, lay.rows_pad, n_q, 128);
-    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_act, c->act, lay.rows_pad, cfg->d_ffn, 128);
-    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_logit_in, c->logit_in, lay.logit_rows_pad, 2ull * cfg->d_model, 128);
-    if (rc == HB_OK) rc = hb_tmap_2d_bf16(&c->tm_lora_u, c->lora_u, lay.rows_pad, HB_LORA_U_COLS, 128);
+    rc = hb_tmap_2d_f16(&c->tm_h, c->h, lay.rows_pad, cfg->d_model, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_f16(&c->tm_attn_out, c->attn_out, lay.rows_pad, n_q, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_f16(&c->tm_act, c->act, lay.rows_pad, cfg->d_ffn, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_f16(&c->tm_logit_in, c->logit_in, lay.logit_rows_pad, 2ull * cfg->d_model, 128);
+    if (rc == HB_OK) rc = hb_tmap_2d_f16(&c->tm_lora_u, c->lora_u, lay.rows_pad, HB_LORA_U_COLS, 128);
   }
   cuda_ok &= cudaDeviceSynchronize() == cudaSuccess;
   if (!cuda_ok || rc != HB_OK) {
@@ -360,7 +387,7 @@ int hb_kv_create(const hb_model_cfg* cfg, void* arena, size_t arena_bytes, int32
     const uint64_t halves = cfg->head_dim / 64;
     const uint64_t rows = static_cast<uint64_t>(cfg->n_layers) * n_pages * cfg->n_kv_heads * 2 * halves * cfg->page_size;
     if (rows > 0x7fffffffull ||
-        hb_tmap_2d_bf16(&kv->map, arena, rows, 64, static_cast<uint32_t>(2 * halves * cfg->page_size)) != HB_OK) {
+        hb_tmap_2d_f16(&kv->map, arena, rows, 64, static_cast<uint32_t>(2 * halves * cfg->page_size)) != HB_OK) {
       delete kv;
       return rows > 0x7fffffffull ? HB_ERR_TOO_LARGE : HB_ERR_CUDA;
     }
@@ -485,7 +512,8 @@ int hb_pool_free_slot(hb_pool* p, int32_t slot) {
 int hb_validate_desc(const hb_model_cfg* cfg, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids,
                      int32_t n_pages, int32_t n_slots, const hb_batch_desc* desc) {
   if (!cfg_ok(cfg)) return HB_ERR_BAD_ARG;
-  return validate(*cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, cfg->max_pos, desc);
+  ValidateScratch vs;   // a stand-alone check has no context to keep its marks in
+  return validate(*cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, cfg->max_pos, desc, vs);
 }
 
 int hb_mixed_step(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, hb_kv* kv, hb_pool* pool,
@@ -502,10 +530,14 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   if (memcmp(&kv->cfg, &c->cfg, sizeof(hb_model_cfg)) != 0) return HB_ERR_BAD_ARG;
   const int32_t n_slots = pool ? pool->n_slots : 0;
   int rc = validate(c->cfg, c->max_tokens, c->max_segs, c->max_page_ids, kv->n_pages, n_slots,
-                    pool ? pool->rowbuf_rows : 0, d);
+                    pool ? pool->rowbuf_rows : 0, d, extra_of(c)->vscratch);
   if (rc != HB_OK) return rc;
   if (d->n_logit_rows > 0 && (!out_logits || !w->lm_head)) return HB_ERR_BAD_ARG;
   if (d->n_emb_rows > 0 && !out_emb) return HB_ERR_BAD_ARG;
+  // the kernels read and write these with 16-byte (gains: 8-byte) vectors
+  if (misaligned(out_logits, 16) || misaligned(out_emb, 16) || misaligned(w->tok_emb, 16) ||
+      misaligned(w->final_norm, 8))
+    return HB_ERR_BAD_ARG;
   bool any_embed = false;
   for (int32_t r = 0; r < d->n_segs; ++r) any_embed |= (d->segs[r].kind == HB_KIND_EMBED_CHUNK);
   if (any_embed && (!pool || !pool->arena)) return HB_ERR_BAD_ARG;
@@ -544,7 +576,8 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   memcpy(tok, d->token_ids, static_cast<size_t>(T) * 4);
   memcpy(segs, d->segs, static_cast<size_t>(R) * sizeof(hb_seg));
   if (d->n_page_ids) memcpy(pages, d->page_ids, static_cast<size_t>(d->n_page_ids) * 4);
-  std::vector<PoolItem> pitems;
+  std::vector<PoolItem>& pitems = ex->pitems;
+  pitems.clear();
   int32_t part_at = 0;
   for (int32_t r = 0; r < R; ++r) {
     const hb_seg& sg = d->segs[r];
@@ -585,7 +618,10 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   if (static_cast<int32_t>(pitems.size()) > ex->lay.max_pool_items) return HB_ERR_TOO_LARGE;
   // attention work list: chunk items (64 query rows x all visible keys) and decode items (one
   // split of ATT_SPLIT_KEYS keys); sorted by cost, largest first, so the tail of the launch is short
-  std::vector<AttnItem> aitems, titems;
+  std::vector<AttnItem>& aitems = ex->aitems;
+  std::vector<AttnItem>& titems = ex->titems;
+  aitems.clear();
+  titems.clear();
   {
     const int G = cfg.n_heads / cfg.n_kv_heads;
     int32_t rec_at = 0;
@@ -625,23 +661,31 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
         }
       }
     }
-    auto cost = [](const AttnItem& a) {
-      return static_cast<int64_t>(a.key1 - a.key0) * (a.mode ? 16 : a.n_rows);
-    };
-    std::stable_sort(aitems.begin(), aitems.end(),
-                     [&](const AttnItem& a, const AttnItem& b) { return cost(a) > cost(b); });
-    std::stable_sort(titems.begin(), titems.end(),
-                     [&](const AttnItem& a, const AttnItem& b) { return cost(a) > cost(b); });
     if (static_cast<int32_t>(aitems.size() + titems.size()) > ex->lay.max_attn_items) return HB_ERR_TOO_LARGE;
     if (static_cast<size_t>(rec_at) * G * (cfg.head_dim + 2) > c->attn_part_floats) return HB_ERR_TOO_LARGE;
   }
+  // Both lists go to the device sorted by cost, largest first (equal costs in list order).  The sort
+  // runs over (cost, index) keys in a vector the context owns (std::sort works in place), and the
+  // items are copied into the staging buffer in that order.
+  auto sorted_into = [&](const std::vector<AttnItem>& items, uint8_t* dst) {
+    std::vector<uint64_t>& keys = ex->sort_keys;
+    keys.clear();
+    for (size_t i = 0; i < items.size(); ++i) {
+      const AttnItem& a = items[i];
+      const uint64_t cost = static_cast<uint64_t>(a.key1 - a.key0) * static_cast<uint64_t>(a.mode ? 16 : a.n_rows);
+      keys.push_back(((0xffffffffull - std::min<uint64_t>(cost, 0xffffffffull)) << 32) | static_cast<uint64_t>(i));
+    }
+    std::sort(keys.begin(), keys.end());
+    AttnItem* out = reinterpret_cast<AttnItem*>(dst);
+    for (size_t i = 0; i < keys.size(); ++i) out[i] = items[static_cast<size_t>(keys[i] & 0xffffffffull)];
+  };
   const size_t o_aitems = place(aitems.size() * sizeof(AttnItem));
   const size_t o_titems = place(titems.size() * sizeof(AttnItem));
   const size_t o_pitems = place(pitems.size() * sizeof(PoolItem));
   if (off > c->desc_cap) return HB_ERR_TOO_LARGE;
   if (!pitems.empty()) memcpy(st.host + o_pitems, pitems.data(), pitems.size() * sizeof(PoolItem));
-  if (!aitems.empty()) memcpy(st.host + o_aitems, aitems.data(), aitems.size() * sizeof(AttnItem));
-  if (!titems.empty()) memcpy(st.host + o_titems, titems.data(), titems.size() * sizeof(AttnItem));
+  sorted_into(aitems, st.host + o_aitems);
+  sorted_into(titems, st.host + o_titems);
   if (cudaMemcpyAsync(c->desc_dev, st.host, off, cudaMemcpyHostToDevice, s) != cudaSuccess) return HB_ERR_CUDA;
   if (cudaEventRecord(st.ev, s) != cudaSuccess) return HB_ERR_CUDA;
   st.pending = true;
@@ -716,6 +760,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   for (int l = 0; l < cfg.n_layers; ++l) {
     const hb_layer_weights& lw = w->layers[l];
     if (!lw.attn_norm || !lw.wqkv || !lw.wo || !lw.ffn_norm || !lw.w_gate_up || !lw.w_down) return HB_ERR_BAD_ARG;
+    if (misaligned(lw.attn_norm, 8) || misaligned(lw.ffn_norm, 8)) return HB_ERR_BAD_ARG;
     hb_ctx::WMaps& wm = c->wmaps[l];
     if (wm.key[0] != lw.wqkv || wm.key[1] != lw.wo || wm.key[2] != lw.w_gate_up || wm.key[3] != lw.w_down) {
       wm.bn_qkv = hb_gemm_pick_bn(c->max_tokens, n_qkv, c->num_sms);
@@ -724,10 +769,10 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
       wm.bn_down = wm.bn_o;
       wm.ks_o = hb_gemm_pick_ksplit(c->max_tokens, cfg.d_model, n_q, wm.bn_o, c->num_sms);
       wm.ks_down = hb_gemm_pick_ksplit(c->max_tokens, cfg.d_model, cfg.d_ffn, wm.bn_down, c->num_sms);
-      if ((rc = hb_tmap_2d_bf16(&wm.qkv, lw.wqkv, n_qkv, cfg.d_model, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
-      if ((rc = hb_tmap_2d_bf16(&wm.o, lw.wo, cfg.d_model, n_q, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
-      if ((rc = hb_tmap_2d_bf16(&wm.gu, lw.w_gate_up, 2ull * cfg.d_ffn, cfg.d_model, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
-      if ((rc = hb_tmap_2d_bf16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_f16(&wm.qkv, lw.wqkv, n_qkv, cfg.d_model, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_f16(&wm.o, lw.wo, cfg.d_model, n_q, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_f16(&wm.gu, lw.w_gate_up, 2ull * cfg.d_ffn, cfg.d_model, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_f16(&wm.down, lw.w_down, cfg.d_model, cfg.d_ffn, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
       wm.key[0] = lw.wqkv; wm.key[1] = lw.wo; wm.key[2] = lw.w_gate_up; wm.key[3] = lw.w_down;
     }
     // adapters: tensor maps of this layer's packed factors (cached by pointer)
@@ -739,14 +784,14 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
         if (!k) return HB_ERR_BAD_ARG;
       lm = &c->lmaps[l];
       if (lm->rank != lora->rank || memcmp(lm->key, keys, sizeof(keys)) != 0) {
-        if ((rc = hb_tmap_2d_bf16(&lm->a_qkv, ll.a_qkv, r3, cfg.d_model, r3 > 128 ? 256 : 128)) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->b_qkv, ll.b_qkv, n_qkv, r3, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->a_o, ll.a_o, r1, n_q, 128)) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->b_o, ll.b_o, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->a_gu, ll.a_gu, r2, cfg.d_model, r2 > 128 ? 256 : 128)) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->b_gu, ll.b_gu, 2ull * cfg.d_ffn, r2, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->a_d, ll.a_d, r1, cfg.d_ffn, 128)) != HB_OK) return rc;
-        if ((rc = hb_tmap_2d_bf16(&lm->b_d, ll.b_d, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->a_qkv, ll.a_qkv, r3, cfg.d_model, r3 > 128 ? 256 : 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->b_qkv, ll.b_qkv, n_qkv, r3, hb_gemm_box_rows(wm.bn_qkv))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->a_o, ll.a_o, r1, n_q, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->b_o, ll.b_o, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_o))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->a_gu, ll.a_gu, r2, cfg.d_model, r2 > 128 ? 256 : 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->b_gu, ll.b_gu, 2ull * cfg.d_ffn, r2, hb_gemm_box_rows(wm.bn_gu))) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->a_d, ll.a_d, r1, cfg.d_ffn, 128)) != HB_OK) return rc;
+        if ((rc = hb_tmap_2d_f16(&lm->b_d, ll.b_d, cfg.d_model, r1, hb_gemm_box_rows(wm.bn_down))) != HB_OK) return rc;
         memcpy(lm->key, keys, sizeof(keys));
         lm->rank = lora->rank;
       }
@@ -834,7 +879,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   }
   if (dd.n_logit > 0) {
     if (c->lm_key != w->lm_head) {
-      if ((rc = hb_tmap_2d_bf16(&c->tm_lm, w->lm_head, cfg.vocab, cfg.d_model, 128)) != HB_OK) return rc;
+      if ((rc = hb_tmap_2d_f16(&c->tm_lm, w->lm_head, cfg.vocab, cfg.d_model, 128)) != HB_OK) return rc;
       c->lm_key = w->lm_head;
     }
     GemmArgs ga = {};
@@ -874,6 +919,10 @@ int hb_pool_chunk(hb_ctx* c, const float* x, const void* gain, int32_t n_rows, i
   if (!c || !x || !gain || !slot_sum || !slot_meta || n_rows < 1) return HB_ERR_BAD_ARG;
   if (mode < HB_POOL_MEAN || mode > HB_POOL_WMEAN) return HB_ERR_BAD_ARG;
   if (is_final && !out_emb) return HB_ERR_BAD_ARG;
+  // 16-byte vector accesses to the rows, the slot and the output; 8-byte ones to the gain
+  if (misaligned(x, 16) || misaligned(slot_sum, 16) || misaligned(out_emb, 16) || misaligned(gain, 8) ||
+      misaligned(slot_meta, 4))
+    return HB_ERR_BAD_ARG;
   if (n_rows > c->max_tokens) return HB_ERR_TOO_LARGE;
   return hb_launch_pool_chunk(c, x, gain, n_rows, mode, first_chunk != 0, is_final != 0, slot_sum, slot_meta,
                               out_emb, static_cast<cudaStream_t>(stream));
@@ -946,13 +995,13 @@ int hb_gemm_pair(hb_ctx* c, const void* A, const void* B, const void* A2, const 
   if (K2 < 0 || (K2 & 63) || ((K2 > 0) != (A2 != nullptr && B2 != nullptr))) return HB_ERR_BAD_ARG;
   const int bn = hb_gemm_pick_bn(M, N, c->num_sms);
   CUtensorMap ta, tb, ta2, tb2;
-  int rc = hb_tmap_2d_bf16(&ta, A, M, K, 128);
+  int rc = hb_tmap_2d_f16(&ta, A, M, K, 128);
   if (rc != HB_OK) return rc;
-  rc = hb_tmap_2d_bf16(&tb, B, N, K, hb_gemm_box_rows(bn));
+  rc = hb_tmap_2d_f16(&tb, B, N, K, hb_gemm_box_rows(bn));
   if (rc != HB_OK) return rc;
   if (K2 > 0) {
-    if ((rc = hb_tmap_2d_bf16(&ta2, A2, M, K2, 128)) != HB_OK) return rc;
-    if ((rc = hb_tmap_2d_bf16(&tb2, B2, N, K2, hb_gemm_box_rows(bn))) != HB_OK) return rc;
+    if ((rc = hb_tmap_2d_f16(&ta2, A2, M, K2, 128)) != HB_OK) return rc;
+    if ((rc = hb_tmap_2d_f16(&tb2, B2, N, K2, hb_gemm_box_rows(bn))) != HB_OK) return rc;
   }
   GemmArgs ga = {};
   ga.C = C; ga.M = M; ga.N = N; ga.K = K; ga.b_kshift = 0; ga.status = c->status;

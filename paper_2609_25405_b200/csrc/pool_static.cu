@@ -66,6 +66,11 @@ extern "C" int hb_pool_chunk_noalloc(const float* x, const void* gain, int32_t n
   if (mode < HB_POOL_MEAN || mode > HB_POOL_WMEAN) return HB_ERR_BAD_ARG;
   if (is_final && !out_emb) return HB_ERR_BAD_ARG;
   if (!(rms_eps >= 0.0f)) return HB_ERR_BAD_ARG;
+  // The kernel moves rows, slot and output as 16-byte vectors and the gain as 8-byte ones.  A caller
+  // that carves these out of its own arena (the caller this entry is for) can easily hand over a
+  // view that starts mid-vector: refuse it here instead of faulting on the device.
+  auto off = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
+  if (off(x, 16) || off(slot_sum, 16) || off(out_emb, 16) || off(gain, 8) || off(slot_meta, 4)) return HB_ERR_BAD_ARG;
   // beyond the fixed scratch: refuse, never truncate
   if (n_rows > MAX_ROWS || d_model > MAX_D) return HB_ERR_TOO_LARGE;
   float* scratch = nullptr;

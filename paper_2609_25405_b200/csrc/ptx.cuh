@@ -239,10 +239,16 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-// Saturating at the largest finite half.
-__device__ __forceinline__ uint32_t pack_half2_sat(float lo, float hi) {
-  return pack_half2(fminf(fmaxf(lo, -65504.0f), 65504.0f), fminf(fmaxf(hi, -65504.0f), 65504.0f));
+// Finite values saturate at the largest finite half instead of becoming infinite; NaN stays NaN
+// (fminf / fmaxf alone would turn it into a finite number and hide it).
+__device__ __forceinline__ float sat_half_range(float v) {
+  return (v != v) ? v : fminf(fmaxf(v, -65504.0f), 65504.0f);
 }
+__device__ __forceinline__ uint32_t pack_half2_sat(float lo, float hi) {
+  return pack_half2(sat_half_range(lo), sat_half_range(hi));
+}
+// True when v does not fit a finite half: NaN, infinite, or beyond +-65504.
+__device__ __forceinline__ bool outside_half_range(float v) { return !(fabsf(v) <= 65504.0f); }
 // 2^x on the special-function unit (-inf -> 0).
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;

@@ -45,12 +45,18 @@ SPECS = {
 }
 
 
-def sweep_spec(frac, seed=1004):
+def sweep_spec(frac, seed=1004, cap_decode=0):
     """Embedding-fraction sweep on the 7B shape: 4096-token budget, decode contexts 2048,
-    embedding lengths U[128,2048], mean pooling, chunk cap 512."""
+    embedding lengths U[128,2048], mean pooling, chunk cap 512.  cap_decode > 0 is the
+    capacity-true variant: the decode rows are capped at what one GPU can hold unaliased (268 MB of
+    K/V per row), the embedding rows stay, so the step is smaller than 4096 rows."""
     n_emb = int(round(4096 * frac))
-    return MixSpec(f"cfg4-7b-f{frac:g}", "7b", 4096 - n_emb, 2048, 2048, 4096, 512, "uniform", 128, 128, 2048,
-                   B.POOL_MEAN, seed)
+    n_dec = 4096 - n_emb
+    name = f"cfg4-7b-f{frac:g}"
+    if cap_decode and n_dec > cap_decode:
+        n_dec = cap_decode
+        name += f"-cap{cap_decode}"
+    return MixSpec(name, "7b", n_dec, 2048, 2048, n_dec + n_emb, 512, "uniform", 128, 128, 2048, B.POOL_MEAN, seed)
 
 
 class _Req:
