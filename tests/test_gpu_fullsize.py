@@ -1,8 +1,12 @@
 """Full-size parity: the 1B-class and 7B-class shapes at their full depth and width, in the launch
 configurations the benchmark times (full token budget per step, decode rows over long synthetic
-contexts plus embedding chunks; for the 7B shape also one point of the embedding-fraction sweep with
-2048 decode rows), checked on sampled requests the CPU oracle can recompute one by one.  Legitimate because a request's outputs do not depend on its batch mates (checked
-bit for bit on the tiny shape, and here on one request run solo and inside the batch).
+contexts plus embedding chunks; for the 7B shape also the middle point of the embedding-fraction
+sweep with 2048 decode rows), checked on sampled requests the CPU oracle can recompute one by one.
+Legitimate because a request's outputs do not depend on its batch mates (checked bit for bit on the
+tiny shape, and here on every sampled request, run again alone and compared with its in-batch
+result).  The other four mixes of the sweep (embedding fractions 0, 0.25, 0.75, 0.95: 4096, 3072,
+1024 and 205 decode rows) run at the 7B width with two layers, and two more cases compare EVERY
+request of full-budget steps with the oracle at the 7B and 1B widths with two layers.
 
 Sampled per shape: two generation requests (prompt prefilled in chunks through the library
 itself, then teacher-forced decode steps) and two embedding requests (one single-chunk, one
@@ -39,22 +43,35 @@ CASES = {
                          gen=(2048,), emb=(), emb_mean=(1500,), seed=1004, n_steps=2, alias=64,
                          fill_len=(128, 2048), fill_mean=True),
 }
+# The other mixes of the sweep at the 7B width with two layers (same kernels, tile shapes and launch
+# configurations per layer as the full depth; the oracle and the weights are 16 times cheaper).  The
+# sampled generation request is prefilled through the library in steps of its own first (at f = 0 a
+# full step has no room for a chunk), then every step is a full 4096-row step of the mix: at f = 0
+# 4096 decode rows and no chunk row at all.
+for _f, _nd in ((0, 4096), (0.25, 3072), (0.75, 1024), (0.95, 205)):
+    CASES[f"cfg4-7b-f{_f:g}-L2"] = dict(shape="7b", layers=2, n_decode=_nd, ctx=(2048, 2048), budget=4096, chunk=512,
+                                        gen=(2048,), emb=(), emb_mean=(1500,) if _f else (), seed=1004 + int(100 * _f),
+                                        n_steps=3, alias=64, fill_len=(128, 2048), fill_mean=True, prefill_first=True)
 
 
 def _threads():
     return max(4, min(32, os.cpu_count() or 8))
 
 
-@pytest.mark.parametrize("name", ["cfg2-1b", "cfg3-7b", "cfg4-7b-f0.5"])
+@pytest.mark.parametrize("name", ["cfg2-1b", "cfg3-7b", "cfg4-7b-f0.5", "cfg4-7b-f0-L2", "cfg4-7b-f0.25-L2",
+                                  "cfg4-7b-f0.75-L2", "cfg4-7b-f0.95-L2"])
 def test_fullsize_sampled_requests_match_oracle(name):
+    from conftest import cached_weights
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
     c = CASES[name]
     shape = synth.SHAPES[c["shape"]]
+    if c.get("layers"):
+        shape = shape.with_layers(c["layers"])
     P = shape.page_size
     rng = np.random.default_rng(c["seed"])
-    W = synth.Weights(shape, 0, cache="bits").prefetch(_threads())
-    dw = B.DeviceWeights.from_synth(W)
+    # the full 7B model (14.5 GB of bit patterns on the host) is not kept between tests; the others are
+    W, dw = cached_weights(shape, keep=not (c["shape"] == "7b" and not c.get("layers")))
     n_steps = c["n_steps"]       # logits rows compared per generation request (prefill row + decode rows)
     max_pos = c["ctx"][1] + n_steps + 8
     n_dec = c["n_decode"]
@@ -115,6 +132,13 @@ def test_fullsize_sampled_requests_match_oracle(name):
     got_emb = {}
     chunk = c["chunk"]
     inflight_fill = []
+    if c.get("prefill_first"):
+        for g in gens:
+            while not g.in_decode:
+                _, lrows, _ = eng.step([(g, min(chunk, g.remaining()))])
+                torch.cuda.synchronize()
+                if g in lrows:
+                    got_lg[g].append(eng.out_logits[lrows[g]].cpu().numpy().astype(np.float64))
     for step in range(n_steps + 3 + max(c["gen"]) // chunk):
         work = []
         rows = 0
@@ -169,14 +193,29 @@ def test_fullsize_sampled_requests_match_oracle(name):
             break
     assert eng.ctx.status_poll() == 0
 
-    # ---- one sampled embedding request again, alone in its steps (same chunking): bit for bit the
-    # result it had inside the full batches
-    solo = Request("embed", list(embs[0].tokens), embs[0].pool_mode)
-    while solo.remaining() > 0:
-        _, _, er = eng.step([(solo, min(chunk, solo.remaining()))])
-    torch.cuda.synchronize()
-    assert np.array_equal(eng.out_emb[er[solo]].cpu().numpy().astype(np.float64), got_emb[embs[0]])
-    eng.release(solo)
+    # ---- every sampled request again, alone in its steps (same chunking, the same fed tokens): bit
+    # for bit the results it had inside the full batches
+    for e in embs:
+        solo = Request("embed", list(e.tokens), e.pool_mode)
+        while solo.remaining() > 0:
+            _, _, er = eng.step([(solo, min(chunk, solo.remaining()))])
+        torch.cuda.synchronize()
+        assert np.array_equal(eng.out_emb[er[solo]].cpu().numpy().astype(np.float64), got_emb[e])
+        eng.release(solo)
+    for g in gens:
+        n0 = g.n_prompt
+        solo = Request("gen", list(g.tokens[:n0]))
+        rows = []
+        while len(rows) < n_steps:
+            if solo.in_decode:
+                solo.tokens.append(g.tokens[n0 + len(rows) - 1])
+            _, lr, _ = eng.step([(solo, 1 if solo.in_decode else min(chunk, solo.remaining()))])
+            torch.cuda.synchronize()
+            if solo in lr:
+                rows.append(eng.out_logits[lr[solo]].cpu().numpy().astype(np.float64))
+        for a, b in zip(rows, got_lg[g]):
+            assert np.array_equal(a, b)
+        eng.release(solo)
     assert eng.ctx.status_poll() == 0
 
     # ---- compare ----
@@ -209,4 +248,120 @@ def test_fullsize_sampled_requests_match_oracle(name):
         if r.kind == "embed":
             meta = eng.pool.meta()[r.slot].cpu().numpy()
             assert list(meta.astype(np.int64)) == [cnt, chunks, r.pool_mode, 1]
+    eng.close()
+
+
+WHOLE = {
+    # width, decode rows, their contexts, token budget, chunk, embedding lengths lognormal(median, lo, hi)
+    "7b": dict(n_decode=16, ctx=(512, 4096), budget=4096, chunk=512, emb=(512, 32, 4096), seed=3003),
+    "1b": dict(n_decode=16, ctx=(128, 1024), budget=2048, chunk=256, emb=(256, 16, 2048), seed=3002),
+}
+
+
+@pytest.mark.parametrize("width", ["7b", "1b"])
+def test_whole_batch_two_layers_every_request_matches_oracle(width):
+    """The 7B-class and 1B-class widths with two layers: EVERY request of full-budget steps against
+    the fp32 oracle, not a sample.  16 generation requests (their contexts written by the library:
+    prompts prefilled in chunks, FCFS under the budget) decode one teacher-forced row per step next
+    to a stream of embedding requests (lengths lognormal as in the configurations, chunked, every
+    third one mean-pooled, the others last-token) admitted FCFS until the budget is full; after three
+    full-budget steps nothing new is admitted and the steps continue until every embedding request
+    in flight has finished.  Compared: every logits row of every decode step of every generation
+    request, and every embedding."""
+    from conftest import cached_weights
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Engine, Request
+    c = WHOLE[width]
+    shape = synth.SHAPES[width].with_layers(2)
+    W, dw = cached_weights(shape)
+    P, budget, chunk = shape.page_size, c["budget"], c["chunk"]
+    rng = np.random.default_rng(c["seed"])
+    n_full, max_drain = 3, c["emb"][2] // chunk + 1
+    max_pos = max(c["ctx"][1] + n_full + max_drain + 2, c["emb"][2] + 2)
+    n_pages = c["n_decode"] * (max_pos // P + 2) + 6 * budget // P + 16 * (c["emb"][2] // P + 2)
+    eng = Engine(shape, dw, n_pages=n_pages, n_slots=128, max_tokens=budget, max_segs=c["n_decode"] + budget // 16 + 8,
+                 max_pos=max_pos, kv_fill=KV_SENTINEL)
+    gens = [Request("gen", synth.token_ids(rng, int(n), shape.V))
+            for n in rng.integers(c["ctx"][0], c["ctx"][1] + 1, size=c["n_decode"])]
+    got_lg = {g: [] for g in gens}
+    got_emb, all_embs = {}, []
+
+    def run(work):
+        _, lrows, erows = eng.step(work)
+        torch.cuda.synchronize()
+        for r, row in lrows.items():
+            got_lg[r].append(eng.out_logits[row].cpu().numpy().astype(np.float64))
+        for r, row in erows.items():
+            got_emb[r] = eng.out_emb[row].cpu().numpy().astype(np.float64)
+            eng.release(r)
+
+    # contexts: prefill the prompts through the library, FCFS, full steps
+    while any(not g.in_decode for g in gens):
+        work, rows = [], 0
+        for g in gens:
+            if not g.in_decode and rows < budget:
+                q = min(chunk, g.remaining(), budget - rows)
+                work.append((g, q)); rows += q
+        run(work)
+    # mixed steps: 16 decode rows + embedding chunks up to the budget; then drain
+    inflight, step, n_mixed_rows = [], 0, []
+    while step < n_full or inflight:
+        assert step < n_full + max_drain + 1
+        work, rows = [], 0
+        for g in gens:
+            g.tokens.append(int(rng.integers(0, shape.V)))       # the token both sides are fed
+            work.append((g, 1)); rows += 1
+        nxt = []
+        for e in inflight:
+            q = min(chunk, e.remaining(), budget - rows)
+            if q > 0:
+                work.append((e, q)); rows += q
+            if e.remaining() - q > 0:
+                nxt.append(e)
+        while step < n_full and rows < budget:
+            n = int(synth.lognormal_lengths(rng, 1, *c["emb"])[0])
+            e = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_MEAN if len(all_embs) % 3 == 2 else B.POOL_LAST)
+            all_embs.append(e)
+            q = min(chunk, n, budget - rows)
+            work.append((e, q)); rows += q
+            if q < n:
+                nxt.append(e)
+        inflight = nxt
+        if step < n_full:
+            assert rows == budget
+        n_mixed_rows.append(rows)
+        run(work)
+        step += 1
+    assert eng.ctx.status_poll() == 0
+    assert len(got_emb) == len(all_embs) and len(all_embs) >= 8
+    # ---- oracle: one whole-sequence pass per request ----
+    head = {B.POOL_LAST: "last", B.POOL_MEAN: "mean"}
+    worst_l = worst_e = 0.0
+    worst_cos = 1.0
+    n_rows = n_agree = 0
+    for g in gens:
+        n0, k = g.n_prompt, len(got_lg[g])
+        assert k == step + 1                                      # the prefill row, then one row per mixed step
+        _, ref = T.forward(shape, W, g.tokens, logit_rows=list(range(n0 - 1, n0 - 1 + k)), dtype=np.float32)
+        for s in range(k):
+            r = ref[s].astype(np.float64)
+            err = float(np.max(np.abs(got_lg[g][s] - r)))
+            worst_l = max(worst_l, err)
+            assert err <= LOGIT_ABS, (width, n0, s, err)
+            same = int(np.argmax(got_lg[g][s]) == np.argmax(r))
+            n_rows += 1
+            n_agree += same
+            if not same:
+                top = np.sort(r)[-2:]
+                print(f"  differing argmax: request of {n0} prompt tokens, row {s}: oracle gap {top[1] - top[0]:.3e}, error {err:.3e}")
+    for e in all_embs:
+        ref = T.embed(shape, W, e.tokens, head[e.pool_mode], dtype=np.float32).astype(np.float64)
+        got = got_emb[e]
+        cos = float(got @ ref / (np.linalg.norm(got) * np.linalg.norm(ref)))
+        worst_cos, worst_e = min(worst_cos, cos), max(worst_e, float(np.max(np.abs(got - ref))))
+        assert cos >= EMB_COS and np.max(np.abs(got - ref)) <= EMB_ABS, (width, len(e.tokens), cos)
+    print(f"\n[{width}, 2 layers] steps of {n_mixed_rows} rows; {n_rows} logits rows: worst max-abs error {worst_l:.3e}, "
+          f"argmax agreement {n_agree}/{n_rows}; {len(all_embs)} embeddings: worst cosine {worst_cos:.6f}, "
+          f"worst max-abs error {worst_e:.3e}")
+    assert n_agree / n_rows >= 0.995, (n_agree, n_rows)
     eng.close()

@@ -70,3 +70,76 @@ def test_phase_workload_tiny():
     assert eng.ctx.status_poll() == 0
     assert n_embed[0] < n_embed[1] < n_embed[2]
     eng.close()
+
+
+def test_trace_prefix_on_the_1b_shape_every_output_matches_oracle():
+    """Configuration 5 on its own shape: the first three sessions of the seed-1005 trace (3-5 rounds
+    each of an embedding request and a generation request with a 512-2048-token prompt and 32-128
+    greedy decode steps) replayed on the full 1B-class model through the scheduler and the engine.
+    EVERY embedding and EVERY logits row of those sessions is compared with the fp32 oracle: the
+    oracle runs one whole-sequence pass per request over the prompt plus the tokens the device chose
+    (teacher-forced on the device's own greedy tokens, so one differing argmax does not spoil the
+    rows after it).  Bookkeeping over a whole trace is checked on the tiny shape above."""
+    from conftest import cached_weights
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200 import trace
+    from paper_2609_25405_b200.engine import Engine
+    shape = synth.SHAPES["1b"]
+    W, dw = cached_weights(shape)
+    sessions = trace.make_trace(shape.V, seed=1005, n_sessions=256)[:3]
+    budget, chunk = 4096, 256
+    max_pos = 2048 + 128 + 8
+    P = shape.page_size
+    n_pages = 3 * ((max_pos + P - 1) // P) + 64
+    eng = Engine(shape, dw, n_pages=n_pages, n_slots=8, max_tokens=budget, max_segs=3 + budget // 16 + 8, max_pos=max_pos)
+    got_emb, got_tok = {}, {}
+
+    def on_emb(si, ri, vec):
+        got_emb[(si, ri)] = vec.cpu().numpy().astype(np.float64)
+
+    def on_tok(si, ri, step, token, row):
+        got_tok[(si, ri, step)] = (token, row.cpu().numpy())          # fp32 rows: ~0.5 MB each
+
+    out = trace.replay(sessions, eng, budget, chunk, pool_mode=B.POOL_LAST, on_embedding=on_emb, on_token=on_tok)
+    assert eng.ctx.status_poll() == 0
+    assert out["sessions_done"] == 3 and out["rows"] == trace.trace_tokens(sessions)
+    assert out["free_pages"] == n_pages
+    n_rows = n_agree = n_embs = 0
+    worst_l = worst_e = 0.0
+    worst_cos = 1.0
+    flips = []
+    for si, s in enumerate(sessions):
+        for ri, r in enumerate(s.requests):
+            if r.kind == "embed":
+                ref = T.embed(shape, W, r.tokens, "last", dtype=np.float32).astype(np.float64)
+                got = got_emb[(si, ri)]
+                cos = float(got @ ref / (np.linalg.norm(got) * np.linalg.norm(ref)))
+                worst_cos, worst_e = min(worst_cos, cos), max(worst_e, float(np.max(np.abs(got - ref))))
+                assert cos >= 0.9995 and np.max(np.abs(got - ref)) <= 2e-2, (si, ri, len(r.tokens), cos)
+                n_embs += 1
+                continue
+            k = r.decode_steps + 1                       # the prompt's last row, then one row per decode step
+            toks = [got_tok[(si, ri, st)][0] for st in range(k)]
+            seq = [int(t) for t in r.tokens] + toks[:-1]
+            n0 = len(r.tokens)
+            _, ref = T.forward(shape, W, seq, logit_rows=list(range(n0 - 1, n0 - 1 + k)), dtype=np.float32)
+            for st in range(k):
+                token, row = got_tok[(si, ri, st)]
+                err = float(np.max(np.abs(row.astype(np.float64) - ref[st])))
+                worst_l = max(worst_l, err)
+                assert err <= 5e-2, (si, ri, st, err)
+                assert token == int(np.argmax(row))          # hb_argmax = the argmax of the device's own logits
+                n_rows += 1
+                if token == int(np.argmax(ref[st])):
+                    n_agree += 1
+                else:
+                    top = np.sort(ref[st])[-2:]
+                    flips.append((si, ri, st, float(top[1] - top[0]), err))
+    print(f"\ntrace prefix, 1B shape: {n_embs} embeddings (worst cosine {worst_cos:.6f}, worst max-abs error {worst_e:.3e}); "
+          f"{n_rows} logits rows (worst max-abs error {worst_l:.3e}), argmax agreement {n_agree}/{n_rows} = "
+          f"{n_agree / max(n_rows, 1):.4f}")
+    for si, ri, st, gap, err in flips:
+        print(f"  differing argmax: session {si} request {ri} step {st}: oracle top-1/top-2 gap {gap:.3e}, "
+              f"logits max-abs error {err:.3e}")
+    assert n_agree / n_rows >= 0.995, (n_agree, n_rows)
+    eng.close()
