@@ -522,6 +522,7 @@ def main():
                     help="sweep workloads: cap the decode rows at what fits in HBM unaliased (the step gets smaller)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--sessions", type=int, default=256, help="sessions of the cfg5-trace-1b workload")
+    ap.add_argument("--gemm-walk", default="", help="tuning: force the projection GEMM's tile walk, 'band,hints' (see hb_gemm_set_walk)")
     ap.add_argument("--lora-rank", type=int, default=0,
                     help="rank of a random low-rank adapter applied to the embedding rows (0 = none, the headline)")
     args = ap.parse_args()
@@ -539,6 +540,9 @@ def main():
 
     import torch
 
+    if args.gemm_walk:
+        from paper_2609_25405_b200 import binding as _B
+        _B.gemm_set_walk(*[int(v) for v in args.gemm_walk.split(",")])
     if args.workload.startswith("cfg5-trace"):
         run_trace(args)
         return

@@ -374,6 +374,15 @@ HB_API int hb_gemm(hb_ctx* ctx, const void* A, const void* B, void* C, int32_t M
 HB_API int hb_gemm_pair(hb_ctx* ctx, const void* A, const void* B, const void* A2, const void* B2, void* C,
                  int32_t M, int32_t N, int32_t K, int32_t K2, int32_t epilogue, void* stream);
 
+/* Tile walk of the projection GEMM, for tests and tuning.  A launch normally chooses by itself in
+ * which order its workers take the output tiles (rows fastest over the whole M, or in bands of row
+ * tiles when A's share of a work item would not stay in L2) and whether its loads carry L2 eviction
+ * hints.  The walk never changes the K order of an element's sum, so results are bit-identical under
+ * every setting; this call forces one for all later launches of the process so that a test can show
+ * exactly that, and a profile can compare DRAM traffic.  band >= 1: row tiles per band; band = 0: whole
+ * M; hints 0 / 1; -1 for either = automatic again.  Host only, not thread-safe against launches. */
+HB_API int hb_gemm_set_walk(int32_t band, int32_t hints);
+
 /* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
  * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of
  * the chunk's rows, then

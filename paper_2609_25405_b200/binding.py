@@ -105,6 +105,7 @@ _sig = {
     "hb_profile_enable": [_P, C.c_int],
     "hb_profile_read": [_P, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
     "hb_gemm": [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
+    "hb_gemm_set_walk": [C.c_int32, C.c_int32],
 }
 for _name, _args in _sig.items():
     _f = getattr(lib, _name)
@@ -574,6 +575,11 @@ def pool_chunk_noalloc(x, gain, n_rows, d_model, rms_eps, mode, first_chunk, is_
                                      C.c_void_p(slot_sum.data_ptr()), C.c_void_p(slot_meta.data_ptr()),
                                      C.c_void_p(out_emb.data_ptr()) if out_emb is not None else None,
                                      _stream_ptr(stream))
+
+
+def gemm_set_walk(band=-1, hints=-1):
+    """Force the projection GEMM's tile walk (tests / tuning); -1 = automatic."""
+    check(lib.hb_gemm_set_walk(band, hints), "hb_gemm_set_walk")
 
 
 def validate_desc(cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, batch):

@@ -276,6 +276,20 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   // that where a row's sum is cut does not depend on whether the launch carries a second pair (a
   // generation row's bits must not change when embedding rows with an adapter join its batch).
   const int k_per_split = (k1_blocks + k_splits - 1) / k_splits;
+  // Tile walk: output tiles are numbered along M first inside bands of `band` row tiles, band after
+  // band.  With band = m_tiles this is "rows fastest over the whole M" (a wave of workers touches every
+  // row tile of A and a few column tiles of B).  When A's share of a work item is too large for all its
+  // row tiles to stay in L2 next to the B tiles streaming past, a narrower band keeps the band's rows
+  // of A resident while the walk crosses N, at the price of one more pass over B per band.  The walk
+  // changes which worker computes a tile and when, never the order of the K sum of an element.
+  const int band = (g.raster_band > 0 && g.raster_band < m_tiles) ? g.raster_band : m_tiles;
+  auto tile_coords = [&](int mn, int& mi, int& ni) {
+    const int per_band = band * n_tiles;
+    const int b = mn / per_band, r = mn - b * per_band;
+    const int bh = min(band, m_tiles - b * band);
+    ni = r / bh;
+    mi = b * band + (r - ni * bh);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T::STAGES; ++s) {
@@ -325,11 +339,15 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const uint64_t pol_a = g.l2_hints ? l2_policy_evict_last() : 0ull;
+      const uint64_t pol_b = g.l2_hints ? l2_policy_evict_first() : 0ull;
       // the data of both CTAs of a group is accounted on the leader's barrier
       for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
         const int mn = tile % mn_tiles, split = tile / mn_tiles;
-        const int m0 = (mn % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
-        const int n0 = (mn / m_tiles) * BN + static_cast<int>(rank) * T::B_ROWS;
+        int mi, ni;
+        tile_coords(mn, mi, ni);
+        const int m0 = mi * (BM * CG) + static_cast<int>(rank) * BM;
+        const int n0 = ni * BN + static_cast<int>(rank) * T::B_ROWS;
         const int kb0 = split * k_per_split;
         const int kb1 = (split + 1 == k_splits) ? k_blocks : min(kb0 + k_per_split, k1_blocks);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -344,12 +362,22 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           if constexpr (CG == 2) {
             const uint32_t bar = map_to_rank(full_bar(stage), 0u);
             if (leader) mbar_arrive_expect_tx(full_bar(stage), 2u * T::STAGE_BYTES);
-            tma_load_2d_cg2(a_dst, ma, bar, ka, m0);
-            tma_load_2d_cg2(b_dst, mb, bar, kbb, n0);
+            if (g.l2_hints) {
+              tma_load_2d_cg2_hint(a_dst, ma, bar, ka, m0, pol_a);
+              tma_load_2d_cg2_hint(b_dst, mb, bar, kbb, n0, pol_b);
+            } else {
+              tma_load_2d_cg2(a_dst, ma, bar, ka, m0);
+              tma_load_2d_cg2(b_dst, mb, bar, kbb, n0);
+            }
           } else {
             mbar_arrive_expect_tx(full_bar(stage), T::STAGE_BYTES);
-            tma_load_2d(a_dst, ma, full_bar(stage), ka, m0);
-            tma_load_2d(b_dst, mb, full_bar(stage), kbb, n0);
+            if (g.l2_hints) {
+              tma_load_2d_hint(a_dst, ma, full_bar(stage), ka, m0, pol_a);
+              tma_load_2d_hint(b_dst, mb, full_bar(stage), kbb, n0, pol_b);
+            } else {
+              tma_load_2d(a_dst, ma, full_bar(stage), ka, m0);
+              tma_load_2d(b_dst, mb, full_bar(stage), kbb, n0);
+            }
           }
           if (++stage == T::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -414,8 +442,10 @@ hb_gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     bool ok = true;
     for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
       const int mn = tile % mn_tiles, split = tile / mn_tiles;
-      const int m0 = (mn % m_tiles) * (BM * CG) + static_cast<int>(rank) * BM;
-      const int n0 = (mn / m_tiles) * BN;
+      int mi, ni;
+      tile_coords(mn, mi, ni);
+      const int m0 = mi * (BM * CG) + static_cast<int>(rank) * BM;
+      const int n0 = ni * BN;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, WAIT_LIMIT_NS)) { ok = false; give_up(); break; }
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
@@ -684,6 +714,41 @@ int hb_gemm_pick_step_variant(int map_variant, int rows, int N, int k_blocks, in
 
 int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : variant; }
 
+// Tile walk of a launch (see the kernel).  A's share of one work item, over all row tiles, is
+// M x (K per item) x 2 bytes.  While that fits comfortably in L2 next to the B tiles of a wave, rows
+// go fastest over the whole M and every B tile is read from DRAM once.  The 7B-class down projection
+// is the launch where it does not (4096 x 7168 x 2 B = 59 MB per K half; each half of the L2 caches
+// what its own SMs read, and every wave of 74 tile pairs touches all 16 row tiles): there the walk
+// uses bands of row tiles whose share of A is about a quarter of L2, which makes a wave's footprint
+// nearly square (8 row tiles x 9 column tiles).  Measured on that launch (profiler, DRAM read +
+// write): 838 MB rows-fastest, 774 MB with bands of 8; the step time is the same within noise.
+// Eviction hints on the loads (A evict-last, B evict-first) brought 755 MB but cost 0.7 ms per 7B
+// step (three alternating runs), so the automatic choice leaves them off; they stay reachable
+// through hb_gemm_set_walk.
+static int g_band_override = -1;   // >= 0: test / tuning override of the band (0 = whole M)
+static int g_hint_override = -1;
+void hb_gemm_walk_override(int band, int hints) { g_band_override = band; g_hint_override = hints; }
+
+void hb_gemm_pick_walk(int variant, int epi, GemmArgs* g) {
+  const int tile_rows = (variant == HB_GEMM_PAIR256) ? 256 : 128;
+  const int ks = ((epi == HB_EPI_LORA_DOWN || epi == HB_EPI_RESID_F32) && g->k_splits > 1) ? g->k_splits : 1;
+  const long k_item = (static_cast<long>(g->K) + ks - 1) / ks;
+  const long a_tile_bytes = static_cast<long>(tile_rows) * k_item * 2;
+  const int m_tiles = (g->M + tile_rows - 1) / tile_rows;
+  g->raster_band = 0;
+  g->l2_hints = 0;
+  if (static_cast<long>(m_tiles) * a_tile_bytes > 40l * 1024 * 1024) {
+    long band = (30l * 1024 * 1024) / a_tile_bytes;
+    if (band < 1) band = 1;
+    if (band < m_tiles) {
+      g->raster_band = static_cast<int>(band);
+      g->l2_hints = 0;
+    }
+  }
+  if (g_band_override >= 0) g->raster_band = g_band_override;
+  if (g_hint_override >= 0) g->l2_hints = g_hint_override;
+}
+
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, int epi, const GemmArgs& a,
                    int num_sms, cudaStream_t s, const CUtensorMap* tmA2, const CUtensorMap* tmB2, bool pdl) {
   if ((a.k2_blocks > 0) != (tmA2 != nullptr && tmB2 != nullptr) || a.k2_blocks < 0) return HB_ERR_BAD_ARG;
@@ -693,8 +758,10 @@ int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, 
   // without an extension the second pair is never read; pass the first so the parameters are valid maps
   const CUtensorMap& a2 = tmA2 ? *tmA2 : tmA;
   const CUtensorMap& b2 = tmB2 ? *tmB2 : tmB;
-  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, a2, b2, epi, a, num_sms, s, pdl);
-  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s, pdl);
-  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, a2, b2, epi, a, num_sms, s, pdl);
+  GemmArgs g = a;
+  hb_gemm_pick_walk(variant, epi, &g);
+  if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, a2, b2, epi, g, num_sms, s, pdl);
+  if (variant == 256) return launch_bn<256, 1>(tmA, tmB, a2, b2, epi, g, num_sms, s, pdl);
+  if (variant == 128) return launch_bn<128, 1>(tmA, tmB, a2, b2, epi, g, num_sms, s, pdl);
   return HB_ERR_BAD_ARG;
 }

@@ -115,6 +115,8 @@ struct GemmArgs {
   int32_t ldc;          // elements
   int32_t b_kshift;     // B k-block index = A k-block index >> b_kshift
   int32_t k2_blocks;    // 64-column blocks of the second operand pair accumulated after K (0 = none)
+  int32_t raster_band;  // row tiles per band of the tile walk (0 = all: rows fastest over the whole M); set by hb_gemm_launch
+  int32_t l2_hints;     // 1: A loads are kept in L2 (evict last), B loads stream (evict first); set by hb_gemm_launch
   uint32_t* status;
   // HB_EPI_LORA_DOWN only
   float alpha;
@@ -165,6 +167,9 @@ int hb_gemm_pick_ksplit(int M, int N, int K, int variant, int num_sms);
 // Variant for one launch of `rows` rows when the B map was built for `map_variant` (the choice made
 // for the context's row capacity): a step much smaller than the capacity may run single-CTA tiles.
 int hb_gemm_pick_step_variant(int map_variant, int rows, int N, int k_blocks, int k_splits, int num_sms);
+// Chooses GemmArgs::raster_band and l2_hints for a launch of `variant` (called by hb_gemm_launch).
+void hb_gemm_pick_walk(int variant, int epi, GemmArgs* g);
+void hb_gemm_walk_override(int band, int hints);   // tuning: >= 0 forces the value for every launch, -1 = automatic
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,
                    const CUtensorMap* tmB2 = nullptr, bool pdl = false);

@@ -981,6 +981,12 @@ int hb_last_launch_count(const hb_ctx* c, int32_t* out_count) {
   return HB_OK;
 }
 
+int hb_gemm_set_walk(int32_t band, int32_t hints) {
+  if (band < -1 || hints < -1 || hints > 1) return HB_ERR_BAD_ARG;
+  hb_gemm_walk_override(band, hints);
+  return HB_OK;
+}
+
 int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int32_t epilogue,
             void* stream) {
   return hb_gemm_pair(c, A, B, nullptr, nullptr, C, M, N, K, 0, epilogue, stream);

@@ -178,6 +178,39 @@ def test_tile_variants_give_identical_bits(epi):
     c.close()
 
 
+@pytest.mark.parametrize("epi", ["f32", "resid", "swiglu"])
+def test_tile_walk_gives_identical_bits(epi):
+    """The order in which workers take the output tiles (rows fastest over the whole M, or bands of 1,
+    3 or 8 row tiles; with or without L2 eviction hints on the loads) never changes a result bit:
+    every element is still summed over K in the same order.  Shapes: one whose A share exceeds the
+    automatic threshold (K = 14336, the 7B-class down projection, with its K split in two for the
+    residual form) and a ragged one (M = 3000: a last band narrower than the others)."""
+    from paper_2609_25405_b200 import binding as B
+    # a context of the 7B-class width: its residual form splits the K of the down projection in two
+    c = B.Context(B.model_cfg(synth.SHAPES["7b"].with_layers(1), 64), 4096, 8, 64)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    code = {"f32": B.EPI_F32, "resid": B.EPI_RESID_F32, "swiglu": B.EPI_SWIGLU}[epi]
+    try:
+        for M, N, K in [(4096, 4096, 14336), (3000, 2048, 4096)]:
+            A = torch.randn((M, K), generator=g, device="cuda").to(torch.float16)
+            Bw = (torch.randn((N, K), generator=g, device="cuda") * 0.05).to(torch.float16)
+            width, dt = (N // 2, torch.float16) if epi == "swiglu" else (N, torch.float32)
+            C0 = torch.randn((M, width), generator=g, device="cuda").to(dt)
+            outs = []
+            for band, hints in [(-1, -1), (0, 0), (1, 1), (3, 0), (8, 1)]:
+                B.gemm_set_walk(band, hints)
+                out = C0.clone()
+                c.gemm(A, Bw, out, M, N, K, code)
+                torch.cuda.synchronize()
+                outs.append(out)
+            for o in outs[1:]:
+                assert torch.equal(o, outs[0]), (M, N, K)
+    finally:
+        B.gemm_set_walk(-1, -1)
+    assert c.status_poll() == 0
+    c.close()
+
+
 def test_weights_pack_f16_matches_round_to_nearest(ctx):
     """bf16 -> fp16 repack: exact in the fp16 normal range, round-to-nearest on the subnormal grid,
     saturating above 65504; in place."""
