@@ -523,6 +523,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--sessions", type=int, default=256, help="sessions of the cfg5-trace-1b workload")
     ap.add_argument("--gemm-walk", default="", help="tuning: force the projection GEMM's tile walk, 'band,hints' (see hb_gemm_set_walk)")
+    ap.add_argument("--gemm-ctas", type=int, default=0, help="tuning: cap the CTAs of every projection GEMM launch")
     ap.add_argument("--lora-rank", type=int, default=0,
                     help="rank of a random low-rank adapter applied to the embedding rows (0 = none, the headline)")
     args = ap.parse_args()
@@ -543,6 +544,9 @@ def main():
     if args.gemm_walk:
         from paper_2609_25405_b200 import binding as _B
         _B.gemm_set_walk(*[int(v) for v in args.gemm_walk.split(",")])
+    if args.gemm_ctas:
+        from paper_2609_25405_b200 import binding as _B
+        _B.gemm_set_cta_limit(args.gemm_ctas)
     if args.workload.startswith("cfg5-trace"):
         run_trace(args)
         return

@@ -382,6 +382,10 @@ HB_API int hb_gemm_pair(hb_ctx* ctx, const void* A, const void* B, const void* A
  * exactly that, and a profile can compare DRAM traffic.  band >= 1: row tiles per band; band = 0: whole
  * M; hints 0 / 1; -1 for either = automatic again.  Host only, not thread-safe against launches. */
 HB_API int hb_gemm_set_walk(int32_t band, int32_t hints);
+/* Tuning: cap the CTAs of every projection launch at max_ctas (even; 0 = one per SM again), e.g. to
+ * leave SMs to kernels of another stream.  Changes the work split between workers only, never a
+ * result bit.  Host only, process-wide. */
+HB_API int hb_gemm_set_cta_limit(int32_t max_ctas);
 
 /* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
  * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of

@@ -106,6 +106,7 @@ _sig = {
     "hb_profile_read": [_P, C.POINTER(C.c_float), C.POINTER(C.c_int32)],
     "hb_gemm": [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
     "hb_gemm_set_walk": [C.c_int32, C.c_int32],
+    "hb_gemm_set_cta_limit": [C.c_int32],
 }
 for _name, _args in _sig.items():
     _f = getattr(lib, _name)
@@ -580,6 +581,11 @@ def pool_chunk_noalloc(x, gain, n_rows, d_model, rms_eps, mode, first_chunk, is_
 def gemm_set_walk(band=-1, hints=-1):
     """Force the projection GEMM's tile walk (tests / tuning); -1 = automatic."""
     check(lib.hb_gemm_set_walk(band, hints), "hb_gemm_set_walk")
+
+
+def gemm_set_cta_limit(max_ctas=0):
+    """Cap the CTAs of every projection GEMM launch (tuning); 0 = one per SM."""
+    check(lib.hb_gemm_set_cta_limit(max_ctas), "hb_gemm_set_cta_limit")
 
 
 def validate_desc(cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, batch):

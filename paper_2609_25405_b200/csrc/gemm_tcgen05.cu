@@ -727,7 +727,9 @@ int hb_gemm_box_rows(int variant) { return variant == HB_GEMM_PAIR256 ? 128 : va
 // through hb_gemm_set_walk.
 static int g_band_override = -1;   // >= 0: test / tuning override of the band (0 = whole M)
 static int g_hint_override = -1;
+static int g_cta_limit = 0;        // > 0: launches use at most this many CTAs (an even number for CTA pairs)
 void hb_gemm_walk_override(int band, int hints) { g_band_override = band; g_hint_override = hints; }
+void hb_gemm_cta_limit(int max_ctas) { g_cta_limit = max_ctas; }
 
 void hb_gemm_pick_walk(int variant, int epi, GemmArgs* g) {
   const int tile_rows = (variant == HB_GEMM_PAIR256) ? 256 : 128;
@@ -760,6 +762,7 @@ int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int variant, 
   const CUtensorMap& b2 = tmB2 ? *tmB2 : tmB;
   GemmArgs g = a;
   hb_gemm_pick_walk(variant, epi, &g);
+  if (g_cta_limit > 0 && g_cta_limit < num_sms) num_sms = g_cta_limit;
   if (variant == HB_GEMM_PAIR256) return launch_bn<256, 2>(tmA, tmB, a2, b2, epi, g, num_sms, s, pdl);
   if (variant == 256) return launch_bn<256, 1>(tmA, tmB, a2, b2, epi, g, num_sms, s, pdl);
   if (variant == 128) return launch_bn<128, 1>(tmA, tmB, a2, b2, epi, g, num_sms, s, pdl);

@@ -169,7 +169,8 @@ int hb_gemm_pick_ksplit(int M, int N, int K, int variant, int num_sms);
 int hb_gemm_pick_step_variant(int map_variant, int rows, int N, int k_blocks, int k_splits, int num_sms);
 // Chooses GemmArgs::raster_band and l2_hints for a launch of `variant` (called by hb_gemm_launch).
 void hb_gemm_pick_walk(int variant, int epi, GemmArgs* g);
-void hb_gemm_walk_override(int band, int hints);   // tuning: >= 0 forces the value for every launch, -1 = automatic
+void hb_gemm_walk_override(int band, int hints);
+void hb_gemm_cta_limit(int max_ctas);   // tuning: > 0 caps the CTAs of every projection launch, 0 = all SMs   // tuning: >= 0 forces the value for every launch, -1 = automatic
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,
                    const CUtensorMap* tmB2 = nullptr, bool pdl = false);

@@ -987,6 +987,12 @@ int hb_gemm_set_walk(int32_t band, int32_t hints) {
   return HB_OK;
 }
 
+int hb_gemm_set_cta_limit(int32_t max_ctas) {
+  if (max_ctas < 0 || (max_ctas & 1)) return HB_ERR_BAD_ARG;
+  hb_gemm_cta_limit(max_ctas);
+  return HB_OK;
+}
+
 int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int32_t epilogue,
             void* stream) {
   return hb_gemm_pair(c, A, B, nullptr, nullptr, C, M, N, K, 0, epilogue, stream);

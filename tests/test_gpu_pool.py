@@ -39,7 +39,10 @@ def test_pool_chunks_match_oracle(d, mode):
         assert list(meta) == [st.count, st.chunks, code, 1 if final else 0]
         if mode in ("mean", "wmean"):
             S = slot_sum.cpu().numpy().astype(np.float64)
-            assert np.max(np.abs(S - st.S)) <= 1e-5 * np.sqrt(st.count) * 4 + 2e-6 * np.max(np.abs(st.S))
+            err = np.max(np.abs(S - st.S))
+            print(f"\n  d={d} {mode} count={st.count}: max |S - oracle| = {err:.3e} = {err / np.max(np.abs(st.S)):.2e} x max|S|"
+                  f" = {err / (np.sqrt(st.count) * 2.0 ** -24 * np.max(np.abs(st.S))):.2f} x sqrt(n) u max|S|")
+            assert err <= 1e-5 * np.sqrt(st.count) * 4 + 1e-6 * np.max(np.abs(st.S))
         if mode == "cls":
             S = slot_sum.cpu().numpy().astype(np.float64)
             assert np.max(np.abs(S - st.retained)) <= 1e-5

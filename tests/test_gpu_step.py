@@ -149,9 +149,12 @@ def test_cfg1_mean_state_after_each_chunk(weights):
         assert list(meta[:2]) == list(M.pool_counters_after([33, 1, 50, 16][:k + 1]))
         S = eng.pool.sums()[req.slot].cpu().numpy().astype(np.float64)
         ref = hh[:at].sum(0)
-        # per-row error of the unit-rms hidden states is bounded like the embedding tolerance;
-        # rounding errors of near-identical rows are correlated, so the bound grows with the count
-        assert np.max(np.abs(S - ref)) <= 1e-2 * at
+        # every row of the unit-rms hidden states carries an fp16-path error of a few 1e-3 against the
+        # oracle; the errors of different rows are largely independent, so the sum's error grows like
+        # sqrt(rows): measured 6.5e-3 to 7.2e-3 x sqrt(rows) over these four states
+        print(f"\n  mean-pool state after {at} rows: max |S - oracle| = {np.max(np.abs(S - ref)):.3e} "
+              f"({np.max(np.abs(S - ref)) / at:.2e} per row, {np.max(np.abs(S - ref)) / np.sqrt(at):.2e} per sqrt(row))")
+        assert np.max(np.abs(S - ref)) <= 2e-2 * np.sqrt(at)
     assert eng.ctx.status_poll() == 0
     eng.close()
 
@@ -433,3 +436,76 @@ def test_bad_descriptor_enqueues_nothing(weights):
     torch.cuda.synchronize()
     assert torch.all(eng.kv.arena == KV_SENTINEL)
     eng.close()
+
+
+class _ScaledWeights:
+    """synth.Weights with the FFN-norm gain of every layer set to `ffn_gain` (a power of two, so it is
+    bf16-exact): the inputs of the gate/up projection, and with them the SwiGLU outputs, leave the
+    range of the N(0, 0.02^2), gain-1 models of the configurations, while attention stays as it is."""
+
+    def __init__(self, W, ffn_gain, nan_token=None):
+        self.W, self.shape, self.ffn_gain, self.nan_token = W, W.shape, np.float32(ffn_gain), nan_token
+
+    def layer(self, l):
+        w = dict(self.W.layer(l))
+        w["ffn_norm"] = np.full_like(w["ffn_norm"], self.ffn_gain)
+        return w
+
+    @property
+    def tok_emb(self):
+        t = self.W.tok_emb
+        if self.nan_token is not None:
+            t = t.copy()
+            t[self.nan_token] = np.nan
+        return t
+
+    @property
+    def lm_head(self):
+        return self.W.lm_head
+
+    @property
+    def final_norm(self):
+        return self.W.final_norm
+
+
+def test_fp16_range_large_ffn_gain_and_nan():
+    """Where the fp16 operand range ends.  With an FFN-norm gain of 64 the inputs of gate/up are 64
+    times the configurations' and the SwiGLU outputs about 4000 times (hundreds to thousands): still
+    inside fp16, the step matches the oracle within the usual tolerances with a clean status word.
+    With a gain of 2048 the SwiGLU outputs pass 65504: they are stored saturated, the step REPORTS it
+    (status bit 64), outputs stay finite and the context stays usable.  A NaN in the residual stream
+    (a NaN token-embedding row) is reported the same way and reaches the logits as NaN instead of
+    being clamped to a finite number."""
+    from paper_2609_25405_b200 import binding as B
+    from paper_2609_25405_b200.engine import Engine, Request
+    rng = np.random.default_rng(99)
+    toks = synth.token_ids(rng, 90, TINY.V)
+    prompt = synth.token_ids(rng, 70, TINY.V)
+
+    def run(W):
+        eng = Engine(TINY, B.DeviceWeights.from_synth(W), 64, 4, 512, 16, 256)
+        e, g = Request("embed", toks, B.POOL_MEAN), Request("gen", prompt)
+        _, lr, er = eng.step([(g, 70), (e, 90)])
+        torch.cuda.synchronize()
+        out = eng.out_logits[lr[g]].cpu().numpy().astype(np.float64), eng.out_emb[er[e]].cpu().numpy().astype(np.float64)
+        status = eng.ctx.status_poll()
+        assert eng.ctx.status_poll() == 0            # polling cleared it; the context is usable
+        eng.close()
+        return out, status
+
+    base = synth.Weights(TINY, 0)
+    # (1) inside the range
+    W = _ScaledWeights(base, 64.0)
+    (lg, emb), status = run(W)
+    assert status == 0
+    _, ref_lg = T.forward(TINY, W, prompt, logit_rows=[69])
+    assert np.max(np.abs(lg - ref_lg[0])) <= LOGIT_ABS
+    _check_emb(emb, T.embed(TINY, W, toks, "mean"))
+    # (2) SwiGLU outputs beyond the largest finite half: saturated and reported
+    (lg, emb), status = run(_ScaledWeights(base, 2048.0))
+    assert status & 64
+    assert np.all(np.isfinite(lg)) and np.all(np.isfinite(emb))
+    # (3) NaN in: reported, and NaN (not a clamped number) out
+    (lg, emb), status = run(_ScaledWeights(base, 1.0, nan_token=int(prompt[-1])))
+    assert status & 64
+    assert np.all(np.isnan(lg))
