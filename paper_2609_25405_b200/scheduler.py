@@ -1,13 +1,14 @@
-"""Intra-batch scheduling (Algorithm 2 of the paper) as host-side glue.
+"""Intra-batch scheduling (Section 4.2 of the paper) as host-side glue.
 
 Composes one iteration's batch from an embedding queue Q_e and a generation queue Q_g under a
-token budget B: capacity is first reserved for in-flight decodes (`ScheduleRunning`), then the rest
-is filled by picking, one item at a time, from the queue with the larger credit.  Credits a_e, a_g
-grow by the queues' remaining-token weights w_e, w_g at every selection step, the chosen queue pays
-w_e + w_g, credits persist across iterations and are reset when their queue is empty
-(Section 4.2).  `ScheduleOne` admits the next request of a queue in arrival order (per-type FCFS)
-as a chunk of at most C tokens that fits the residual budget; a request contributes at most one
-chunk per iteration because chunk k + 1 reads the K/V chunk k writes.
+token budget B: capacity is first reserved for in-flight decodes, then the rest is filled one
+admission at a time from the type with the larger credit.  Credits grow by the queues'
+remaining-token weights at every selection, the chosen type pays the sum of both weights, credits
+persist across iterations and are reset when their queue is empty.  An admission is the next
+request of a type in arrival order (per-type FCFS) as a chunk of at most C tokens that fits the
+residual budget; a request contributes at most one chunk per iteration because chunk k + 1 reads
+the K/V chunk k writes.  One deliberate difference from a literal reading of Algorithm 2: a type
+that can contribute nothing more to the iteration stops earning credit for the rest of it.
 
 This module decides WHAT goes into a batch; `engine.Engine.step` runs it.  It holds no arithmetic of
 the forward pass.
@@ -29,6 +30,39 @@ class Work:
         return f"Work({self.kind}, remaining={self.remaining}, decode_left={self.decode_left})"
 
 
+class _Credits:
+    """Token-weighted credits of the two request types (Section 4.2).  A type that can still
+    contribute to the batch being composed earns its backlog weight at every selection; the type
+    picked pays the sum of both weights, so over a run of selections the picks follow the weights
+    within one selection (the paper's fairness bound).  Credits are kept between iterations and
+    dropped for a type whose queue is empty."""
+
+    def __init__(self):
+        self.a = {"embed": 0, "gen": 0}
+
+    def start_iteration(self, weights):
+        self.w = dict(weights)
+        for kind, w in weights.items():
+            if w == 0:
+                self.a[kind] = 0            # an empty queue carries no claim into the future
+
+    def accrue(self, candidates):
+        """One selection opportunity: only types that can still be admitted in this iteration earn
+        (a type closed for the iteration would otherwise pile up credit it could never have spent
+        here, beyond the one-opportunity bound)."""
+        for kind in candidates:
+            self.a[kind] += self.w[kind]
+
+    def pick(self, candidates):
+        """The candidate with the larger credit; embedding wins ties."""
+        if len(candidates) == 1:
+            return candidates[0]
+        return "embed" if self.a["embed"] >= self.a["gen"] else "gen"
+
+    def charge(self, kind):
+        self.a[kind] -= self.w["embed"] + self.w["gen"]
+
+
 class IBS:
     def __init__(self, budget, chunk, chunked=True, decode_rows=1):
         """budget B (tokens per iteration), chunk cap C; chunked=False makes embedding requests
@@ -36,14 +70,25 @@ class IBS:
         decode_rows = budget tokens an in-flight decode takes per iteration (1 in the real step)."""
         self.B, self.C, self.chunked = int(budget), int(chunk), bool(chunked)
         self.decode_rows = int(decode_rows)
-        self.a_e = 0
-        self.a_g = 0
+        self.credits = _Credits()
         self.Qe, self.Qg = deque(), deque()
         self.running = {}                   # generation requests in their decode phase (insertion-ordered set)
+
+    # credits as the paper names them
+    @property
+    def a_e(self):
+        return self.credits.a["embed"]
+
+    @property
+    def a_g(self):
+        return self.credits.a["gen"]
 
     # ---- queues ----
     def submit(self, work):
         (self.Qe if work.kind == "embed" else self.Qg).append(work)
+
+    def _queue(self, kind):
+        return self.Qe if kind == "embed" else self.Qg
 
     def _weight(self, Q):
         return sum(w.remaining for w in Q)
@@ -54,8 +99,9 @@ class IBS:
         else:
             Q.remove(w)
 
-    # ---- Algorithm 2 ----
-    def _schedule_running(self, budget):
+    # ---- composing one iteration (Section 4.2) ----
+    def _reserve_running(self, budget):
+        """In-flight decodes come first: each takes its rows out of the budget."""
         batch, used = [], 0
         for w in self.running:
             if used + self.decode_rows > budget:
@@ -64,51 +110,38 @@ class IBS:
             used += self.decode_rows
         return batch, used
 
-    def _schedule_one(self, Q, budget, taken):
-        """Next request of Q in arrival order that has not contributed this iteration; a chunk of at
-        most C tokens that fits.  Returns (item or None, tokens used)."""
-        for w in Q:
+    def _next_admission(self, kind, budget, taken):
+        """The next request of `kind` in arrival order that has not contributed to this iteration, as
+        (work, rows): a chunk of at most C tokens that fits the residual budget.  None when the type
+        can contribute nothing more (per-type FCFS: a request that does not fit is not overtaken)."""
+        for w in self._queue(kind):
             if id(w) in taken:
                 continue
             if w.kind == "embed" and not self.chunked:
                 rows = w.remaining if w.remaining <= budget else 0      # atomic: whole request or nothing
             else:
                 rows = min(self.C, w.remaining, budget)
-            if rows <= 0:
-                return None, 0              # the next request in line does not fit: per-type FCFS forbids overtaking
-            return (w, rows), rows
-        return None, 0
+            return (w, rows) if rows > 0 else None
+        return None
 
     def schedule(self):
         """One call = one iteration.  Returns the batch as a list of (Work, rows)."""
-        batch, used = self._schedule_running(self.B)
-        B = self.B - used
-        w_e, w_g = self._weight(self.Qe), self._weight(self.Qg)
-        if not self.Qe:
-            self.a_e = 0
-        if not self.Qg:
-            self.a_g = 0
+        batch, used = self._reserve_running(self.B)
+        left = self.B - used
+        self.credits.start_iteration({"embed": self._weight(self.Qe), "gen": self._weight(self.Qg)})
         taken = set()
-        open_e, open_g = bool(self.Qe), bool(self.Qg)
-        while B > 0 and (open_e or open_g):
-            self.a_e += w_e
-            self.a_g += w_g
-            pick_e = (not open_g) or (open_e and self.a_e >= self.a_g)
-            Q = self.Qe if pick_e else self.Qg
-            item, u = self._schedule_one(Q, B, taken)
-            if item is None:                # nothing more from this queue in this iteration
-                if pick_e:
-                    open_e = False
-                else:
-                    open_g = False
+        candidates = [k for k in ("embed", "gen") if self._queue(k)]
+        while left > 0 and candidates:
+            self.credits.accrue(candidates)
+            kind = self.credits.pick(candidates)
+            item = self._next_admission(kind, left, taken)
+            if item is None:
+                candidates.remove(kind)     # closed for this iteration: it neither earns nor is picked again
                 continue
             batch.append(item)
             taken.add(id(item[0]))
-            B -= u
-            if pick_e:
-                self.a_e -= (w_e + w_g)
-            else:
-                self.a_g -= (w_e + w_g)
+            left -= item[1]
+            self.credits.charge(kind)
         return batch
 
     def commit(self, batch):

@@ -180,3 +180,28 @@ def test_compute_calls_fail_loudly_without_a_device():
         pytest.skip("has a device")
     with pytest.raises(RuntimeError):
         B.Context(CFG, 64, 8, 64)
+
+
+def test_misaligned_pointers_and_bad_tuning_arguments_are_refused_on_the_host():
+    """The no-allocation pooler checks its pointers before it touches CUDA: a view that starts in the
+    middle of a 16-byte vector (x, slot, output) or of an 8-byte one (gain) is HB_ERR_BAD_ARG, and
+    nothing is launched (no device is needed to see the refusal).  The GEMM tuning calls refuse
+    values outside their documented ranges."""
+    import ctypes as C
+    P = C.c_void_p
+    ok = dict(x=0x10000, gain=0x20000, s=0x30000, m=0x40000, e=0x50000)
+
+    def call(**kw):
+        a = dict(ok, **kw)
+        return B.lib.hb_pool_chunk_noalloc(P(a["x"]), P(a["gain"]), 8, 256, C.c_float(1e-5), B.POOL_MEAN, 1, 1, P(a["s"]),
+                                           P(a["m"]), P(a["e"]), None)
+    assert call(x=0x10004) == -1 and call(s=0x30008) == -1 and call(e=0x5000c) == -1
+    assert call(gain=0x20002) == -1 and call(gain=0x20004) == -1 and call(m=0x40002) == -1
+    assert B.lib.hb_pool_chunk_noalloc(P(ok["x"]), P(ok["gain"]), 8, 254, C.c_float(1e-5), B.POOL_MEAN, 1, 1, P(ok["s"]),
+                                       P(ok["m"]), P(ok["e"]), None) == -1          # d_model not a multiple of 4
+    assert B.lib.hb_pool_chunk_noalloc(P(ok["x"]), P(ok["gain"]), 4096, 256, C.c_float(1e-5), B.POOL_MEAN, 1, 1,
+                                       P(ok["s"]), P(ok["m"]), P(ok["e"]), None) == -5   # beyond the fixed scratch
+    assert B.lib.hb_gemm_set_walk(-2, 0) == -1 and B.lib.hb_gemm_set_walk(0, 2) == -1
+    assert B.lib.hb_gemm_set_walk(-1, -1) == 0
+    assert B.lib.hb_gemm_set_cta_limit(7) == -1 and B.lib.hb_gemm_set_cta_limit(-2) == -1
+    assert B.lib.hb_gemm_set_cta_limit(0) == 0

@@ -142,3 +142,22 @@ def test_printed_packing_simulation_direction():
         atomic = packing_fill(256, 64, chunked=False, n_iters=3000, seed=seed, arrivals_per_iter=0.5)
         chunked = packing_fill(256, 64, chunked=True, n_iters=3000, seed=seed, arrivals_per_iter=0.5)
         assert chunked > atomic + 0.02
+
+
+def test_a_type_closed_for_the_iteration_stops_earning_credit():
+    """Per-type FCFS can close a type early (its next request does not fit the residual budget when
+    requests are atomic).  From then on only the other type earns and pays within the iteration, so
+    the closed type's credit is what it was when it closed: it cannot bank more than the one
+    selection opportunity the fairness bound of Section 4.2 allows."""
+    sch = IBS(100, 100, chunked=False)
+    sch.submit(Work("embed", 90))            # atomic: fits once, then the next one (90) does not fit
+    sch.submit(Work("embed", 90))
+    for _ in range(30):
+        sch.submit(Work("gen", 1))
+    batch = sch.schedule()
+    kinds = [w.kind for w, _ in batch]
+    assert kinds.count("embed") == 1 and kinds.count("gen") == 10
+    w_e, w_g = 180, 30
+    # the embedding type earned at most for the selections up to the one that closed it: its credit is
+    # bounded by one opportunity's worth, not by the ten generation picks that followed
+    assert sch.a_e <= w_e + w_g
