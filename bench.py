@@ -31,7 +31,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # a small data file beside the capture's summary holds the bytes per projection and the hash of the
 # kernel source at capture time.  When the kernel source has changed since, the figure is stale and
 # the line says `traffic: null`.
-GEMM_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "gemm_tcgen05_cfg3-7b_layers2.traffic.json")
+GEMM_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "gemm_tcgen05_cfg3-7b_layers2.traffic.txt")
 GEMM_SOURCE = os.path.join(ROOT, "paper_2609_25405_b200", "csrc", "gemm_tcgen05.cu")
 
 
