@@ -1,7 +1,7 @@
 """Decode rows over long cached contexts against the oracle, at every count of key splits the host
-can choose, on two small shapes: the tiny one (head_dim 64, one query head per KV head) and a
-head_dim-128 shape with four query heads sharing one KV head, the head geometry of the 7B-class
-configuration.  The cached contexts are written by the library itself (the prompts are prefilled
+can choose, on small shapes: the tiny one (head_dim 64, one query head per KV head), a
+head_dim-128 shape with four query heads sharing one KV head (the head geometry of the 7B-class
+configuration), and two more group sizes (eight heads x 64 on one KV head; four x 128 on two).  The cached contexts are written by the library itself (the prompts are prefilled
 through hb_mixed_step in chunks of 512, so chunk rows with more than 1024 earlier tokens are
 compared too), then every request decodes one row.
 
@@ -30,6 +30,9 @@ SHAPES = {
     "tiny": synth.SHAPES["tiny"],
     # 2 layers, d 512, 4 query heads x 128 on 1 KV head (group of 4), FFN 1024, vocabulary 1024
     "dh128": synth.ModelShape("dh128", 2, 512, 4, 1, 128, 1024, 1024),
+    # the other group sizes the attention tiles allow: 8 query heads x 64 on 1 KV head, and 4 x 128 on 2
+    "g8": synth.ModelShape("g8", 2, 512, 8, 1, 64, 1024, 1024),
+    "g2dh128": synth.ModelShape("g2dh128", 2, 512, 4, 2, 128, 1024, 1024),
 }
 
 
@@ -42,7 +45,7 @@ def test_split_rule_of_the_chosen_contexts():
         assert (n + per - 1) // per == want, (ctx, want)
 
 
-@pytest.mark.parametrize("name", ["tiny", "dh128"])
+@pytest.mark.parametrize("name", ["tiny", "dh128", "g8", "g2dh128"])
 def test_decode_rows_at_every_split_count_match_oracle(name):
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
