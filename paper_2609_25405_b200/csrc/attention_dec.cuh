@@ -161,10 +161,20 @@ __device__ __forceinline__ void warp_attend(const uint32_t (&qf)[DH / 16][4], ui
 template <int DH>
 constexpr int smem_bytes(int max_pos) { return TILE_KEYS * DH * 2 * (2 * STAGES) + 64 + (max_pos / 16 + 2) * 4 + 1024; }
 
-// One CTA of ATT_THREADS threads, item `item` of p.items.  `kv_map_p` points at the kernel's
-// __grid_constant__ tensor map.
+// The item's barrier words stop being barriers (the block's next item may lay its shared memory out
+// differently).  One thread, after the block has met at a barrier.
 template <int DH>
-__device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const AttnParams& p, int item) {
+__device__ __forceinline__ void retire_barriers(uint32_t smem_base) {
+  const uint32_t kv_s = (smem_base + 1023u) & ~1023u;
+  for (int st = 0; st < STAGES; ++st) mbar_inval(kv_s + STAGES * 2 * (TILE_KEYS * DH * 2) + 8u * st);
+}
+
+// One CTA of ATT_THREADS threads, item `item` of p.items.  `kv_map_p` points at the kernel's
+// __grid_constant__ tensor map.  Returns false in thread 0 when the block must not take further items.
+// `at_start` is called once, first thing, by thread ATT_COMPUTE + 32 (first lane of the warp that
+// neither computes nor talks to TMA): whatever it waits for hides behind the item's first loads.
+template <int DH, class AtStart>
+__device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const AttnParams& p, int item, AtStart&& at_start) {
   constexpr int CH = DH / 8;                          // 16-byte chunks per row
   constexpr int TILE_BYTES = TILE_KEYS * DH * 2;
   constexpr int REC = DH + 2;                         // floats per row of a partial record
@@ -250,6 +260,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
       issued = n_init;
     }
   }
+  if (tid == ATT_COMPUTE + 32) at_start();
   // page ids of the keys this item reads -> shared memory (checked once)
   for (int i = tid; i < n_blk; i += ATT_THREADS) {
     const int blk = first_blk + i;
@@ -274,7 +285,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
     }
     cp_async_wait<0>();
     __syncthreads();
-    return;
+    return false;
   }
 
   // rows of this thread: chunk items: warp-private rows; decode items: rows 0..15 for every warp
@@ -342,10 +353,10 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
   if (__syncthreads_or(failed)) {
     if (prod) {
       atomicOr(p.status, HB_DEV_ATTN_WAIT_EXPIRED);
-      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block retires
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block goes on
     }
     __syncthreads();
-    return;
+    return false;
   }
   // row sums: add the four threads of a quad
 #pragma unroll
@@ -355,7 +366,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
   }
 
   if (!decode) {
-    if (!compute) return;
+    if (!compute) return true;
     // ---- chunk item: normalise, stage the warp's 16 rows in shared memory, store 16-byte vectors ----
     const float inv_a = (l[0] > 0.0f) ? 1.0f / l[0] : 0.0f, inv_b = (l[1] > 0.0f) ? 1.0f / l[1] : 0.0f;
     uint8_t* stage = smem;  // the ring is idle now; this warp touches its own 16 rows of the first tile only
@@ -376,7 +387,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
         *reinterpret_cast<uint4*>(p.out + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8) = v;
       }
     }
-    return;
+    return true;
   }
 
   // ---- decode item: merge the four warps' partials in shared memory ----
@@ -425,7 +436,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
       }
     }
   }
-  if (it.n_splits == 1) return;
+  if (it.n_splits == 1) return true;
   // ---- splits of this (row, kv head): the CTA that arrives last merges them in split order ----
   __threadfence();
   __syncthreads();
@@ -435,7 +446,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
     is_last_s = (prev + 1u == static_cast<uint32_t>(it.n_splits)) ? 1u : 0u;
   }
   __syncthreads();
-  if (!is_last_s) return;
+  if (!is_last_s) return true;
   __threadfence();
   const float* recs = p.part + static_cast<size_t>(it.part_base) * G * REC;
   for (int idx = tid; idx < G * DH; idx += ATT_THREADS) {
@@ -453,6 +464,7 @@ __device__ __forceinline__ void small_item(const CUtensorMap* kv_map_p, const At
     p.out[(static_cast<size_t>(tok) * Hq + hk * G + g) * DH + d] = __float2half_rn(L > 0.0f ? o / L : 0.0f);
   }
   if (tid == 0) *counter = 0u;  // ready for the next launch
+  return true;
 }
 
 // Parameters of the decode / small chunk items of one layer.

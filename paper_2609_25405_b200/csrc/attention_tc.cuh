@@ -17,8 +17,9 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises a status bit and leaves without
 // storing.  The work split depends on the segment's own lengths only.
 //
-// This file is the body of one CTA; attention.cu includes it and calls it from the one attention
-// kernel of the step for the blocks that hold a chunk item.
+// This file is the body of one item; attention.cu includes it and calls it from the one attention
+// kernel of the step, whose blocks stay resident and take one item after the other.  The block's
+// 256 tensor-memory columns are allocated once by the kernel and handed in.
 #pragma once
 #include "hb_internal.h"
 #include "ptx.cuh"
@@ -60,19 +61,31 @@ struct TcCfg {
 template <int DH>
 constexpr int smem_bytes() { return TcCfg<DH>::BAR_OFF + 8 * (2 * TcCfg<DH>::STAGES + 6) + 16; }
 
-// One CTA of TC_THREADS threads, item `item` of p.items.  `kv_map` points at the kernel's
-// __grid_constant__ tensor map.
+// The item's barrier words stop being barriers: the next item of the block may lay its shared memory
+// out differently.  One thread, after the block has met at a barrier.
 template <int DH>
-__device__ __forceinline__ void chunk_item(const CUtensorMap* kv_map, const TcParams& p, int item) {
+__device__ __forceinline__ void retire_barriers(uint32_t smem_base) {
+  for (int i = 0; i < 2 * TcCfg<DH>::STAGES + 6; ++i) mbar_inval(smem_base + TcCfg<DH>::BAR_OFF + 8u * i);
+}
+
+// One CTA of TC_THREADS threads, item `item` of p.items, with TcCfg::TMEM_COLS columns of tensor memory
+// at `tmem`.  `kv_map` points at the kernel's __grid_constant__ tensor map.  Returns false (the same
+// value in every thread) when the block must not take further items; *barriers_live tells whether
+// retire_barriers is due.  `last_issue` is called once by thread 0 (the thread that talks to TMA) when
+// it has requested the item's last key tile, i.e. a few tiles before the item ends (not on error paths).
+template <int DH, class LastIssue>
+__device__ __forceinline__ bool chunk_item(const CUtensorMap* kv_map, const TcParams& p, int item, uint32_t tmem,
+                                           bool* barriers_live, LastIssue&& last_issue) {
   using C = TcCfg<DH>;
   extern __shared__ uint8_t smem_raw[];
   // The kernel has no static shared memory, so the dynamic window starts at the CTA's (1 KiB
   // aligned) shared-memory base, which the swizzled tiles need; checked, not assumed.
   const uint32_t base = smem_u32(smem_raw);
   uint8_t* smem = smem_raw;
+  *barriers_live = false;
   if (base & 1023u) {
     if (threadIdx.x == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
-    return;
+    return false;
   }
   const uint32_t ring_s = base, p_s = ring_s + C::RING, bar_s = base + C::BAR_OFF;
   auto kv_full = [&](int s) { return bar_s + 8u * s; };
@@ -82,8 +95,7 @@ __device__ __forceinline__ void chunk_item(const CUtensorMap* kv_map, const TcPa
   // while the softmax threads are still producing the second
   const uint32_t q_ready = bar_s + 8u * (2 * C::STAGES + 2), p_ready2 = bar_s + 8u * (2 * C::STAGES + 3),
                  p_ready = bar_s + 8u * (2 * C::STAGES + 4), pv_done = bar_s + 8u * (2 * C::STAGES + 5);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
-  volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile uint32_t* abort_flag = reinterpret_cast<uint32_t*>(smem + C::BAR_OFF + 8 * (2 * C::STAGES + 6));
 
   const AttnItem it = p.items[item];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -108,19 +120,12 @@ __device__ __forceinline__ void chunk_item(const CUtensorMap* kv_map, const TcPa
     const int pg = (i < it.pt_len) ? p.pages[it.pt_start + i] : -1;
     bad |= (pg < 0 || pg >= p.n_pages);
   }
-  if (__syncthreads_or(bad)) {
+  *barriers_live = true;
+  if (__syncthreads_or(bad)) {   // also publishes the barrier initialisation
     if (tid == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
-    return;             // nothing requested from TMA, no TMEM held
+    return false;       // nothing requested from TMA
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(static_cast<uint32_t>(C::TMEM_COLS)) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  tc_fence_after();     // tensor-memory accesses of the block's previous item are ordered before this one's
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -153,6 +158,7 @@ __device__ __forceinline__ void chunk_item(const CUtensorMap* kv_map, const TcPa
             tma_load_2d(k_dst + pi * C::PAGE_BYTES, kv_map, kv_full(st), 0, row);   // K and V of this head, one copy
           }
         }
+        if (j == n_tiles - 1) last_issue();
       }
     }
     __syncwarp();
@@ -360,18 +366,15 @@ __device__ __forceinline__ void chunk_item(const CUtensorMap* kv_map, const TcPa
 
   tc_fence_before();
   __syncthreads();
-  if (*abort_flag) {
+  const bool aborted = (*abort_flag != 0u);
+  if (aborted) {
     if (tid == 0) {
       atomicOr(p.status, HB_DEV_ATTN_WAIT_EXPIRED);
-      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block retires
+      for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let requested copies land before the block goes on
     }
     __syncthreads();
   }
-  if (warp == 1) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
-                 "r"(static_cast<uint32_t>(C::TMEM_COLS)) : "memory");
-  }
+  return !aborted;
 }
 
 // Parameters of the chunk items of one layer.

@@ -12,6 +12,8 @@
 
 #include "../../include/hb.h"
 
+// Words of the status block the attention kernel uses as its work queue (tickets, blocks gone).
+constexpr int HB_STATUS_ATTN_QUEUE_WORD = 8;
 // Device status codes (OR-ed into the context's status word).
 enum : uint32_t {
   HB_DEV_GEMM_WAIT_EXPIRED = 1u << 0,
@@ -238,7 +240,7 @@ struct hb_ctx {
   float* pool_part;         // pooling partial sums
   uint32_t* counters;       // arrival counters of the pooling merge, one per segment
   uint32_t* attn_counters;  // arrival counters of the split-KV merge, one per (segment, kv head)
-  uint32_t* status;         // device status word
+  uint32_t* status;         // device status word (256-byte block: word 0 status, words 8 and 9 the attention work queue)
   uint8_t* desc_dev;        // packed descriptor
   size_t desc_cap;
   void* extra;              // host-side state (pinned descriptor staging ring, layout)

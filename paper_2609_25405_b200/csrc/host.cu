@@ -667,12 +667,14 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   // Both lists go to the device sorted by cost, largest first (equal costs in list order).  The sort
   // runs over (cost, index) keys in a vector the context owns (std::sort works in place), and the
   // items are copied into the staging buffer in that order.
-  auto sorted_into = [&](const std::vector<AttnItem>& items, uint8_t* dst) {
+  // (a tensor-core tile costs its 128 rows whatever part of them is filled)
+  auto sorted_into = [&](const std::vector<AttnItem>& items, uint8_t* dst, bool full_tiles) {
     std::vector<uint64_t>& keys = ex->sort_keys;
     keys.clear();
     for (size_t i = 0; i < items.size(); ++i) {
       const AttnItem& a = items[i];
-      const uint64_t cost = static_cast<uint64_t>(a.key1 - a.key0) * static_cast<uint64_t>(a.mode ? 16 : a.n_rows);
+      const uint64_t cost = static_cast<uint64_t>(a.key1 - a.key0) *
+                            static_cast<uint64_t>(full_tiles ? ATT_TC_ROWS : (a.mode ? 16 : a.n_rows));
       keys.push_back(((0xffffffffull - std::min<uint64_t>(cost, 0xffffffffull)) << 32) | static_cast<uint64_t>(i));
     }
     std::sort(keys.begin(), keys.end());
@@ -684,8 +686,8 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   const size_t o_pitems = place(pitems.size() * sizeof(PoolItem));
   if (off > c->desc_cap) return HB_ERR_TOO_LARGE;
   if (!pitems.empty()) memcpy(st.host + o_pitems, pitems.data(), pitems.size() * sizeof(PoolItem));
-  sorted_into(aitems, st.host + o_aitems);
-  sorted_into(titems, st.host + o_titems);
+  sorted_into(aitems, st.host + o_aitems, false);
+  sorted_into(titems, st.host + o_titems, true);
   if (cudaMemcpyAsync(c->desc_dev, st.host, off, cudaMemcpyHostToDevice, s) != cudaSuccess) return HB_ERR_CUDA;
   if (cudaEventRecord(st.ev, s) != cudaSuccess) return HB_ERR_CUDA;
   st.pending = true;
@@ -947,7 +949,8 @@ int hb_status_poll(hb_ctx* c, void* stream, uint32_t* out_code) {
         cudaMemsetAsync(c->lora_counters, 0, static_cast<size_t>(c->n_lora_counters) * 4, s) != cudaSuccess ||
         cudaMemsetAsync(c->resid_turns, 0, static_cast<size_t>(c->n_resid_turns) * 4, s) != cudaSuccess)
       return HB_ERR_CUDA;
-    if (cudaMemsetAsync(c->status, 0, 4, s) != cudaSuccess) return HB_ERR_CUDA;
+    // (the status block also holds the attention kernel's work queue: words 8 and 9)
+    if (cudaMemsetAsync(c->status, 0, 64, s) != cudaSuccess) return HB_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return HB_ERR_CUDA;
   }
   if (out_code) *out_code = code;
