@@ -386,6 +386,13 @@ HB_API int hb_gemm_set_walk(int32_t band, int32_t hints);
  * leave SMs to kernels of another stream.  Changes the work split between workers only, never a
  * result bit.  Host only, process-wide. */
 HB_API int hb_gemm_set_cta_limit(int32_t max_ctas);
+/* The attention launch of a step runs min(items, 2 per SM) resident blocks that take the step's
+ * attention items (decode splits, chunk tiles) one after the other from a ticket.  This call caps the
+ * blocks of every later attention launch of the process at max_blocks (0 = automatic again), so that a
+ * test can make one block walk through many items of both kinds.  Which block runs an item never
+ * changes a result bit (an item's arithmetic is its own; the splits of a decode row are merged in
+ * split order by whichever block arrives last).  Host only, not thread-safe against launches. */
+HB_API int hb_attn_set_block_limit(int32_t max_blocks);
 
 /* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
  * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of

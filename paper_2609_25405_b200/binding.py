@@ -107,6 +107,7 @@ _sig = {
     "hb_gemm": [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P],
     "hb_gemm_set_walk": [C.c_int32, C.c_int32],
     "hb_gemm_set_cta_limit": [C.c_int32],
+    "hb_attn_set_block_limit": [C.c_int32],
 }
 for _name, _args in _sig.items():
     _f = getattr(lib, _name)
@@ -586,6 +587,11 @@ def gemm_set_walk(band=-1, hints=-1):
 def gemm_set_cta_limit(max_ctas=0):
     """Cap the CTAs of every projection GEMM launch (tuning); 0 = one per SM."""
     check(lib.hb_gemm_set_cta_limit(max_ctas), "hb_gemm_set_cta_limit")
+
+
+def attn_set_block_limit(max_blocks=0):
+    """Cap the resident blocks of every attention launch (tests); 0 = two per SM."""
+    check(lib.hb_attn_set_block_limit(max_blocks), "hb_attn_set_block_limit")
 
 
 def validate_desc(cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, batch):

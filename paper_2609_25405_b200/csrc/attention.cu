@@ -108,6 +108,8 @@ attn_varlen_kernel(const __grid_constant__ CUtensorMap kv_map, const hb_tc::TcPa
   }
 }
 
+int g_block_limit = 0;   // > 0: launches use at most this many blocks
+
 template <int DH>
 int launch(const CUtensorMap& kv_map, const hb_tc::TcParams& tp, const hb_dec::AttnParams& dp, int n_tc, int n_small,
            int max_pos, int num_sms, uint32_t* queue, cudaStream_t s, bool pdl) {
@@ -117,11 +119,14 @@ int launch(const CUtensorMap& kv_map, const hb_tc::TcParams& tp, const hb_dec::A
   const int v = n_tc > 0 ? 1 : 0;
   auto kern = v ? attn_varlen_kernel<DH, true> : attn_varlen_kernel<DH, false>;
   if (hb_ensure_dyn_smem(reinterpret_cast<const void*>(kern), configured[v], smem) != HB_OK) return HB_ERR_CUDA;
-  const int blocks = std::min(n_tc + n_small, 2 * num_sms);
+  int blocks = std::min(n_tc + n_small, 2 * num_sms);
+  if (g_block_limit > 0) blocks = std::min(blocks, g_block_limit);
   return hb_launch_kernel(kern, blocks, ATTN_THREADS, smem, s, pdl, kv_map, tp, dp, n_tc, n_small, queue, smem);
 }
 
 }  // namespace
+
+void hb_attn_block_limit(int max_blocks) { g_block_limit = max_blocks; }
 
 int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s, int which) {
   const int n_tc = (which & HB_ATTN_CHUNK_TILES) ? c->dd.n_tc_items : 0;

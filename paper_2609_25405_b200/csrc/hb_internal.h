@@ -172,6 +172,7 @@ int hb_gemm_pick_step_variant(int map_variant, int rows, int N, int k_blocks, in
 // Chooses GemmArgs::raster_band and l2_hints for a launch of `variant` (called by hb_gemm_launch).
 void hb_gemm_pick_walk(int variant, int epi, GemmArgs* g);
 void hb_gemm_walk_override(int band, int hints);
+void hb_attn_block_limit(int max_blocks);   // tests: > 0 caps the resident blocks of every attention launch, 0 = two per SM
 void hb_gemm_cta_limit(int max_ctas);   // tuning: > 0 caps the CTAs of every projection launch, 0 = all SMs   // tuning: >= 0 forces the value for every launch, -1 = automatic
 int hb_gemm_launch(const CUtensorMap& tmA, const CUtensorMap& tmB, int bn, int epi,
                    const GemmArgs& a, int num_sms, cudaStream_t s, const CUtensorMap* tmA2 = nullptr,

@@ -996,6 +996,12 @@ int hb_gemm_set_cta_limit(int32_t max_ctas) {
   return HB_OK;
 }
 
+int hb_attn_set_block_limit(int32_t max_blocks) {
+  if (max_blocks < 0) return HB_ERR_BAD_ARG;
+  hb_attn_block_limit(max_blocks);
+  return HB_OK;
+}
+
 int hb_gemm(hb_ctx* c, const void* A, const void* B, void* C, int32_t M, int32_t N, int32_t K, int32_t epilogue,
             void* stream) {
   return hb_gemm_pair(c, A, B, nullptr, nullptr, C, M, N, K, 0, epilogue, stream);
