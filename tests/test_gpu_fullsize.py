@@ -258,16 +258,8 @@ WHOLE = {
 }
 
 
-@pytest.mark.parametrize("width", ["7b", "1b"])
-def test_whole_batch_two_layers_every_request_matches_oracle(width):
-    """The 7B-class and 1B-class widths with two layers: EVERY request of full-budget steps against
-    the fp32 oracle, not a sample.  16 generation requests (their contexts written by the library:
-    prompts prefilled in chunks, FCFS under the budget) decode one teacher-forced row per step next
-    to a stream of embedding requests (lengths lognormal as in the configurations, chunked, every
-    third one mean-pooled, the others last-token) admitted FCFS until the budget is full; after three
-    full-budget steps nothing new is admitted and the steps continue until every embedding request
-    in flight has finished.  Compared: every logits row of every decode step of every generation
-    request, and every embedding."""
+def _run_whole_batch(width, block_limit=0):
+    """The GPU side of the whole-batch tests: returns (shape, W, gens, all_embs, got_lg, got_emb, steps, rows per mixed step)."""
     from conftest import cached_weights
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
@@ -279,61 +271,98 @@ def test_whole_batch_two_layers_every_request_matches_oracle(width):
     n_full, max_drain = 3, c["emb"][2] // chunk + 1
     max_pos = max(c["ctx"][1] + n_full + max_drain + 2, c["emb"][2] + 2)
     n_pages = c["n_decode"] * (max_pos // P + 2) + 6 * budget // P + 16 * (c["emb"][2] // P + 2)
-    eng = Engine(shape, dw, n_pages=n_pages, n_slots=128, max_tokens=budget, max_segs=c["n_decode"] + budget // 16 + 8,
-                 max_pos=max_pos, kv_fill=KV_SENTINEL)
-    gens = [Request("gen", synth.token_ids(rng, int(n), shape.V))
-            for n in rng.integers(c["ctx"][0], c["ctx"][1] + 1, size=c["n_decode"])]
-    got_lg = {g: [] for g in gens}
-    got_emb, all_embs = {}, []
+    B.attn_set_block_limit(block_limit)
+    try:
+        eng = Engine(shape, dw, n_pages=n_pages, n_slots=128, max_tokens=budget, max_segs=c["n_decode"] + budget // 16 + 8,
+                     max_pos=max_pos, kv_fill=KV_SENTINEL)
+        gens = [Request("gen", synth.token_ids(rng, int(n), shape.V))
+                for n in rng.integers(c["ctx"][0], c["ctx"][1] + 1, size=c["n_decode"])]
+        got_lg = {g: [] for g in gens}
+        got_emb, all_embs = {}, []
 
-    def run(work):
-        _, lrows, erows = eng.step(work)
-        torch.cuda.synchronize()
-        for r, row in lrows.items():
-            got_lg[r].append(eng.out_logits[row].cpu().numpy().astype(np.float64))
-        for r, row in erows.items():
-            got_emb[r] = eng.out_emb[row].cpu().numpy().astype(np.float64)
-            eng.release(r)
+        def run(work):
+            _, lrows, erows = eng.step(work)
+            torch.cuda.synchronize()
+            for r, row in lrows.items():
+                got_lg[r].append(eng.out_logits[row].cpu().numpy().astype(np.float64))
+            for r, row in erows.items():
+                got_emb[r] = eng.out_emb[row].cpu().numpy().astype(np.float64)
+                eng.release(r)
 
-    # contexts: prefill the prompts through the library, FCFS, full steps
-    while any(not g.in_decode for g in gens):
-        work, rows = [], 0
-        for g in gens:
-            if not g.in_decode and rows < budget:
-                q = min(chunk, g.remaining(), budget - rows)
-                work.append((g, q)); rows += q
-        run(work)
-    # mixed steps: 16 decode rows + embedding chunks up to the budget; then drain
-    inflight, step, n_mixed_rows = [], 0, []
-    while step < n_full or inflight:
-        assert step < n_full + max_drain + 1
-        work, rows = [], 0
-        for g in gens:
-            g.tokens.append(int(rng.integers(0, shape.V)))       # the token both sides are fed
-            work.append((g, 1)); rows += 1
-        nxt = []
-        for e in inflight:
-            q = min(chunk, e.remaining(), budget - rows)
-            if q > 0:
+        # contexts: prefill the prompts through the library, FCFS, full steps
+        while any(not g.in_decode for g in gens):
+            work, rows = [], 0
+            for g in gens:
+                if not g.in_decode and rows < budget:
+                    q = min(chunk, g.remaining(), budget - rows)
+                    work.append((g, q)); rows += q
+            run(work)
+        # mixed steps: 16 decode rows + embedding chunks up to the budget; then drain
+        inflight, step, n_mixed_rows = [], 0, []
+        while step < n_full or inflight:
+            assert step < n_full + max_drain + 1
+            work, rows = [], 0
+            for g in gens:
+                g.tokens.append(int(rng.integers(0, shape.V)))       # the token both sides are fed
+                work.append((g, 1)); rows += 1
+            nxt = []
+            for e in inflight:
+                q = min(chunk, e.remaining(), budget - rows)
+                if q > 0:
+                    work.append((e, q)); rows += q
+                if e.remaining() - q > 0:
+                    nxt.append(e)
+            while step < n_full and rows < budget:
+                n = int(synth.lognormal_lengths(rng, 1, *c["emb"])[0])
+                e = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_MEAN if len(all_embs) % 3 == 2 else B.POOL_LAST)
+                all_embs.append(e)
+                q = min(chunk, n, budget - rows)
                 work.append((e, q)); rows += q
-            if e.remaining() - q > 0:
-                nxt.append(e)
-        while step < n_full and rows < budget:
-            n = int(synth.lognormal_lengths(rng, 1, *c["emb"])[0])
-            e = Request("embed", synth.token_ids(rng, n, shape.V), B.POOL_MEAN if len(all_embs) % 3 == 2 else B.POOL_LAST)
-            all_embs.append(e)
-            q = min(chunk, n, budget - rows)
-            work.append((e, q)); rows += q
-            if q < n:
-                nxt.append(e)
-        inflight = nxt
-        if step < n_full:
-            assert rows == budget
-        n_mixed_rows.append(rows)
-        run(work)
-        step += 1
-    assert eng.ctx.status_poll() == 0
-    assert len(got_emb) == len(all_embs) and len(all_embs) >= 8
+                if q < n:
+                    nxt.append(e)
+            inflight = nxt
+            if step < n_full:
+                assert rows == budget
+            n_mixed_rows.append(rows)
+            run(work)
+            step += 1
+        assert eng.ctx.status_poll() == 0
+        assert len(got_emb) == len(all_embs) and len(all_embs) >= 8
+        eng.close()
+    finally:
+        B.attn_set_block_limit(0)
+    return shape, W, gens, all_embs, got_lg, got_emb, step, n_mixed_rows
+
+
+def test_whole_batch_at_7b_width_is_bitwise_the_same_with_37_attention_blocks():
+    """The full-budget steps of the next test (7B-class width, two layers: 16 decode rows with up to
+    four key splits, chunk tiles of up to 64 key tiles, short chunk tiles) with the attention launch
+    capped at 37 resident blocks instead of two per SM: every block then runs dozens of items of both
+    kinds one after the other.  Every logits row and every embedding must come out bit for bit the
+    same."""
+    _, _, gens_a, embs_a, lg_a, emb_a, steps_a, _ = _run_whole_batch("7b", 0)
+    _, _, gens_b, embs_b, lg_b, emb_b, steps_b, _ = _run_whole_batch("7b", 37)
+    assert steps_a == steps_b and len(embs_a) == len(embs_b)
+    for ga, gb in zip(gens_a, gens_b):
+        assert len(lg_a[ga]) == len(lg_b[gb])
+        for x, y in zip(lg_a[ga], lg_b[gb]):
+            assert np.array_equal(x, y)
+    for ea, eb in zip(embs_a, embs_b):
+        assert np.array_equal(emb_a[ea], emb_b[eb])
+
+
+@pytest.mark.parametrize("width", ["7b", "1b"])
+def test_whole_batch_two_layers_every_request_matches_oracle(width):
+    """The 7B-class and 1B-class widths with two layers: EVERY request of full-budget steps against
+    the fp32 oracle, not a sample.  16 generation requests (their contexts written by the library:
+    prompts prefilled in chunks, FCFS under the budget) decode one teacher-forced row per step next
+    to a stream of embedding requests (lengths lognormal as in the configurations, chunked, every
+    third one mean-pooled, the others last-token) admitted FCFS until the budget is full; after three
+    full-budget steps nothing new is admitted and the steps continue until every embedding request
+    in flight has finished.  Compared: every logits row of every decode step of every generation
+    request, and every embedding."""
+    from paper_2609_25405_b200 import binding as B
+    shape, W, gens, all_embs, got_lg, got_emb, step, n_mixed_rows = _run_whole_batch(width)
     # ---- oracle: one whole-sequence pass per request ----
     head = {B.POOL_LAST: "last", B.POOL_MEAN: "mean"}
     worst_l = worst_e = 0.0
@@ -364,4 +393,3 @@ def test_whole_batch_two_layers_every_request_matches_oracle(width):
           f"argmax agreement {n_agree}/{n_rows}; {len(all_embs)} embeddings: worst cosine {worst_cos:.6f}, "
           f"worst max-abs error {worst_e:.3e}")
     assert n_agree / n_rows >= 0.995, (n_agree, n_rows)
-    eng.close()
