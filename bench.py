@@ -588,6 +588,25 @@ def main():
                    "frac_of_burst": (ach_tf / peaks["bf16_tflops"]) if ach_tf else None,
                    "launches": gemm_n, "flops_per_launch": gemm_flops_launch,
                    "traffic": traffic, "traffic_from": traffic_note}
+    # the two attention item lists, each timed alone in the per-class pass (in the step they share one launch)
+    attention_kernels = {}
+    dec_ms, dec_n = prof.get("attention", (0.0, 0))
+    if dec_n and dec_ms > 0:
+        gbs = w["kv_read_bytes_decode"] * K / (dec_ms * 1e-3) / 1e9
+        attention_kernels["decode_items"] = {
+            "kernel": "attn_varlen_kernel, small items alone (decode splits over paged KV; chunk tiles of at most 64 rows)",
+            "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+            "bytes_per_launch": w["kv_read_bytes_decode"] * K / dec_n, "launches": dec_n,
+            "note": "algorithmic bytes: keys and values the decode rows read; events around every launch, "
+                    "~10 us of gap per launch included"}
+    tc_ms, tc_n = prof.get("attention_tc", (0.0, 0))
+    if tc_n and tc_ms > 0:
+        tf = w["attn_flops_chunk"] * K / (tc_ms * 1e-3) / 1e12
+        attention_kernels["chunk_tiles"] = {
+            "kernel": "attn_varlen_kernel, chunk tiles alone (tcgen05 body)", "bound": "tensor", "achieved": tf,
+            "unit": "TFLOP/s", "peak": peaks["bf16_tflops"], "frac": tf / peaks["bf16_tflops"],
+            "flops_per_launch": w["attn_flops_chunk"] * K / tc_n, "launches": tc_n,
+            "note": "4 Dh flop per visible (query, key, head) triple, chunk rows of all lengths; against the burst peak"}
     # The headline fraction is the STEP's: the whole mixed step against the slower of its GEMM flop at
     # the measured bf16 burst peak and its weight + KV bytes at the measured HBM rate.
     if step_roof["bound"] == "tensor":
@@ -599,7 +618,7 @@ def main():
                 "peak_kind": f"{peak_kind}: cuBLAS bf16 burst / copy bandwidth (the conservative denominators; "
                              f"against the sustained cuBLAS rate the step is at {step_roof['frac_of_sustained_roof']:.3f})",
                 "traffic_scope": "mean DRAM bytes per projection-GEMM launch (profiler capture), see gemm_kernel",
-                "gemm_kernel": gemm_kernel}
+                "gemm_kernel": gemm_kernel, "attention_kernels": attention_kernels}
     breakdown = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in prof.items()}
     line = {"metric": METRIC, "value": m["tokens"] / (m["ms"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",

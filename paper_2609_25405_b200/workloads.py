@@ -166,12 +166,20 @@ def step_work(shape, entries):
     gemm = 2.0 * s.L * per_layer * T + 2.0 * s.d * s.V * n_logit
     pairs = 0
     kv_tok_read = 0
+    pairs_chunk = 0          # (query, key) pairs of chunk rows: the tensor-bound share of attention
+    kv_tok_read_decode = 0   # keys decode rows read: the HBM-bound share
     for e in entries:
         q, p0 = len(e["tokens"]), e["pos_start"]
         pairs += q * p0 + q * (q + 1) // 2
         kv_tok_read += p0 + q
+        if e["kind"] == B.KIND_DECODE:
+            kv_tok_read_decode += p0 + q
+        else:
+            pairs_chunk += q * p0 + q * (q + 1) // 2
     attn = 4.0 * s.Dh * s.Hq * s.L * pairs
     kv_tok = s.L * 2 * s.Hkv * s.Dh * 2
     w_bytes = 2.0 * (s.L * per_layer + (s.d * s.V if n_logit else 0)) + 2.0 * s.d * T
     return dict(T=T, n_logit=n_logit, gemm_flops=gemm, attn_flops=attn, weight_bytes=w_bytes,
-                kv_read_bytes=float(kv_tok) * kv_tok_read, kv_write_bytes=float(kv_tok) * T)
+                kv_read_bytes=float(kv_tok) * kv_tok_read, kv_write_bytes=float(kv_tok) * T,
+                attn_flops_chunk=4.0 * s.Dh * s.Hq * s.L * pairs_chunk,
+                kv_read_bytes_decode=float(kv_tok) * kv_tok_read_decode)
