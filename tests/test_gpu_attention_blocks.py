@@ -26,10 +26,11 @@ CONTEXTS = (130, 700, 1535, 2559)      # decode rows over 1, 1, 2 and 3 splits o
 EMBED_LEN = (300, 77)                  # two embedding requests: chunks of 200 + 100 (a 128-row tile and a remainder) and 77
 
 
-def _run(shape, dw, limit):
+def _run(shape, dw, limit, contexts=CONTEXTS, embed_len=EMBED_LEN, embed_chunks=((200, 77), (100, 0)), seed=99):
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
-    rng = np.random.default_rng(99)
+    rng = np.random.default_rng(seed)
+    CONTEXTS, EMBED_LEN = contexts, embed_len
     P = shape.page_size
     n_pages = sum((c + 2 + P - 1) // P for c in CONTEXTS) + sum((n + P - 1) // P for n in EMBED_LEN) + 4
     outs = []
@@ -46,7 +47,7 @@ def _run(shape, dw, limit):
             torch.cuda.synchronize()
             outs.extend(eng.out_logits[lrows[g]].clone() for g in gens if g in lrows)
         # two mixed steps: every decode row + one embedding chunk each
-        for s, chunks in enumerate(((200, 77), (100, 0))):
+        for s, chunks in enumerate(embed_chunks):
             work = []
             for g, f in zip(gens, forced):
                 g.tokens.append(f[s])
@@ -76,6 +77,26 @@ def test_outputs_do_not_depend_on_the_number_of_resident_blocks(name):
         assert len(got) == len(ref)
         for i, (a, b) in enumerate(zip(got, ref)):
             assert torch.equal(a, b), (name, limit, i)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4, 5, 6])
+def test_random_mixes_with_one_and_seven_blocks(seed):
+    """Random contexts (1 to 4 key splits), random embedding lengths and chunkings on the tiny shape:
+    one block, seven blocks and the uncapped launch agree bit for bit."""
+    from paper_2609_25405_b200 import binding as B
+    shape = SHAPES["tiny"]
+    dw = B.DeviceWeights.from_synth(synth.Weights(shape, 0))
+    rng = np.random.default_rng(1000 + seed)
+    contexts = tuple(int(c) for c in rng.integers(17, 3600, size=int(rng.integers(2, 6))))
+    embed_len = tuple(int(n) for n in rng.integers(20, 500, size=2))
+    first = tuple(int(rng.integers(1, n)) for n in embed_len)
+    chunks = (first, tuple(n - f for n, f in zip(embed_len, first)))
+    ref = _run(shape, dw, 0, contexts, embed_len, chunks, seed)
+    for limit in (1, 7):
+        got = _run(shape, dw, limit, contexts, embed_len, chunks, seed)
+        assert len(got) == len(ref)
+        for i, (a, b) in enumerate(zip(got, ref)):
+            assert torch.equal(a, b), (seed, limit, i, contexts, embed_len, chunks)
 
 
 def test_block_limit_rejects_negative_values():
