@@ -1,7 +1,8 @@
 // The step's attention kernel: one launch per layer serves every row of the mixed batch (Section 3.2
 // of the paper: decode tokens attend over their cached context, embedding / prefill chunks attend
 // causally over their own earlier chunks plus themselves).  The host turns the batch descriptor
-// into two cost-sorted item lists; a block of the grid takes one item:
+// into two cost-sorted item lists; the blocks of the grid stay resident and take one item after the
+// other:
 //   chunk items of 65-128 query rows     -> tcgen05 body (attention_tc.cuh): tensor-bound
 //   decode items, chunk items <= 64 rows -> mma.sync body (attention_dec.cuh): HBM-bound
 // Both bodies run with the same block size and register budget (two blocks per SM); shared memory
