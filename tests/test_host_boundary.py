@@ -205,3 +205,24 @@ def test_misaligned_pointers_and_bad_tuning_arguments_are_refused_on_the_host():
     assert B.lib.hb_gemm_set_walk(-1, -1) == 0
     assert B.lib.hb_gemm_set_cta_limit(7) == -1 and B.lib.hb_gemm_set_cta_limit(-2) == -1
     assert B.lib.hb_gemm_set_cta_limit(0) == 0
+    assert B.lib.hb_attn_set_block_limit(-1) == -1 and B.lib.hb_attn_set_block_limit(0) == 0
+
+
+def test_step_work_splits_attention_by_row_kind():
+    """The work counts that the bench divides by measured times: a decode row reads its context plus
+    itself, a chunk row of length q over p earlier tokens sees q p + q (q + 1) / 2 (query, key) pairs;
+    the per-kind figures add up to the totals."""
+    from paper_2609_25405_b200 import synth, workloads
+    s = synth.SHAPES["tiny"]
+    ent = [dict(kind=B.KIND_DECODE, tokens=[1], pos_start=10, is_final=True),
+           dict(kind=B.KIND_EMBED_CHUNK, tokens=[1, 2, 3], pos_start=4, is_final=False),
+           dict(kind=B.KIND_PREFILL_CHUNK, tokens=[5, 6], pos_start=0, is_final=True)]
+    w = workloads.step_work(s, ent)
+    kv_tok = s.L * 2 * s.Hkv * s.Dh * 2
+    per_pair = 4.0 * s.Dh * s.Hq * s.L
+    assert w["T"] == 6 and w["n_logit"] == 2
+    assert w["kv_read_bytes_decode"] == kv_tok * 11
+    assert w["kv_read_bytes"] == kv_tok * (11 + 7 + 2)
+    assert w["attn_flops_chunk"] == per_pair * ((3 * 4 + 6) + (0 + 3))
+    assert w["attn_flops"] == per_pair * (11 + (3 * 4 + 6) + 3)
+    assert w["kv_write_bytes"] == kv_tok * 6
