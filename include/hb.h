@@ -393,6 +393,16 @@ HB_API int hb_gemm_set_cta_limit(int32_t max_ctas);
  * changes a result bit (an item's arithmetic is its own; the splits of a decode row are merged in
  * split order by whichever block arrives last).  Host only, not thread-safe against launches. */
 HB_API int hb_attn_set_block_limit(int32_t max_blocks);
+/* Keys per decode attention item.  A decode row with n = context + 1 keys is cut into
+ * max(1, (n + keys / 2) div keys) equal splits (rounded up to whole 64-key tiles) that different blocks
+ * may run; their partial results are merged in split order.  The count depends on the row's own context
+ * and on this value only, never on the rest of the batch, so a request's result does not depend on its
+ * batch; it does depend on this value (another summation order: results differ in the last bits).
+ * Default 2048 (keys = 0 restores it); multiples of 64 from 256 to 65536.  A smaller value keeps more
+ * blocks busy when steps hold only a few long decode rows, at the cost of a partial record, a fence, an
+ * atomic and a share of the merge per split.  Process-wide; hb_workspace_bytes and hb_create read it,
+ * and a context keeps the value it was created with.  Host only. */
+HB_API int hb_attn_set_split_keys(int32_t keys);
 
 /* The incremental pooler on its own (Section 3.3, Eq. 1-2 and the last-token
  * head), as hb_mixed_step runs it on an embedding segment: final RMSNorm of

@@ -108,6 +108,7 @@ _sig = {
     "hb_gemm_set_walk": [C.c_int32, C.c_int32],
     "hb_gemm_set_cta_limit": [C.c_int32],
     "hb_attn_set_block_limit": [C.c_int32],
+    "hb_attn_set_split_keys": [C.c_int32],
 }
 for _name, _args in _sig.items():
     _f = getattr(lib, _name)
@@ -592,6 +593,11 @@ def gemm_set_cta_limit(max_ctas=0):
 def attn_set_block_limit(max_blocks=0):
     """Cap the resident blocks of every attention launch (tests); 0 = two per SM."""
     check(lib.hb_attn_set_block_limit(max_blocks), "hb_attn_set_block_limit")
+
+
+def attn_set_split_keys(keys=0):
+    """Keys per decode attention item for contexts created from now on; 0 = the default (2048)."""
+    check(lib.hb_attn_set_split_keys(keys), "hb_attn_set_split_keys")
 
 
 def validate_desc(cfg, max_tokens, max_segs, max_page_ids, n_pages, n_slots, batch):

@@ -14,7 +14,13 @@ namespace {
 constexpr int POOL_ROWS = 32;   // rows per pooling work item
 constexpr int ATT_TILE_ROWS = 64;   // query rows (tokens x grouped heads) per small chunk attention item
 constexpr int ATT_TC_ROWS = 128;    // query rows per tcgen05 chunk attention item
-constexpr int ATT_SPLIT_KEYS = 1024; // keys per decode attention item; depends on nothing but this constant
+// Keys per decode attention item (a row's keys are cut into about this many per split; the count depends
+// on the row's own context and this value only).  A split costs a partial record, a fence, an atomic and
+// a share of the merge: with the attention blocks resident and the chunk tiles filling the tail of the
+// launch, 2048 measured 6 % faster than 1024 on the decode items of the 7B mixed step and 8-12 % faster
+// per step on the sweep's mixes (contexts of 2048: no split at all); 1024 keeps more blocks busy when a
+// step holds only a few long decode rows.  Process-wide, read when a context is created.
+int g_att_split_keys = 2048;
 constexpr int N_STAGING = 4;    // pinned descriptor staging ring
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -50,6 +56,7 @@ struct Layout {
       status, desc;
   size_t total, desc_cap, attn_part_floats, pool_part_floats;
   int32_t rows_pad, logit_rows_pad, n_counters, max_pool_items, max_attn_items, n_resid_turns;
+  int32_t split_keys;   // keys per decode attention item of this context
 };
 
 Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, int32_t max_page_ids) {
@@ -76,7 +83,8 @@ Layout make_layout(const hb_model_cfg& c, int32_t max_tokens, int32_t max_segs, 
   L.rope_sin = cv.take(static_cast<size_t>(c.max_pos) * (c.head_dim / 2) * 4);
   L.max_pool_items = max_tokens / POOL_ROWS + max_segs + 1;
   const int G = c.n_heads / c.n_kv_heads;
-  const int max_splits = (c.max_pos + ATT_SPLIT_KEYS - 1) / ATT_SPLIT_KEYS;
+  L.split_keys = g_att_split_keys;
+  const int max_splits = (c.max_pos + L.split_keys - 1) / L.split_keys;
   L.max_attn_items = c.n_kv_heads * (max_tokens * G / ATT_TILE_ROWS + max_segs + max_segs * max_splits);
   L.attn_part_floats = static_cast<size_t>(max_segs) * c.n_kv_heads * max_splits * G * (c.head_dim + 2);
   L.pool_part_floats = static_cast<size_t>(L.max_pool_items) * c.d_model;
@@ -617,7 +625,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
   }
   if (static_cast<int32_t>(pitems.size()) > ex->lay.max_pool_items) return HB_ERR_TOO_LARGE;
   // attention work list: chunk items (64 query rows x all visible keys) and decode items (one
-  // split of ATT_SPLIT_KEYS keys); sorted by cost, largest first, so the tail of the launch is short
+  // split of about split_keys keys); sorted by cost, largest first, so the tail of the launch is short
   std::vector<AttnItem>& aitems = ex->aitems;
   std::vector<AttnItem>& titems = ex->titems;
   aitems.clear();
@@ -630,8 +638,9 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
       for (int32_t hk = 0; hk < cfg.n_kv_heads; ++hk) {
         if (sg.kind == HB_KIND_DECODE) {
           const int32_t n_keys = sg.pos_start + 1;
-          // about ATT_SPLIT_KEYS keys per split, equal parts rounded up to whole 64-key tiles
-          const int32_t ns0 = std::max(1, (n_keys + ATT_SPLIT_KEYS / 2) / ATT_SPLIT_KEYS);
+          // about split_keys keys per split, equal parts rounded up to whole 64-key tiles
+          const int32_t split_keys = ex->lay.split_keys;
+          const int32_t ns0 = std::max(1, (n_keys + split_keys / 2) / split_keys);
           const int32_t per = ((n_keys + ns0 - 1) / ns0 + 63) / 64 * 64;
           const int32_t ns = (n_keys + per - 1) / per;
           for (int32_t sp = 0; sp < ns; ++sp) {
@@ -993,6 +1002,13 @@ int hb_gemm_set_walk(int32_t band, int32_t hints) {
 int hb_gemm_set_cta_limit(int32_t max_ctas) {
   if (max_ctas < 0 || (max_ctas & 1)) return HB_ERR_BAD_ARG;
   hb_gemm_cta_limit(max_ctas);
+  return HB_OK;
+}
+
+int hb_attn_set_split_keys(int32_t keys) {
+  if (keys == 0) keys = 2048;
+  if (keys < 256 || keys > 65536 || (keys & 63)) return HB_ERR_BAD_ARG;
+  g_att_split_keys = keys;
   return HB_OK;
 }
 

@@ -5,10 +5,13 @@ configuration), and two more group sizes (eight heads x 64 on one KV head; four 
 through hb_mixed_step in chunks of 512, so chunk rows with more than 1024 earlier tokens are
 compared too), then every request decodes one row.
 
-The host splits a decode row's keys into about 1024-key pieces: with n = context + 1 keys the count
-is max(1, (n + 512) div 1024), so contexts 1534 | 1535, 2558 | 2559 and 3582 | 3583 lie on the two
-sides of the boundaries between 1, 2, 3 and 4 pieces; 4096 (the longest context of the
-configurations) gives 4 and 4607 gives 5.
+The host splits a decode row's keys into pieces of about S keys (S = 2048 unless
+hb_attn_set_split_keys says otherwise): with n = context + 1 keys the count is
+max(1, (n + S / 2) div S).  With S = 1024 the contexts 1534 | 1535, 2558 | 2559 and 3582 | 3583 lie
+on the two sides of the boundaries between 1, 2, 3 and 4 pieces, 4096 gives 4 and 4607 gives 5 (all
+four shapes); with the default S = 2048 the contexts 3070 | 3071 and 5118 | 5119 lie on the two sides
+of the boundaries between 1, 2 and 3 pieces and 4096 (the longest context of the configurations)
+gives 2 (two shapes).
 
 Also here: the tiny mixed workload over 16 more workload seeds, for an argmax-agreement figure over
 a few hundred logits rows, with the oracle's top-1 / top-2 logit gap printed for every row whose
@@ -23,8 +26,11 @@ from paper_2609_25405_b200 import synth
 pytestmark = pytest.mark.gpu
 
 LOGIT_ABS, ARGMAX_RATE = 5e-2, 0.995
-CONTEXTS = (511, 1534, 1535, 2558, 2559, 3582, 3583, 4096, 4607)
-N_SPLITS = (1, 1, 2, 2, 3, 3, 4, 4, 5)
+# split size -> (contexts, pieces the host's rule gives them)
+CASES = {
+    1024: ((511, 1534, 1535, 2558, 2559, 3582, 3583, 4096, 4607), (1, 1, 2, 2, 3, 3, 4, 4, 5)),
+    2048: ((511, 3070, 3071, 4096, 5118, 5119), (1, 1, 2, 2, 2, 3)),
+}
 
 SHAPES = {
     "tiny": synth.SHAPES["tiny"],
@@ -37,16 +43,27 @@ SHAPES = {
 
 
 def test_split_rule_of_the_chosen_contexts():
-    """The contexts above do produce 1, 1, 2, 2, 3, 3, 4, 4, 5 pieces under the host's rule."""
-    for ctx, want in zip(CONTEXTS, N_SPLITS):
-        n = ctx + 1
-        ns0 = max(1, (n + 512) // 1024)
-        per = ((n + ns0 - 1) // ns0 + 63) // 64 * 64
-        assert (n + per - 1) // per == want, (ctx, want)
+    """The contexts above do produce the stated numbers of pieces under the host's rule."""
+    for S, (contexts, pieces) in CASES.items():
+        for ctx, want in zip(contexts, pieces):
+            n = ctx + 1
+            ns0 = max(1, (n + S // 2) // S)
+            per = ((n + ns0 - 1) // ns0 + 63) // 64 * 64
+            assert (n + per - 1) // per == want, (S, ctx, want)
 
 
-@pytest.mark.parametrize("name", ["tiny", "dh128", "g8", "g2dh128"])
-def test_decode_rows_at_every_split_count_match_oracle(name):
+@pytest.mark.parametrize("name,split_keys", [("tiny", 1024), ("dh128", 1024), ("g8", 1024), ("g2dh128", 1024),
+                                             ("tiny", 2048), ("dh128", 2048)])
+def test_decode_rows_at_every_split_count_match_oracle(name, split_keys):
+    from paper_2609_25405_b200 import binding as B
+    B.attn_set_split_keys(split_keys)        # read when the engines below create their contexts
+    try:
+        _decode_rows_case(name, CASES[split_keys][0])
+    finally:
+        B.attn_set_split_keys(0)
+
+
+def _decode_rows_case(name, CONTEXTS):
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200.engine import Engine, Request
     shape = SHAPES[name]

@@ -206,6 +206,9 @@ def test_misaligned_pointers_and_bad_tuning_arguments_are_refused_on_the_host():
     assert B.lib.hb_gemm_set_cta_limit(7) == -1 and B.lib.hb_gemm_set_cta_limit(-2) == -1
     assert B.lib.hb_gemm_set_cta_limit(0) == 0
     assert B.lib.hb_attn_set_block_limit(-1) == -1 and B.lib.hb_attn_set_block_limit(0) == 0
+    assert B.lib.hb_attn_set_split_keys(100) == -1 and B.lib.hb_attn_set_split_keys(1000) == -1   # too small; not a multiple of 64
+    assert B.lib.hb_attn_set_split_keys(131072) == -1
+    assert B.lib.hb_attn_set_split_keys(1024) == 0 and B.lib.hb_attn_set_split_keys(0) == 0        # 0 restores the default
 
 
 def test_step_work_splits_attention_by_row_kind():
