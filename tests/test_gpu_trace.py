@@ -73,25 +73,30 @@ def test_phase_workload_tiny():
 
 
 def test_trace_prefix_on_the_1b_shape_every_output_matches_oracle():
-    """Configuration 5 on its own shape: the first three sessions of the seed-1005 trace (3-5 rounds
+    """Configuration 5 on its own shape: the first eight sessions of the seed-1005 trace (3-5 rounds
     each of an embedding request and a generation request with a 512-2048-token prompt and 32-128
     greedy decode steps) replayed on the full 1B-class model through the scheduler and the engine.
     EVERY embedding and EVERY logits row of those sessions is compared with the fp32 oracle: the
     oracle runs one whole-sequence pass per request over the prompt plus the tokens the device chose
     (teacher-forced on the device's own greedy tokens, so one differing argmax does not spoil the
-    rows after it).  Bookkeeping over a whole trace is checked on the tiny shape above."""
+    rows after it).  Eight sessions give about 2800 logits rows: at this shape (vocabulary 128256,
+    logits errors of about 1e-2) roughly 0.3 % of the rows are near-ties of the oracle that the fp16
+    path decides the other way, and the 99.5 % criterion needs a sample in which that rate shows
+    (three sessions, about 1000 rows, gave 3 to 5 such rows depending on the rounding order of the
+    attention merge: either side of the limit).  Bookkeeping over a whole trace is checked on the tiny
+    shape above."""
     from conftest import cached_weights
     from paper_2609_25405_b200 import binding as B
     from paper_2609_25405_b200 import trace
     from paper_2609_25405_b200.engine import Engine
     shape = synth.SHAPES["1b"]
     W, dw = cached_weights(shape)
-    sessions = trace.make_trace(shape.V, seed=1005, n_sessions=256)[:3]
+    sessions = trace.make_trace(shape.V, seed=1005, n_sessions=256)[:8]
     budget, chunk = 4096, 256
     max_pos = 2048 + 128 + 8
     P = shape.page_size
-    n_pages = 3 * ((max_pos + P - 1) // P) + 64
-    eng = Engine(shape, dw, n_pages=n_pages, n_slots=8, max_tokens=budget, max_segs=3 + budget // 16 + 8, max_pos=max_pos)
+    n_pages = 8 * ((max_pos + P - 1) // P) + 64
+    eng = Engine(shape, dw, n_pages=n_pages, n_slots=8, max_tokens=budget, max_segs=8 + budget // 16 + 8, max_pos=max_pos)
     got_emb, got_tok = {}, {}
 
     def on_emb(si, ri, vec):
@@ -102,7 +107,7 @@ def test_trace_prefix_on_the_1b_shape_every_output_matches_oracle():
 
     out = trace.replay(sessions, eng, budget, chunk, pool_mode=B.POOL_LAST, on_embedding=on_emb, on_token=on_tok)
     assert eng.ctx.status_poll() == 0
-    assert out["sessions_done"] == 3 and out["rows"] == trace.trace_tokens(sessions)
+    assert out["sessions_done"] == 8 and out["rows"] == trace.trace_tokens(sessions)
     assert out["free_pages"] == n_pages
     n_rows = n_agree = n_embs = 0
     worst_l = worst_e = 0.0
