@@ -1,15 +1,12 @@
-// Attention over the paged KV cache for decode rows and for chunk tiles of at most 64 rows
-// (Section 3.2 of the paper: decode tokens attend over their cached context, embedding / prefill
-// chunks attend causally over their own earlier chunks plus themselves).  Row j of a segment has
-// position pos = pos_start + j and sees keys 0 .. pos of its own request; all keys, the row's own
-// included, are read from the pages (the projection's epilogue appended them before).
+// Attention over the paged KV cache for decode rows (Section 3.2 of the paper: decode tokens attend
+// over their cached context).  A decode row at position pos sees keys 0 .. pos of its own request; all
+// keys, the row's own included, are read from the pages (the projection's epilogue appended them
+// before).  Chunk rows take the tcgen05 body (attention_tc.cuh), whatever the size of their tile: a
+// 64-row remainder costs that body less per key tile than it cost this one.
 //
 // Work items come from the batch descriptor (host-built list):
-//   chunk item   at most 64 query rows = (64 / G) tokens x G query heads of one KV head
-//                (G = Hq / Hkv), all visible keys; the four compute warps own 16 rows each and
-//                share the K/V tiles.
-//   decode item  the G query heads of one KV head of one decode row over one split of at most
-//                SPLIT keys; the four warps share the rows and own 16 keys of every 64-key tile;
+//   decode item  the G query heads of one KV head (G = Hq / Hkv) of one decode row over one split of
+//                its keys; the four warps share the rows and own 16 keys of every 64-key tile;
 //                their partial (max, sum, output) are merged in shared memory, and the splits
 //                of a row through a scratch record per split, merged in split order by the CTA
 //                that arrives last (integer arrival counter; no floating-point atomics).
@@ -191,7 +188,10 @@ __device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const At
   const AttnItem it = p.items[item];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = p.G, Hq = p.Hq;
-  const bool decode = (it.mode != 0);
+  if (it.mode == 0) {   // chunk tiles all go to the tcgen05 body; the host never lists one here
+    if (tid == 0) atomicOr(p.status, HB_DEV_ATTN_BAD_INDEX);
+    return false;
+  }
   const int hk = it.kv_head;
 
   const int n_tiles = (it.key1 - it.key0 + TILE_KEYS - 1) / TILE_KEYS;
@@ -268,8 +268,8 @@ __device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const At
     bad |= (pg < 0 || pg >= p.kv.n_pages);
     pg_s[i] = pg;
   }
-  // ---- Q tile -> shared memory (rows past n_rows are zero) ----
-  for (int u = tid; u < TILE_ROWS * CH; u += ATT_THREADS) {
+  // ---- Q rows -> shared memory: the 16 rows of the one MMA row tile (rows past n_rows are zero) ----
+  for (int u = tid; u < 16 * CH; u += ATT_THREADS) {
     const int rr = u / CH, c = u - rr * CH;
     const int r = it.row0 + rr;
     const bool valid = rr < it.n_rows;
@@ -288,18 +288,12 @@ __device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const At
     return false;
   }
 
-  // rows of this thread: chunk items: warp-private rows; decode items: rows 0..15 for every warp
-  const int row_base = decode ? 0 : warp * 16;
+  // rows of this thread: rows 0..15 of the tile for every warp (the G heads of the decode row first)
+  constexpr int row_base = 0;
   const int ra = row_base + (lane >> 2), rb = ra + 8;
   // position of the rows (rows past n_rows get -1: nothing visible)
   const int pos_a = (ra < it.n_rows) ? it.pos_start + (it.row0 + ra) / G : -1;
   const int pos_b = (rb < it.n_rows) ? it.pos_start + (it.row0 + rb) / G : -1;
-  // last position any row of this warp can see (skip tiles past it)
-  int warp_last = -1;
-  {
-    const int last_row = min(row_base + 15, it.n_rows - 1);
-    if (last_row >= row_base) warp_last = it.pos_start + (it.row0 + last_row) / G;
-  }
 
   uint32_t qf[DH / 16][4];
   float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.0f, 0.0f};
@@ -340,15 +334,9 @@ __device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const At
       }
       __syncthreads();
     }
-    if (!compute) {
-      // the TMA warp has nothing to compute
-    } else if (decode) {
-      if (key_base + warp * 16 < it.key1)
-        warp_attend<DH, 2>(qf, k_tile, warp * 16, key_base, it.key1, pos_a, pos_b, p.scale_log2, m, l, oacc);
-    } else {
-      if (key_base <= warp_last)
-        warp_attend<DH, 8>(qf, k_tile, 0, key_base, it.key1, pos_a, pos_b, p.scale_log2, m, l, oacc);
-    }
+    // (the TMA warp and the sixth warp have nothing to compute)
+    if (compute && key_base + warp * 16 < it.key1)
+      warp_attend<DH, 2>(qf, k_tile, warp * 16, key_base, it.key1, pos_a, pos_b, p.scale_log2, m, l, oacc);
   }
   if (__syncthreads_or(failed)) {
     if (prod) {
@@ -363,31 +351,6 @@ __device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const At
   for (int h = 0; h < 2; ++h) {
     l[h] += __shfl_xor_sync(0xffffffffu, l[h], 1);
     l[h] += __shfl_xor_sync(0xffffffffu, l[h], 2);
-  }
-
-  if (!decode) {
-    if (!compute) return true;
-    // ---- chunk item: normalise, stage the warp's 16 rows in shared memory, store 16-byte vectors ----
-    const float inv_a = (l[0] > 0.0f) ? 1.0f / l[0] : 0.0f, inv_b = (l[1] > 0.0f) ? 1.0f / l[1] : 0.0f;
-    uint8_t* stage = smem;  // the ring is idle now; this warp touches its own 16 rows of the first tile only
-#pragma unroll
-    for (int dn = 0; dn < DH / 8; ++dn) {
-      const uint32_t va = pack_half2(oacc[dn][0] * inv_a, oacc[dn][1] * inv_a);
-      const uint32_t vb = pack_half2(oacc[dn][2] * inv_b, oacc[dn][3] * inv_b);
-      *reinterpret_cast<uint32_t*>(stage + tile_off<DH>(ra, dn) + (lane & 3) * 4) = va;
-      *reinterpret_cast<uint32_t*>(stage + tile_off<DH>(rb, dn) + (lane & 3) * 4) = vb;
-    }
-    __syncwarp();
-    for (int u = lane; u < 16 * CH; u += 32) {
-      const int rr = row_base + u / CH, c = u % CH;
-      if (rr < it.n_rows) {
-        const int r = it.row0 + rr;
-        const int tok = it.q_start + r / G, head = hk * G + r % G;
-        const uint4 v = *reinterpret_cast<const uint4*>(stage + tile_off<DH>(rr, c));
-        *reinterpret_cast<uint4*>(p.out + (static_cast<size_t>(tok) * Hq + head) * DH + c * 8) = v;
-      }
-    }
-    return true;
   }
 
   // ---- decode item: merge the four warps' partials in shared memory ----
@@ -467,7 +430,7 @@ __device__ __forceinline__ bool small_item(const CUtensorMap* kv_map_p, const At
   return true;
 }
 
-// Parameters of the decode / small chunk items of one layer.
+// Parameters of the decode items of one layer.
 inline AttnParams make_params(hb_ctx* c, const KvGeom& kv, int layer) {
   AttnParams p;
   p.q = c->q;

@@ -12,7 +12,7 @@
 namespace {
 
 constexpr int POOL_ROWS = 32;   // rows per pooling work item
-constexpr int ATT_TILE_ROWS = 64;   // query rows (tokens x grouped heads) per small chunk attention item
+constexpr int ATT_TILE_ROWS = 64;   // sizing only: the item list is reserved for chunk tiles as short as this
 constexpr int ATT_TC_ROWS = 128;    // query rows per tcgen05 chunk attention item
 // Keys per decode attention item (a row's keys are cut into about this many per split; the count depends
 // on the row's own context and this value only).  A split costs a partial record, a fence, an atomic and
@@ -624,7 +624,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
     }
   }
   if (static_cast<int32_t>(pitems.size()) > ex->lay.max_pool_items) return HB_ERR_TOO_LARGE;
-  // attention work list: chunk items (64 query rows x all visible keys) and decode items (one
+  // attention work list: chunk tiles (up to 128 query rows x all visible keys) and decode items (one
   // split of about split_keys keys); sorted by cost, largest first, so the tail of the launch is short
   std::vector<AttnItem>& aitems = ex->aitems;
   std::vector<AttnItem>& titems = ex->titems;
@@ -654,8 +654,9 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
           }
           rec_at += ns;
         } else {
-          // chunk rows: full 128-row tiles (and a remainder above 64 rows) go to the tcgen05 kernel,
-          // a remainder of at most 64 rows to the mma.sync kernel
+          // chunk rows: tiles of up to 128 rows, all for the tcgen05 body (a short remainder tile costs
+          // it less per key tile than it cost the mma.sync body, and that body, left with decode items
+          // only, needs fewer registers)
           const int32_t rows = sg.q_len * G;
           for (int32_t row0 = 0; row0 < rows; row0 += ATT_TC_ROWS) {
             AttnItem it{};
@@ -664,8 +665,7 @@ int hb_mixed_step_lora(hb_ctx* c, const hb_batch_desc* d, const hb_weights* w, c
             it.key1 = sg.pos_start + (row0 + it.n_rows - 1) / G + 1;
             it.split = 0; it.n_splits = 1; it.part_base = 0; it.mode = 0;
             it.q_start = sg.q_start; it.pos_start = sg.pos_start; it.pt_start = sg.pt_start; it.pt_len = sg.pt_len;
-            if (it.n_rows <= ATT_TILE_ROWS) aitems.push_back(it);
-            else titems.push_back(it);
+            titems.push_back(it);
           }
         }
       }
