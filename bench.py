@@ -594,7 +594,7 @@ def main():
     if dec_n and dec_ms > 0:
         gbs = w["kv_read_bytes_decode"] * K / (dec_ms * 1e-3) / 1e9
         attention_kernels["decode_items"] = {
-            "kernel": "attn_varlen_kernel, small items alone (decode splits over paged KV; chunk tiles of at most 64 rows)",
+            "kernel": "attn_varlen_kernel, decode splits alone (mma.sync body over paged KV)",
             "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
             "bytes_per_launch": w["kv_read_bytes_decode"] * K / dec_n, "launches": dec_n,
             "note": "algorithmic bytes: keys and values the decode rows read; events around every launch, "

@@ -326,7 +326,7 @@ HB_API int hb_status_poll(hb_ctx* ctx, void* stream, uint32_t* out_code);
  * launch count of a step is higher than in normal operation.  Classes: */
 enum {
   HB_CLASS_GEMM = 0,      /* QKV, O, gate/up, down projections                          */
-  HB_CLASS_ATTENTION = 1, /* attention launch (when timed: decode splits, short chunk tiles) */
+  HB_CLASS_ATTENTION = 1, /* attention launch (when timed: the decode splits alone) */
   HB_CLASS_NORM_ROPE = 2, /* gather + RMSNorm, RMSNorm, RoPE + KV append                */
   HB_CLASS_POOL = 3,      /* final RMSNorm + pooler / logits-row preparation            */
   HB_CLASS_LM_HEAD = 4,   /* LM-head projection                                         */

@@ -3,8 +3,8 @@
 // causally over their own earlier chunks plus themselves).  The host turns the batch descriptor
 // into two cost-sorted item lists; the blocks of the grid stay resident and take one item after the
 // other:
-//   chunk items of 65-128 query rows     -> tcgen05 body (attention_tc.cuh): tensor-bound
-//   decode items, chunk items <= 64 rows -> mma.sync body (attention_dec.cuh): HBM-bound
+//   chunk tiles of up to 128 query rows -> tcgen05 body (attention_tc.cuh): tensor-bound
+//   decode items (one split of a row)   -> mma.sync body (attention_dec.cuh): HBM-bound
 // Both bodies run with the same block size and register budget (two blocks per SM); shared memory
 // is the larger of their needs.  A launch without chunk tiles runs an instantiation without the
 // tcgen05 body.

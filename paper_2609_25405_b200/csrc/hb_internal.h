@@ -65,8 +65,8 @@ struct DeviceDesc {
   const hb_seg* segs;       // [R]
   const int32_t* pages;     // [n_page_ids]
   const int32_t* logit_src; // [n_logit_rows] token row feeding logits row i
-  const AttnItem* attn_items;  // decode splits and small chunk tiles (mma.sync kernel)
-  const AttnItem* tc_items;    // 128-row chunk tiles (tcgen05 kernel)
+  const AttnItem* attn_items;  // decode splits (mma.sync body)
+  const AttnItem* tc_items;    // chunk tiles of up to 128 rows (tcgen05 body)
   const PoolItem* pool_items;
   int32_t T, R, n_logit, n_attn_items, n_tc_items, n_pool_items;
 };
@@ -202,8 +202,8 @@ int hb_launch_embed_norm(hb_ctx* c, const void* tok_emb, const void* gain, cudaS
 int hb_launch_rmsnorm(hb_ctx* c, const void* gain, cudaStream_t s);
 // The step's attention launch of one layer.  `which` selects the item lists it serves (both in the
 // step itself; one at a time when launches are timed per class).
-constexpr int HB_ATTN_CHUNK_TILES = 1;   // chunk items of 65-128 rows (tcgen05 body)
-constexpr int HB_ATTN_SMALL_ITEMS = 2;   // decode items and chunk items of at most 64 rows (mma.sync body)
+constexpr int HB_ATTN_CHUNK_TILES = 1;   // chunk tiles of up to 128 rows (tcgen05 body)
+constexpr int HB_ATTN_SMALL_ITEMS = 2;   // decode items (mma.sync body)
 constexpr int HB_ATTN_ALL = 3;
 int hb_launch_attention(hb_ctx* c, const KvGeom& kv, const CUtensorMap& kv_map, int layer, cudaStream_t s, int which);
 int hb_launch_final(hb_ctx* c, const void* gain, float* pool_sum, uint32_t* pool_meta,

@@ -1,5 +1,5 @@
 """The attention launch runs resident blocks that take the step's attention items (decode splits,
-chunk tiles of 128 rows, short chunk tiles) from a ticket.  Which block runs an item, and how many
+chunk tiles of up to 128 rows) from a ticket.  Which block runs an item, and how many
 items a block runs one after the other, must not change a result bit: an item's arithmetic is its
 own, a block re-initialises its barriers and reuses its tensor memory between items, and the splits
 of a decode row are merged in split order by whichever block arrives last.

@@ -336,7 +336,7 @@ def _run_whole_batch(width, block_limit=0):
 
 def test_whole_batch_at_7b_width_is_bitwise_the_same_with_37_attention_blocks():
     """The full-budget steps of the next test (7B-class width, two layers: 16 decode rows with up to
-    two key splits, chunk tiles of up to 64 key tiles, short chunk tiles) with the attention launch
+    two key splits, chunk tiles of up to 64 key tiles, short remainder tiles) with the attention launch
     capped at 37 resident blocks instead of two per SM: every block then runs dozens of items of both
     kinds one after the other.  Every logits row and every embedding must come out bit for bit the
     same."""
